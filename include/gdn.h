@@ -1,0 +1,120 @@
+/*
+ * libgdn_b200 -- chunkwise-parallel training backward of the gated delta rule (GDN) linear recurrence
+ * for NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no framework types.
+ *
+ * The operation (paper Eq. 1 with one scalar gate triple per (token, head); Table 2 lists the family
+ * members as gate settings).  Per (sequence n, head h) chain with state h_t of shape d_k x d_v:
+ *
+ *     h_t = e^{g_t} h_{t-1} + k_t (w_t v_t - b_t (e^{g_t} h_{t-1})^T k_t)^T ,     o_t = scale * h_t^T q_t
+ *
+ * delta_rule = 1 is GDN (erase gate b_t = write gate w_t = beta_t); delta_rule = 0 is the scalar-gate
+ * linear recurrence h_t = e^{g_t} h_{t-1} + k_t v_t^T (b = 0, w = 1; beta is not read).
+ * The backward differentiates  L = sum_t <dO_t, o_t> + <dhT, h_T>  and follows Section 4.2: sequences
+ * are cut into chunks of 64 tokens; chunk-local WY/UT-transform factors T = (I + M)^-1 are rebuilt,
+ * per-chunk states are recomputed by a forward carry, dS is propagated by a reverse carry across
+ * chunks (the paper's K#1), and the intra-chunk gradients including the vector-Jacobian product of
+ * the triangular solve (the paper's K#2) are formed from T without re-inverting.
+ *
+ * Layout (row-major, innermost last).  "dev" = device pointer, "host" = host pointer.
+ *     q, k, dq, dk      dev [B, T, H, d_k]   element type desc->dtype
+ *     v, dO, o, dv      dev [B, T, H, d_v]   element type desc->dtype
+ *     g, beta, dg, dbeta dev [B, T, H]       float32
+ *     h0, hT, dhT, dh0  dev [N, H, d_k, d_v] float32 (state orientation d_k x d_v as in Eq. 1)
+ *     cu_seqlens        dev int32 [N + 1], cu[0] = 0, non-decreasing, cu[N] = T; requires B == 1.
+ *                       NULL means B independent sequences of T tokens each (then N must equal B).
+ * Every pointer must be 16-byte aligned.  States reset at sequence boundaries; a sequence whose length
+ * is not a multiple of 64 ends in a short chunk; an empty sequence passes dhT through to dh0.
+ *
+ * Ownership and execution.  The caller owns every buffer; the library allocates no device memory and
+ * frees nothing.  Inputs are never written.  Outputs are overwritten for every valid token.  All work
+ * is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL = default stream) and the
+ * calls return without synchronising; cu_seqlens is never read on the host.  The workspace is scratch
+ * owned by the caller; two calls may not share one workspace concurrently.
+ *
+ * Errors.  Argument errors are detected on the host before anything is launched and returned as a
+ * status; nothing is thrown, aborted or trapped.  Conditions only visible on the device (malformed
+ * cu_seqlens contents, a bounded device-side wait that ran out) are recorded in the workspace header
+ * and read back by gdn_last_device_status().  Non-finite inputs propagate into the outputs.
+ */
+#ifndef GDN_B200_H_
+#define GDN_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gdn_status {
+    GDN_OK = 0,
+    GDN_ERR_NULL_ARG = 1,
+    GDN_ERR_BAD_SHAPE = 2,          /* non-positive dims, N inconsistent with B / cu_seqlens           */
+    GDN_ERR_UNSUPPORTED_SHAPE = 3,  /* outside the envelope: chunk == 64, d_k, d_v in {64, 128}        */
+    GDN_ERR_MISALIGNED = 4,         /* a pointer is not 16-byte aligned                                */
+    GDN_ERR_BAD_SEQLENS = 5,        /* device-side: cu_seqlens not starting at 0 / decreasing / != T   */
+    GDN_ERR_WORKSPACE_TOO_SMALL = 6,
+    GDN_ERR_CUDA = 7,               /* a CUDA runtime call or launch failed                            */
+    GDN_ERR_DEVICE_TIMEOUT = 8      /* device-side: a bounded wait gave up                             */
+} gdn_status;
+
+typedef enum gdn_dtype { GDN_F32 = 0, GDN_BF16 = 1 } gdn_dtype;
+
+typedef struct gdn_desc {
+    int32_t B, T, H;      /* batch rows, tokens per row, heads                                          */
+    int32_t d_k, d_v;     /* head dims, each 64 or 128                                                  */
+    int32_t chunk;        /* must be 64 (Section 4.2)                                                   */
+    int32_t N;            /* number of sequences: B without cu_seqlens; with cu_seqlens B must be 1     */
+    int32_t dtype;        /* gdn_dtype of q, k, v, dO, o, dq, dk, dv. F32: fp32 FFMA arithmetic;        */
+                          /* BF16: bf16 operands with fp32 accumulation and fp32 carried states         */
+    float   scale;        /* o_t = scale * h_t^T q_t                                                    */
+    int32_t delta_rule;   /* 1: b = w = beta (GDN).  0: b = 0, w = 1, beta / dbeta ignored              */
+} gdn_desc;
+
+/* Bytes of workspace needed by gdn_fwd_recompute (*fwd_bytes) and by gdn_bwd (*bwd_bytes >= *fwd_bytes;
+ * the forward's workspace is a prefix of the backward's).  Either output pointer may be NULL. */
+gdn_status gdn_workspace_bytes(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
+
+/* Recompute stage of the backward (Section 4.2, "chunking"): chunk table, chunk-local cumulative decay,
+ * UT-transform factors T, W, U~ and the forward inter-chunk carry that leaves every chunk's incoming
+ * state in the workspace.  Optionally also emits the forward outputs:
+ *     o  dev [B,T,H,d_v] or NULL      hT dev [N,H,d_k,d_v] or NULL
+ * beta may be NULL iff delta_rule == 0; h0 NULL means zero. */
+gdn_status gdn_fwd_recompute(const gdn_desc* desc,
+                             const void* q, const void* k, const void* v,
+                             const float* g, const float* beta, const float* h0,
+                             const int32_t* cu_seqlens_dev,
+                             void* o, float* hT,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Full backward (Sections 4.1-4.2, Appendix A "the GDN backward's two hard stages").
+ *     dq, dk, dv   required outputs        dg      required, gradient w.r.t. the log-decay g
+ *     dbeta        required iff delta_rule dh0     optional (NULL: not written)
+ *     dhT          optional (NULL = zero)  h0      optional (NULL = zero)
+ * workspace_is_fresh_from_fwd != 0 asserts that `workspace` was filled by gdn_fwd_recompute with the same
+ * desc, q, k, v, g, beta, h0 and cu_seqlens and not touched since; the recompute stage is then skipped. */
+gdn_status gdn_bwd(const gdn_desc* desc,
+                   const void* q, const void* k, const void* v,
+                   const float* g, const float* beta, const float* h0,
+                   const void* dO, const float* dhT,
+                   const int32_t* cu_seqlens_dev,
+                   void* dq, void* dk, void* dv, float* dg, float* dbeta, float* dh0,
+                   void* workspace, size_t workspace_bytes, int32_t workspace_is_fresh_from_fwd,
+                   void* cuda_stream);
+
+/* Synchronises the stream, reads the device-side status word of the last call that used `workspace`
+ * and returns it (GDN_OK, GDN_ERR_BAD_SEQLENS or GDN_ERR_DEVICE_TIMEOUT; GDN_ERR_CUDA if the stream
+ * itself reports an error). */
+gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char* gdn_status_string(gdn_status s);
+
+/* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16"),
+ * or NULL for an unsupported descriptor.  Diagnostic only. */
+const char* gdn_kernel_path(const gdn_desc* desc);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GDN_B200_H_ */

@@ -1,0 +1,138 @@
+// Host side of the C ABI: argument validation, workspace layout, launch sequencing.
+#include <stdint.h>
+#include <string.h>
+
+#include "gdn_internal.cuh"
+
+namespace gdn {
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+enum class Path { None, SimtF32, SimtBf16, TcBf16 };
+
+Path pick_path(const gdn_desc& d) {
+    if (d.dtype == GDN_F32) return Path::SimtF32;
+    if (d.dtype == GDN_BF16) return Path::SimtBf16;
+    return Path::None;
+}
+
+gdn_status check_desc(const gdn_desc* d) {
+    if (!d) return GDN_ERR_NULL_ARG;
+    if (d->B <= 0 || d->T < 0 || d->H <= 0 || d->N <= 0 || d->d_k <= 0 || d->d_v <= 0) return GDN_ERR_BAD_SHAPE;
+    if ((long long)d->B * d->T > 0x7fffffffLL - 64 * 1024) return GDN_ERR_BAD_SHAPE;
+    if (d->chunk != kC) return GDN_ERR_UNSUPPORTED_SHAPE;
+    if (!((d->d_k == 64 || d->d_k == 128) && (d->d_v == 64 || d->d_v == 128))) return GDN_ERR_UNSUPPORTED_SHAPE;
+    if (d->dtype != GDN_F32 && d->dtype != GDN_BF16) return GDN_ERR_UNSUPPORTED_SHAPE;
+    if (d->delta_rule != 0 && d->delta_rule != 1) return GDN_ERR_BAD_SHAPE;
+    return GDN_OK;
+}
+
+WsLayout layout_for(const gdn_desc& d) {
+    // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
+    return make_layout(d, sizeof(float), simt_scratch_per_chunkhead(d));
+}
+
+// Sequences are described either by cu_seqlens (then B must be 1) or by B rows of T tokens (then N == B).
+gdn_status check_seq(const gdn_desc& d, const int32_t* cu) {
+    if (cu) { if (d.B != 1) return GDN_ERR_BAD_SHAPE; }
+    else if (d.N != d.B) return GDN_ERR_BAD_SHAPE;
+    return GDN_OK;
+}
+
+}  // namespace
+}  // namespace gdn
+
+using namespace gdn;
+
+extern "C" {
+
+gdn_status gdn_workspace_bytes(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    const WsLayout L = layout_for(*desc);
+    if (fwd_bytes) *fwd_bytes = L.fwd_end;
+    if (bwd_bytes) *bwd_bytes = L.total;
+    return GDN_OK;
+}
+
+gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g,
+                             const float* beta, const float* h0, const int32_t* cu, void* o, float* hT,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
+    if (!q || !k || !v || !g || !workspace) return GDN_ERR_NULL_ARG;
+    if (desc->delta_rule && !beta) return GDN_ERR_NULL_ARG;
+    const void* ptrs[] = {q, k, v, g, beta, h0, cu, o, hT, workspace};
+    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
+    Problem p{};
+    p.d = *desc;
+    p.Ttot = desc->B * desc->T;
+    p.L = layout_for(*desc);
+    if (workspace_bytes < p.L.fwd_end) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.h0 = h0; p.cu = cu; p.o = o; p.hT = hT;
+    p.ws = static_cast<char*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    return simt_launch_fwd(p, st) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
+                   const float* h0, const void* dO, const float* dhT, const int32_t* cu, void* dq, void* dk, void* dv,
+                   float* dg, float* dbeta, float* dh0, void* workspace, size_t workspace_bytes,
+                   int32_t workspace_is_fresh_from_fwd, void* cuda_stream) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
+    if (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg || !workspace) return GDN_ERR_NULL_ARG;
+    if (desc->delta_rule && (!beta || !dbeta)) return GDN_ERR_NULL_ARG;
+    const void* ptrs[] = {q, k, v, g, beta, h0, dO, dhT, cu, dq, dk, dv, dg, dbeta, dh0, workspace};
+    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
+    Problem p{};
+    p.d = *desc;
+    p.Ttot = desc->B * desc->T;
+    p.L = layout_for(*desc);
+    if (workspace_bytes < p.L.total) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.h0 = h0; p.dO = dO; p.dhT = dhT; p.cu = cu;
+    p.dq = dq; p.dk = dk; p.dv = dv; p.dg = dg; p.dbeta = dbeta; p.dh0 = dh0;
+    p.ws = static_cast<char*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    return simt_launch_bwd(p, workspace_is_fresh_from_fwd != 0, st) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream) {
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return GDN_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GDN_ERR_CUDA;
+    if (word == GDN_OK || word == GDN_ERR_BAD_SEQLENS || word == GDN_ERR_DEVICE_TIMEOUT) return (gdn_status)word;
+    return GDN_ERR_CUDA;
+}
+
+const char* gdn_status_string(gdn_status s) {
+    switch (s) {
+        case GDN_OK: return "ok";
+        case GDN_ERR_NULL_ARG: return "a required pointer is NULL";
+        case GDN_ERR_BAD_SHAPE: return "invalid shape or sequence description";
+        case GDN_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (chunk must be 64, d_k and d_v in {64,128}, dtype f32 or bf16)";
+        case GDN_ERR_MISALIGNED: return "a pointer is not 16-byte aligned";
+        case GDN_ERR_BAD_SEQLENS: return "cu_seqlens is malformed (must start at 0, be non-decreasing and end at T)";
+        case GDN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case GDN_ERR_CUDA: return "a CUDA call failed";
+        case GDN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    }
+    return "unknown status";
+}
+
+const char* gdn_kernel_path(const gdn_desc* desc) {
+    if (check_desc(desc) != GDN_OK) return nullptr;
+    switch (pick_path(*desc)) {
+        case Path::SimtF32: return "simt_f32";
+        case Path::SimtBf16: return "simt_bf16";
+        case Path::TcBf16: return "tcgen05_bf16";
+        default: return nullptr;
+    }
+}
+
+}  // extern "C"

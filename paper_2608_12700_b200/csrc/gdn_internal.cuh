@@ -1,0 +1,94 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "gdn.h"
+
+namespace gdn {
+
+constexpr int kC = 64;  // chunk length (Section 4.2: chunks of 64 steps)
+
+// Workspace header, first 256 bytes of the workspace.
+struct WsHeader {
+    int32_t status;    // device-side gdn_status (0 = ok)
+    int32_t n_chunks;  // chunks actually present (<= max_chunks)
+    int32_t detail;    // where a bounded wait gave up / offending sequence index
+    int32_t pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "header size");
+
+// Byte offsets of every workspace region.  Chunk-head index = chunk * H + head.
+struct WsLayout {
+    int max_chunks;        // bound on the number of chunks: sum over sequences of ceil(len/64) <= ceil(T_total/64) + N
+    size_t seq_first;      // int32 [N + 1]   first chunk index of each sequence
+    size_t chunk_seq;      // int32 [max_chunks]
+    size_t chunk_tok0;     // int32 [max_chunks]   global token index of the chunk's first row
+    size_t chunk_len;      // int32 [max_chunks]   valid rows (1..64)
+    size_t gamma;          // f32 [CH, 64]         chunk-local cumulative log decay
+    size_t Tm;             // f32|bf16 [CH, 64, 64]    T = (I + A)^-1
+    size_t W;              // [CH, 64, d_k]
+    size_t Ut;             // [CH, 64, d_v]            U~ = T Diag(w) V
+    size_t Nm;             // [CH, d_k, d_k]           Kb^T W
+    size_t Bf;             // [CH, d_k, d_v]           Kb^T U~
+    size_t hc;             // [CH, d_k, d_v]           state entering the chunk
+    size_t fwd_end;        // bytes needed by the forward recompute
+    size_t E;              // [CH, d_k, d_v]           scale (Gam Q - P W)^T dO
+    size_t dhn;            // [CH, d_k, d_v]           gradient w.r.t. the state leaving the chunk
+    size_t scratch;        // kernel-private staging, per chunk-head
+    size_t scratch_per_ch; // bytes of scratch per chunk-head
+    size_t total;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// elem = bytes per stored factor element (4 on the fp32 path).
+inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t scratch_per_ch) {
+    WsLayout L{};
+    const size_t Ttot = (size_t)d.B * (size_t)d.T;
+    L.max_chunks = (int)((Ttot + kC - 1) / kC + (size_t)d.N);
+    const size_t CH = (size_t)L.max_chunks * d.H;
+    size_t o = sizeof(WsHeader);
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    L.seq_first = take(4 * ((size_t)d.N + 1));
+    L.chunk_seq = take(4 * (size_t)L.max_chunks);
+    L.chunk_tok0 = take(4 * (size_t)L.max_chunks);
+    L.chunk_len = take(4 * (size_t)L.max_chunks);
+    L.gamma = take(4 * CH * kC);
+    L.Tm = take(elem * CH * kC * kC);
+    L.W = take(elem * CH * kC * d.d_k);
+    L.Ut = take(elem * CH * kC * d.d_v);
+    L.Nm = take(elem * CH * d.d_k * d.d_k);
+    L.Bf = take(elem * CH * d.d_k * d.d_v);
+    L.hc = take(elem * CH * d.d_k * d.d_v);
+    L.fwd_end = o;
+    L.E = take(elem * CH * d.d_k * d.d_v);
+    L.dhn = take(elem * CH * d.d_k * d.d_v);
+    L.scratch_per_ch = scratch_per_ch;
+    L.scratch = take(scratch_per_ch * CH);
+    L.total = o;
+    return L;
+}
+
+// Everything a kernel needs to know about one call.
+struct Problem {
+    gdn_desc d;
+    int Ttot;  // B * T
+    const void *q, *k, *v, *dO;
+    const float *g, *beta, *h0, *dhT;
+    const int32_t* cu;
+    void *o, *dq, *dk, *dv;
+    float *hT, *dg, *dbeta, *dh0;
+    char* ws;
+    WsLayout L;
+};
+
+// Kernel families (each defined in its own translation unit).  They enqueue on `st` and return the
+// first CUDA error seen.
+cudaError_t simt_launch_fwd(const Problem& p, cudaStream_t st);
+cudaError_t simt_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
+size_t simt_scratch_per_chunkhead(const gdn_desc& d);
+
+}  // namespace gdn

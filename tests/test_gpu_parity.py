@@ -1,0 +1,143 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU fp64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_12700_b200 import binding, runner, synth
+from helpers import TOL, check_against_oracle, oracle_grads, rel
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, **kw):
+    base = dict(dtype="f32", H=2, d_k=64, d_v=64, seed=100)
+    base.update(kw)
+    return synth.make_workload(name, **base)
+
+
+def test_config0_fp32():
+    wl = synth.config(0)
+    errs = check_against_oracle(wl, runner.backward(wl))
+    print("cfg0", errs)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("dk,dv", [(64, 64), (128, 128), (128, 64), (64, 128)])
+def test_shapes_with_states(dtype, dk, dv):
+    wl = small(f"shape_{dtype}_{dk}_{dv}", dtype=dtype, B=2, T=192, H=2, d_k=dk, d_v=dv, states=True, seed=7)
+    check_against_oracle(wl, runner.backward(wl))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_ragged_varlen_and_empty_sequence(dtype):
+    # lengths: a tail of 1, an exact multiple, an empty sequence, a sub-chunk sequence, a long ragged one
+    wl = small("ragged_" + dtype, dtype=dtype, lengths=[65, 128, 0, 37, 300], H=3, d_k=128, d_v=128,
+               states=True, seed=11)
+    got = runner.backward(wl)
+    check_against_oracle(wl, got)
+    # the empty sequence passes its terminal-state gradient straight through
+    assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_scalar_gate_recurrence_delta_rule_off(dtype):
+    wl = small("beta_off_" + dtype, dtype=dtype, B=2, T=200, H=2, d_k=64, d_v=64, delta_rule=0, g_scale=0.05,
+               seed=12)
+    check_against_oracle(wl, runner.backward(wl))
+
+
+def test_scale_argument():
+    wl = small("scaled", B=1, T=130, scale=0.125, states=True, seed=13)
+    check_against_oracle(wl, runner.backward(wl))
+
+
+def test_forward_outputs_match_oracle():
+    wl = small("fwd", lengths=[70, 130], H=2, d_k=64, d_v=128, states=True, seed=14)
+    buf = runner.to_device(wl, want_o=True)
+    runner.run_fwd(buf)
+    got = runner.fetch(buf)
+    ref = oracle_grads(wl)
+    assert rel(got["o"], ref["o"]) < 1e-4
+    assert rel(got["hT"], ref["hT"]) < 1e-4
+
+
+def test_fresh_workspace_reuse_gives_identical_gradients():
+    wl = small("fresh", B=1, T=256, H=2, states=True, seed=15)
+    a = runner.backward(wl)
+    buf = runner.to_device(wl, want_o=True)
+    runner.run_fwd(buf)
+    runner.run_bwd(buf, fresh=1)
+    b = runner.fetch(buf)
+    for n in ("dq", "dk", "dv", "dg", "dbeta", "dh0"):
+        assert np.array_equal(a[n], b[n]), n
+
+
+def test_bitwise_determinism_over_repeats():
+    wl = small("determinism", dtype="bf16", lengths=[100, 260], H=4, d_k=128, d_v=128, states=True, seed=16)
+    buf = runner.to_device(wl)
+    runner.run_bwd(buf)
+    first = {k: v.clone() for k, v in buf.outputs.items() if v is not None}
+    for _ in range(4):
+        for v in buf.outputs.values():
+            if v is not None:
+                v.fill_(float("nan"))
+        runner.run_bwd(buf)
+        torch.cuda.synchronize()
+        for k, v in first.items():
+            assert torch.equal(v.view(torch.uint8), buf.outputs[k].view(torch.uint8)), k
+
+
+def test_zero_upstream_gradient_gives_zero():
+    wl = small("zeros", B=1, T=128, states=True, seed=17)
+    wl.dO[:] = 0
+    wl.dhT[:] = 0
+    got = runner.backward(wl)
+    for n in ("dq", "dk", "dv", "dg", "dbeta", "dh0"):
+        assert not np.any(got[n]), n
+
+
+def test_inputs_are_not_modified_and_padding_is_not_written():
+    wl = small("readonly", lengths=[70], H=2, seed=18, states=True)
+    buf = runner.to_device(wl)
+    before = {k: v.clone() for k, v in buf.inputs.items() if v is not None}
+    runner.run_bwd(buf)
+    runner.fetch(buf)
+    for k, v in before.items():
+        assert torch.equal(v, buf.inputs[k]), k
+
+
+def test_nan_in_v_propagates_within_its_chain_only():
+    wl = small("nan", B=2, T=128, H=2, seed=19)
+    wl.v[70, 1, 3] = np.nan        # batch row 0, token 70, head 1
+    got = runner.backward(wl)
+    assert np.isnan(got["dk"][:128, 1]).any() and np.isnan(got["dbeta"][:128, 1]).any()
+    assert np.isfinite(got["dk"][:, 0]).all() and np.isfinite(got["dq"][:, 0]).all()   # other head
+    assert np.isfinite(got["dk"][128:]).all()                                          # other batch row
+
+
+def test_malformed_cu_seqlens_is_reported_not_faulted():
+    wl = small("badcu", lengths=[64, 64], H=1, seed=20)
+    buf = runner.to_device(wl)
+    buf.inputs["cu_seqlens"] = torch.tensor([0, 100, 64, 128][:3], dtype=torch.int32, device="cuda")  # decreasing
+    runner.run_bwd(buf)
+    assert binding.gdn_last_device_status(buf.workspace) == 5   # GDN_ERR_BAD_SEQLENS
+    buf.inputs["cu_seqlens"] = torch.tensor([0, 64, 120], dtype=torch.int32, device="cuda")           # does not end at T
+    runner.run_bwd(buf)
+    assert binding.gdn_last_device_status(buf.workspace) == 5
+    buf.inputs["cu_seqlens"] = torch.tensor([0, 64, 128], dtype=torch.int32, device="cuda")
+    runner.run_bwd(buf)
+    assert binding.gdn_last_device_status(buf.workspace) == 0
+
+
+# ---- the benchmark configurations at full size: sampled (sequence, head) chains against the oracle ----
+@pytest.mark.parametrize("idx,heads", [(1, [0, 9]), (2, [5]), (3, [3]), (4, [0, 31])])
+def test_full_size_configs_sampled_chains(idx, heads):
+    wl = synth.config(idx)
+    got = runner.backward(wl)
+    sub = wl.take_heads(heads)
+    ref = oracle_grads(sub)
+    got_sub = {n: (v[:, heads] if v.ndim >= 2 else v) for n, v in got.items()}
+    errs = check_against_oracle(sub, got_sub, ref=ref)
+    print(wl.name, errs)
+    for n, v in got.items():
+        assert np.isfinite(v).all(), n
