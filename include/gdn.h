@@ -114,6 +114,18 @@ const char* gdn_status_string(gdn_status s);
  * or NULL for an unsupported descriptor.  Diagnostic only. */
 const char* gdn_kernel_path(const gdn_desc* desc);
 
+/* ---- measurement hooks (not part of the method; the paper has no counterpart) -------------------
+ * gdn_launch_count: number of kernels this library has launched in this process.
+ * gdn_stage_timing_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events
+ * recorded on the launching stream (events are created lazily and reused; no device memory).
+ * gdn_stage_timing_read: synchronises the recorded events, adds up per-stage durations since the last
+ * read, writes up to max_stages entries (total_ms, launches, names: static strings) and resets the
+ * record.  Returns the number of stages through *n_stages.  Not thread-safe; diagnostic use only. */
+uint64_t gdn_launch_count(void);
+gdn_status gdn_stage_timing_enable(int32_t on);
+gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* launches, const char** names,
+                                 int32_t* n_stages);
+
 #ifdef __cplusplus
 }
 #endif

@@ -21,7 +21,8 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
                 7: "GDN_ERR_CUDA", 8: "GDN_ERR_DEVICE_TIMEOUT"}
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
-           "gdn_status_string", "gdn_kernel_path"]
+           "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
+           "gdn_stage_timing_read"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -62,6 +63,12 @@ def lib():
         L.gdn_status_string.argtypes = [I]
         L.gdn_kernel_path.restype = ctypes.c_char_p
         L.gdn_kernel_path.argtypes = [D]
+        L.gdn_launch_count.restype = ctypes.c_uint64
+        L.gdn_launch_count.argtypes = []
+        L.gdn_stage_timing_enable.restype = I
+        L.gdn_stage_timing_enable.argtypes = [I]
+        L.gdn_stage_timing_read.restype = I
+        L.gdn_stage_timing_read.argtypes = [I, P, P, P, P]
         _lib = L
     return _lib
 
@@ -130,3 +137,24 @@ def gdn_bwd(desc, q, k, v, g, beta, h0, dO, dhT, cu_seqlens, dq, dk, dv, dg, dbe
 
 def gdn_last_device_status(workspace, stream=None) -> int:
     return lib().gdn_last_device_status(_p(workspace), _stream(stream))
+
+
+def gdn_launch_count() -> int:
+    return int(lib().gdn_launch_count())
+
+
+def gdn_stage_timing_enable(on: bool) -> None:
+    lib().gdn_stage_timing_enable(1 if on else 0)
+
+
+def gdn_stage_timing_read():
+    """Returns {stage_name: (total_ms, launches)} accumulated since the previous read."""
+    n = 32
+    ms = (ctypes.c_float * n)()
+    cnt = (ctypes.c_int32 * n)()
+    names = (ctypes.c_char_p * n)()
+    got = ctypes.c_int32(0)
+    s = lib().gdn_stage_timing_read(n, ms, cnt, names, ctypes.byref(got))
+    if s != GDN_OK:
+        raise GdnError(s, "gdn_stage_timing_read")
+    return {names[i].decode(): (float(ms[i]), int(cnt[i])) for i in range(got.value)}

@@ -2,9 +2,44 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
+#include <vector>
+
 #include "gdn_internal.cuh"
 
 namespace gdn {
+
+// ---- launch counting and optional per-stage event timing ----
+namespace {
+std::atomic<uint64_t> g_launches{0};
+bool g_timing = false;
+struct Rec { Stage s; cudaEvent_t a, b; };
+std::vector<Rec> g_recs;          // recorded since the last read
+std::vector<cudaEvent_t> g_pool;  // reusable events
+cudaEvent_t g_open = nullptr;
+const char* kStageNames[ST_COUNT] = {"table", "prep", "fscan", "out", "eprep", "rscan", "intra"};
+cudaEvent_t take_event() {
+    if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+}  // namespace
+
+void stage_begin(Stage, cudaStream_t st) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (!g_timing) return;
+    g_open = take_event();
+    cudaEventRecord(g_open, st);
+}
+void stage_end(Stage s, cudaStream_t st) {
+    if (!g_timing || !g_open) return;
+    cudaEvent_t b = take_event();
+    cudaEventRecord(b, st);
+    g_recs.push_back({s, g_open, b});
+    g_open = nullptr;
+}
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -123,6 +158,34 @@ const char* gdn_status_string(gdn_status s) {
         case GDN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
     }
     return "unknown status";
+}
+
+uint64_t gdn_launch_count(void) { return g_launches.load(); }
+
+gdn_status gdn_stage_timing_enable(int32_t on) {
+    g_timing = on != 0;
+    return GDN_OK;
+}
+
+gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* launches, const char** names,
+                                 int32_t* n_stages) {
+    if (!total_ms || !launches || !names || !n_stages) return GDN_ERR_NULL_ARG;
+    float ms[ST_COUNT] = {};
+    int32_t cnt[ST_COUNT] = {};
+    gdn_status rc = GDN_OK;
+    for (const Rec& r : g_recs) {
+        float t = 0.f;
+        if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) rc = GDN_ERR_CUDA;
+        ms[r.s] += t;
+        cnt[r.s] += 1;
+        g_pool.push_back(r.a);
+        g_pool.push_back(r.b);
+    }
+    g_recs.clear();
+    const int n = max_stages < (int)ST_COUNT ? max_stages : (int)ST_COUNT;
+    for (int i = 0; i < n; ++i) { total_ms[i] = ms[i]; launches[i] = cnt[i]; names[i] = kStageNames[i]; }
+    *n_stages = n;
+    return rc;
 }
 
 const char* gdn_kernel_path(const gdn_desc* desc) {

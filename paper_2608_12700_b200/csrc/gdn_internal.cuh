@@ -85,6 +85,17 @@ struct Problem {
     WsLayout L;
 };
 
+// Launch bookkeeping: every kernel launch goes through stage_begin / stage_end so that launches can be
+// counted and, when enabled, timed per stage with CUDA events on the launching stream.
+enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_COUNT };
+void stage_begin(Stage s, cudaStream_t st);
+void stage_end(Stage s, cudaStream_t st);
+struct StageScope {
+    Stage s; cudaStream_t st;
+    StageScope(Stage s_, cudaStream_t st_) : s(s_), st(st_) { stage_begin(s, st); }
+    ~StageScope() { stage_end(s, st); }
+};
+
 // Kernel families (each defined in its own translation unit).  They enqueue on `st` and return the
 // first CUDA error seen.
 cudaError_t simt_launch_fwd(const Problem& p, cudaStream_t st);

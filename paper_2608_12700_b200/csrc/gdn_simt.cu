@@ -575,13 +575,13 @@ __global__ void __launch_bounds__(kThreads) intra_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 cudaError_t launch_fwd_t(const Problem& p, cudaStream_t st) {
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
-    table_kernel<<<1, 256, 0, st>>>(p);
-    if (CH > 0) prep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p);
+    { StageScope t(ST_TABLE, st); table_kernel<<<1, 256, 0, st>>>(p); }
+    if (CH > 0) { StageScope t(ST_PREP, st); prep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
     const size_t sm = 2 * sizeof(float) * DK * DV;
     cudaError_t e = cudaFuncSetAttribute(scan_kernel<DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    if (chains > 0) scan_kernel<DK, DV, false><<<chains, kThreads, sm, st>>>(p);
-    if (p.o && CH > 0) out_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p);
+    if (chains > 0) { StageScope t(ST_FSCAN, st); scan_kernel<DK, DV, false><<<chains, kThreads, sm, st>>>(p); }
+    if (p.o && CH > 0) { StageScope t(ST_OUT, st); out_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
     return cudaGetLastError();
 }
 
@@ -593,14 +593,14 @@ cudaError_t launch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st)
         if (e != cudaSuccess) return e;
     }
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
-    if (CH > 0) eprep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p);
+    if (CH > 0) { StageScope t(ST_EPREP, st); eprep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
     const size_t sm = 2 * sizeof(float) * DK * DV;
     e = cudaFuncSetAttribute(scan_kernel<DK, DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    if (chains > 0) scan_kernel<DK, DV, true><<<chains, kThreads, sm, st>>>(p);
+    if (chains > 0) { StageScope t(ST_RSCAN, st); scan_kernel<DK, DV, true><<<chains, kThreads, sm, st>>>(p); }
     e = cudaFuncSetAttribute(intra_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(IntraSmem));
     if (e != cudaSuccess) return e;
-    if (CH > 0) intra_kernel<IO, DK, DV><<<CH, kThreads, sizeof(IntraSmem), st>>>(p);
+    if (CH > 0) { StageScope t(ST_INTRA, st); intra_kernel<IO, DK, DV><<<CH, kThreads, sizeof(IntraSmem), st>>>(p); }
     return cudaGetLastError();
 }
 
