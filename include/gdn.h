@@ -126,6 +126,17 @@ gdn_status gdn_stage_timing_enable(int32_t on);
 gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* launches, const char** names,
                                  int32_t* n_stages);
 
+/* ---- debugging hooks (the paper has no counterpart) ---------------------------------------------
+ * gdn_debug_read: synchronises the device and copies one workspace quantity of one (chunk, head) to
+ * host memory as row-major float32, whatever the internal storage format:
+ *   "gamma" [64]   "T" [64,64]   "W" [64,d_k]   "Ut" [64,d_v]   "Nm" [d_k,d_k]
+ *   "Bf", "E", "hc", "dhn" [d_k,d_v]
+ * gdn_debug_force_family: 0 = automatic dispatch, 1 = always use the FFMA kernels (tests use this to
+ * exercise both families on the same inputs).  Process-wide; affects workspace sizes as well. */
+gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
+                          float* host_out);
+gdn_status gdn_debug_force_family(int32_t family);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
-           "gdn_stage_timing_read"]
+           "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -69,6 +69,10 @@ def lib():
         L.gdn_stage_timing_enable.argtypes = [I]
         L.gdn_stage_timing_read.restype = I
         L.gdn_stage_timing_read.argtypes = [I, P, P, P, P]
+        L.gdn_debug_read.restype = I
+        L.gdn_debug_read.argtypes = [D, P, ctypes.c_char_p, I, I, P]
+        L.gdn_debug_force_family.restype = I
+        L.gdn_debug_force_family.argtypes = [I]
         _lib = L
     return _lib
 
@@ -158,3 +162,23 @@ def gdn_stage_timing_read():
     if s != GDN_OK:
         raise GdnError(s, "gdn_stage_timing_read")
     return {names[i].decode(): (float(ms[i]), int(cnt[i])) for i in range(got.value)}
+
+
+def gdn_debug_force_family(family: int) -> None:
+    s = lib().gdn_debug_force_family(int(family))
+    if s != GDN_OK:
+        raise GdnError(s, "gdn_debug_force_family")
+
+
+def gdn_debug_read(desc: gdn_desc, workspace, what: str, chunk: int, head: int):
+    """One workspace quantity of one (chunk, head) as a row-major float32 numpy array."""
+    import numpy as np
+    dk, dv = desc.d_k, desc.d_v
+    shapes = {"gamma": (64,), "T": (64, 64), "W": (64, dk), "Ut": (64, dv), "Nm": (dk, dk), "Bf": (dk, dv),
+              "hc": (dk, dv), "E": (dk, dv), "dhn": (dk, dv)}
+    out = np.zeros(shapes[what], dtype=np.float32)
+    s = lib().gdn_debug_read(ctypes.byref(desc), _p(workspace), what.encode(), int(chunk), int(head),
+                             out.ctypes.data_as(ctypes.c_void_p))
+    if s != GDN_OK:
+        raise GdnError(s, "gdn_debug_read")
+    return out

@@ -17,7 +17,7 @@ struct Rec { Stage s; cudaEvent_t a, b; };
 std::vector<Rec> g_recs;          // recorded since the last read
 std::vector<cudaEvent_t> g_pool;  // reusable events
 cudaEvent_t g_open = nullptr;
-const char* kStageNames[ST_COUNT] = {"table", "prep", "fscan", "out", "eprep", "rscan", "intra"};
+const char* kStageNames[ST_COUNT] = {"table", "prep", "fscan", "out", "eprep", "rscan", "intra", "scans"};
 cudaEvent_t take_event() {
     if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
     cudaEvent_t e = nullptr;
@@ -46,9 +46,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 enum class Path { None, SimtF32, SimtBf16, TcBf16 };
 
+int g_force_family = 0;
+
 Path pick_path(const gdn_desc& d) {
     if (d.dtype == GDN_F32) return Path::SimtF32;
-    if (d.dtype == GDN_BF16) return Path::SimtBf16;
+    if (d.dtype == GDN_BF16) return (tc_supported(d) && g_force_family != 1) ? Path::TcBf16 : Path::SimtBf16;
     return Path::None;
 }
 
@@ -64,8 +66,10 @@ gdn_status check_desc(const gdn_desc* d) {
 }
 
 WsLayout layout_for(const gdn_desc& d) {
+    // tcgen05 path: bf16 tile images for the factors and states, fp32 for the additive terms of the carries.
+    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 4, 0);
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
-    return make_layout(d, sizeof(float), simt_scratch_per_chunkhead(d));
+    return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
 }
 
 // Sequences are described either by cu_seqlens (then B must be 1) or by B rows of T tokens (then N == B).
@@ -109,7 +113,8 @@ gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k,
     p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.h0 = h0; p.cu = cu; p.o = o; p.hT = hT;
     p.ws = static_cast<char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    return simt_launch_fwd(p, st) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    const cudaError_t e = pick_path(*desc) == Path::TcBf16 ? tc_launch_fwd(p, st) : simt_launch_fwd(p, st);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -132,7 +137,9 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     p.dq = dq; p.dk = dk; p.dv = dv; p.dg = dg; p.dbeta = dbeta; p.dh0 = dh0;
     p.ws = static_cast<char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    return simt_launch_bwd(p, workspace_is_fresh_from_fwd != 0, st) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    const bool fresh = workspace_is_fresh_from_fwd != 0;
+    const cudaError_t e = pick_path(*desc) == Path::TcBf16 ? tc_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream) {
@@ -158,6 +165,59 @@ const char* gdn_status_string(gdn_status s) {
         case GDN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
     }
     return "unknown status";
+}
+
+gdn_status gdn_debug_force_family(int32_t family) {
+    if (family != 0 && family != 1) return GDN_ERR_BAD_SHAPE;
+    g_force_family = family;
+    return GDN_OK;
+}
+
+gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
+                          float* host_out) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if (!workspace || !what || !host_out) return GDN_ERR_NULL_ARG;
+    const WsLayout L = layout_for(*desc);
+    if (chunk < 0 || chunk >= L.max_chunks || head < 0 || head >= desc->H) return GDN_ERR_BAD_SHAPE;
+    const bool tcp = pick_path(*desc) == Path::TcBf16;
+    const size_t ch = (size_t)chunk * desc->H + head;
+    const int dk = desc->d_k, dv = desc->d_v;
+    struct Q { const char* name; size_t off; int rows, cols; int kind; };  // kind 0: fp32 row-major always
+    // kind 1: factor (fp32 row-major | bf16 tile image [rows][cols]); kind 2: factor stored transposed as an image
+    // [cols][rows] on the tcgen05 path; kind 3: additive term (fp32 row-major | fp32 column-chunk-major)
+    const Q table[] = {{"gamma", L.gamma, 1, kC, 0}, {"T", L.Tm, kC, kC, 1},    {"W", L.W, kC, dk, 2},
+                       {"Ut", L.Ut, kC, dv, 2},      {"Nm", L.Nm, dk, dk, 1},   {"Bf", L.Bf, dk, dv, 3},
+                       {"hc", L.hc, dk, dv, 1},      {"E", L.E, dk, dv, 3},     {"dhn", L.dhn, dk, dv, 1}};
+    const Q* q = nullptr;
+    for (const Q& t : table) if (strcmp(t.name, what) == 0) q = &t;
+    if (!q) return GDN_ERR_BAD_SHAPE;
+    if (cudaDeviceSynchronize() != cudaSuccess) return GDN_ERR_CUDA;
+    const size_t n = (size_t)q->rows * q->cols;
+    const char* base = static_cast<const char*>(workspace) + q->off;
+    if (q->kind == 0 || !tcp) {
+        return cudaMemcpy(host_out, base + ch * n * 4, n * 4, cudaMemcpyDeviceToHost) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    }
+    if (q->kind == 3) {
+        std::vector<float> tmp(n);
+        if (cudaMemcpy(tmp.data(), base + ch * n * 4, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GDN_ERR_CUDA;
+        for (int r = 0; r < q->rows; ++r)
+            for (int c = 0; c < q->cols; ++c) host_out[(size_t)r * q->cols + c] = tmp[((size_t)(c / 4) * q->rows + r) * 4 + (c % 4)];
+        return GDN_OK;
+    }
+    std::vector<uint16_t> img(n);
+    if (cudaMemcpy(img.data(), base + ch * n * 2, n * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return GDN_ERR_CUDA;
+    const int R = q->kind == 2 ? q->cols : q->rows;       // rows of the stored tile
+    auto at = [&](int r, int c) -> float {                 // element (r, c) of the stored tile
+        const size_t off = (size_t)(c >> 6) * R * 128 + (size_t)r * 128 + ((((c & 63) >> 3) ^ (r & 7)) << 4) + ((c & 7) << 1);
+        const uint32_t bits = (uint32_t)img[off / 2] << 16;
+        float f;
+        memcpy(&f, &bits, 4);
+        return f;
+    };
+    for (int r = 0; r < q->rows; ++r)
+        for (int c = 0; c < q->cols; ++c) host_out[(size_t)r * q->cols + c] = q->kind == 2 ? at(c, r) : at(r, c);
+    return GDN_OK;
 }
 
 uint64_t gdn_launch_count(void) { return g_launches.load(); }

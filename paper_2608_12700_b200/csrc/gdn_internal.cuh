@@ -44,8 +44,9 @@ struct WsLayout {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// elem = bytes per stored factor element (4 on the fp32 path).
-inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t scratch_per_ch) {
+// elem = bytes per element of the chunk factors and stored states (T, W, U~, Nm, hc, dhn): 4 on the fp32
+// path, 2 for the bf16 tile images of the tcgen05 path.  elem_add = bytes per element of Bf and E.
+inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, size_t scratch_per_ch) {
     WsLayout L{};
     const size_t Ttot = (size_t)d.B * (size_t)d.T;
     L.max_chunks = (int)((Ttot + kC - 1) / kC + (size_t)d.N);
@@ -61,10 +62,10 @@ inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t scratch_per_c
     L.W = take(elem * CH * kC * d.d_k);
     L.Ut = take(elem * CH * kC * d.d_v);
     L.Nm = take(elem * CH * d.d_k * d.d_k);
-    L.Bf = take(elem * CH * d.d_k * d.d_v);
+    L.Bf = take(elem_add * CH * d.d_k * d.d_v);
     L.hc = take(elem * CH * d.d_k * d.d_v);
     L.fwd_end = o;
-    L.E = take(elem * CH * d.d_k * d.d_v);
+    L.E = take(elem_add * CH * d.d_k * d.d_v);
     L.dhn = take(elem * CH * d.d_k * d.d_v);
     L.scratch_per_ch = scratch_per_ch;
     L.scratch = take(scratch_per_ch * CH);
@@ -87,7 +88,7 @@ struct Problem {
 
 // Launch bookkeeping: every kernel launch goes through stage_begin / stage_end so that launches can be
 // counted and, when enabled, timed per stage with CUDA events on the launching stream.
-enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_COUNT };
+enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_SCANS, ST_COUNT };
 void stage_begin(Stage s, cudaStream_t st);
 void stage_end(Stage s, cudaStream_t st);
 struct StageScope {
@@ -98,8 +99,14 @@ struct StageScope {
 
 // Kernel families (each defined in its own translation unit).  They enqueue on `st` and return the
 // first CUDA error seen.
+cudaError_t launch_table(const Problem& p, cudaStream_t st);
 cudaError_t simt_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t simt_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 size_t simt_scratch_per_chunkhead(const gdn_desc& d);
+
+// tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
+bool tc_supported(const gdn_desc& d);
+cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
+cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 
 }  // namespace gdn

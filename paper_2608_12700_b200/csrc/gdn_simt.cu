@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kThreads) intra_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 cudaError_t launch_fwd_t(const Problem& p, cudaStream_t st) {
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
-    { StageScope t(ST_TABLE, st); table_kernel<<<1, 256, 0, st>>>(p); }
+    launch_table(p, st);
     if (CH > 0) { StageScope t(ST_PREP, st); prep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
     const size_t sm = 2 * sizeof(float) * DK * DV;
     cudaError_t e = cudaFuncSetAttribute(scan_kernel<DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
@@ -605,6 +605,12 @@ cudaError_t launch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st)
 }
 
 }  // namespace
+
+cudaError_t launch_table(const Problem& p, cudaStream_t st) {
+    StageScope t(ST_TABLE, st);
+    table_kernel<<<1, 256, 0, st>>>(p);
+    return cudaGetLastError();
+}
 
 size_t simt_scratch_per_chunkhead(const gdn_desc& d) { return sizeof(float) * kC * 3 * ((size_t)d.d_k + d.d_v); }
 

@@ -1,0 +1,198 @@
+// Thin inline-PTX layer for sm_100a: mbarrier, bulk/TMA copies, tensor memory and tcgen05.mma.
+// Everything here is a one-to-one wrapper of a PTX instruction plus the shared-memory tile format the
+// kernels agree on.
+//
+// Tile format ("blocked-64, 128-byte swizzle"): a bf16 matrix of R rows and 64*nb columns is stored as
+// nb column blocks of R rows x 64 columns; a block row is 128 bytes; the eight 16-byte chunks of a row are
+// permuted by XOR with (row % 8).  Blocks are R*128 bytes apart and must start on 1024-byte boundaries.
+// The same bytes serve tcgen05.mma as a K-major operand (contraction over columns) and as an MN-major
+// operand (contraction over rows), so no explicit transposes are ever made.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace gdn {
+namespace tc {
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// ---------------------------------------------------------------- tile addressing
+// Byte offset of element (r, c) inside a tile with R rows.
+__device__ __forceinline__ uint32_t tile_off(int R, int r, int c) {
+    return (uint32_t)((c >> 6) * R * 128 + r * 128 + ((((c & 63) >> 3) ^ (r & 7)) << 4) + ((c & 7) << 1));
+}
+// Byte offset of the 16-byte chunk holding columns [8*ch, 8*ch + 8) of row r.
+__device__ __forceinline__ uint32_t tile_chunk_off(int R, int r, int ch) {
+    return (uint32_t)((ch >> 3) * R * 128 + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
+}
+
+// ---------------------------------------------------------------- mbarrier
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after about two seconds and returns false; the caller records the failure and
+// leaves through its normal teardown (no trap, no endless spin).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int i = 0; i < 64; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+// ---------------------------------------------------------------- proxies and copies
+// Make generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// 2-D tiled TMA load: box lands at smem_dst, completion bytes are counted on bar.
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+// Contiguous bulk copy global -> shared (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+// Contiguous bulk copy shared -> global, tracked by the bulk async-group of the issuing thread.
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until at most N of this thread's bulk groups still read their shared-memory source.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+
+// ---------------------------------------------------------------- tensor memory
+// One warp allocates `cols` (power of two >= 32) columns; the base address is written to *slot (shared).
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Each thread of a warp reads 32 consecutive fp32 columns of its own lane (lane = 32 * (warp % 4) + laneid).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---------------------------------------------------------------- tcgen05.mma (bf16 x bf16 -> fp32)
+// Instruction descriptor: dense, fp32 accumulate, bf16 A and B.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major, bool neg_a = false) {
+    return (1u << 4)                          // D format: fp32
+           | (1u << 7) | (1u << 10)           // A, B format: bf16
+           | ((neg_a ? 1u : 0u) << 13)        // negate A
+           | ((a_mn_major ? 1u : 0u) << 15)   // A major
+           | ((b_mn_major ? 1u : 0u) << 16)   // B major
+           | ((uint32_t)(N >> 3) << 17)       // N / 8
+           | ((uint32_t)(M >> 4) << 24);      // M / 16
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle; lbo/sbo in bytes.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)((lbo >> 4) & 0x3FFF) << 16) | ((uint64_t)((sbo >> 4) & 0x3FFF) << 32) |
+           (1ull << 46)   // descriptor version of this architecture
+           | (2ull << 61);  // 128-byte swizzle
+}
+
+// Operand view of a tile (or of a row/column window of it) for one MMA with contraction length Kt.
+struct Operand {
+    uint32_t base;     // shared address of element (row0, col0) of the window (row0 % 8 == 0, col0 % 64 == 0)
+    uint32_t R;        // rows of the underlying tile (block stride = R * 128 bytes)
+    bool mn_major;     // false: contraction runs over tile columns; true: over tile rows
+};
+// Window whose MN index runs over tile rows starting at row0 and whose K index runs over columns from col0.
+__device__ __forceinline__ Operand op_k_major(const void* tile, int R, int row0 = 0, int col0 = 0) {
+    return Operand{smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), (uint32_t)R, false};
+}
+// Window whose MN index runs over tile columns starting at col0 and whose K index runs over rows from row0.
+__device__ __forceinline__ Operand op_mn_major(const void* tile, int R, int row0 = 0, int col0 = 0) {
+    return Operand{smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), (uint32_t)R, true};
+}
+// Descriptor of the k-th K=16 slice.
+__device__ __forceinline__ uint64_t op_desc(const Operand& o, int ks) {
+    if (!o.mn_major)   // 16 columns = 32 bytes inside a 128-byte row; every 4th step moves to the next column block
+        return make_desc(o.base + (uint32_t)((ks >> 2) * o.R * 128 + (ks & 3) * 32), 16, 1024);
+    // 16 rows = 2048 bytes; LBO = distance between 64-column blocks, SBO = distance between 8-row groups
+    return make_desc(o.base + (uint32_t)ks * 2048, o.R * 128, 1024);
+}
+
+__device__ __forceinline__ void mma_issue(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+// D[M x N] (+)= A[M x Kt] * B[Kt x N]; one thread issues Kt/16 instructions.
+__device__ __forceinline__ void mma_tile(uint32_t tmem_d, const Operand& a, const Operand& b, int M, int N, int Kt, bool accumulate,
+                                         bool neg_a = false) {
+    const uint32_t idesc = make_idesc(M, N, a.mn_major, b.mn_major, neg_a);
+    for (int ks = 0; ks < Kt / 16; ++ks) mma_issue(tmem_d, op_desc(a, ks), op_desc(b, ks), idesc, accumulate || ks > 0);
+}
+// Arrive on `bar` when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// ---------------------------------------------------------------- small conversions
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+}  // namespace tc
+}  // namespace gdn
