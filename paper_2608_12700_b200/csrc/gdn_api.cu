@@ -101,8 +101,10 @@ gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k,
     gdn_status s = check_desc(desc);
     if (s != GDN_OK) return s;
     if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
-    if (!q || !k || !v || !g || !workspace) return GDN_ERR_NULL_ARG;
-    if (desc->delta_rule && !beta) return GDN_ERR_NULL_ARG;
+    const bool empty = (long long)desc->B * desc->T == 0;   // no tokens: token tensors may be NULL
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    if (!empty && (!q || !k || !v || !g)) return GDN_ERR_NULL_ARG;
+    if (!empty && desc->delta_rule && !beta) return GDN_ERR_NULL_ARG;
     const void* ptrs[] = {q, k, v, g, beta, h0, cu, o, hT, workspace};
     for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
     Problem p{};
@@ -124,8 +126,10 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     gdn_status s = check_desc(desc);
     if (s != GDN_OK) return s;
     if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
-    if (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg || !workspace) return GDN_ERR_NULL_ARG;
-    if (desc->delta_rule && (!beta || !dbeta)) return GDN_ERR_NULL_ARG;
+    const bool empty = (long long)desc->B * desc->T == 0;   // no tokens: token tensors may be NULL
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    if (!empty && (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg)) return GDN_ERR_NULL_ARG;
+    if (!empty && desc->delta_rule && (!beta || !dbeta)) return GDN_ERR_NULL_ARG;
     const void* ptrs[] = {q, k, v, g, beta, h0, dO, dhT, cu, dq, dk, dv, dg, dbeta, dh0, workspace};
     for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
     Problem p{};

@@ -9,6 +9,15 @@ from helpers import TOL, check_against_oracle, oracle_grads, rel
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["auto", "ffma"])
+def family(request):
+    """Runs a test once with automatic dispatch (tcgen05 kernels where supported) and once with the FFMA
+    kernels forced, so both families see the same inputs."""
+    binding.gdn_debug_force_family(1 if request.param == "ffma" else 0)
+    yield request.param
+    binding.gdn_debug_force_family(0)
+
+
 def small(name, **kw):
     base = dict(dtype="f32", H=2, d_k=64, d_v=64, seed=100)
     base.update(kw)
@@ -23,13 +32,13 @@ def test_config0_fp32():
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("dk,dv", [(64, 64), (128, 128), (128, 64), (64, 128)])
-def test_shapes_with_states(dtype, dk, dv):
+def test_shapes_with_states(dtype, dk, dv, family):
     wl = small(f"shape_{dtype}_{dk}_{dv}", dtype=dtype, B=2, T=192, H=2, d_k=dk, d_v=dv, states=True, seed=7)
     check_against_oracle(wl, runner.backward(wl))
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_ragged_varlen_and_empty_sequence(dtype):
+def test_ragged_varlen_and_empty_sequence(dtype, family):
     # lengths: a tail of 1, an exact multiple, an empty sequence, a sub-chunk sequence, a long ragged one
     wl = small("ragged_" + dtype, dtype=dtype, lengths=[65, 128, 0, 37, 300], H=3, d_k=128, d_v=128,
                states=True, seed=11)
@@ -51,18 +60,35 @@ def test_scale_argument():
     check_against_oracle(wl, runner.backward(wl))
 
 
-def test_forward_outputs_match_oracle():
-    wl = small("fwd", lengths=[70, 130], H=2, d_k=64, d_v=128, states=True, seed=14)
+@pytest.mark.parametrize("dtype,dk,dv", [("f32", 64, 128), ("bf16", 128, 128), ("bf16", 64, 64)])
+def test_forward_outputs_match_oracle(dtype, dk, dv):
+    wl = small("fwd", dtype=dtype, lengths=[70, 130], H=2, d_k=dk, d_v=dv, states=True, seed=14)
     buf = runner.to_device(wl, want_o=True)
     runner.run_fwd(buf)
     got = runner.fetch(buf)
     ref = oracle_grads(wl)
-    assert rel(got["o"], ref["o"]) < 1e-4
-    assert rel(got["hT"], ref["hT"]) < 1e-4
+    assert rel(got["o"], ref["o"]) < TOL[dtype]
+    assert rel(got["hT"], ref["hT"]) < TOL[dtype]
 
 
-def test_fresh_workspace_reuse_gives_identical_gradients():
-    wl = small("fresh", B=1, T=256, H=2, states=True, seed=15)
+def test_kernel_family_dispatch():
+    mk = lambda **kw: binding.make_desc(**dict(dict(B=1, T=64, H=1, d_k=128, d_v=128, N=1, dtype="bf16"), **kw))
+    assert binding.gdn_kernel_path(mk()) == "tcgen05_bf16"
+    assert binding.gdn_kernel_path(mk(dtype="f32")) == "simt_f32"
+    assert binding.gdn_kernel_path(mk(d_k=64, d_v=64)) == "simt_bf16"
+    assert binding.gdn_kernel_path(mk(delta_rule=0)) == "simt_bf16"
+
+
+def test_zero_tokens_passes_the_state_gradient_through():
+    for dtype, d in (("f32", 64), ("bf16", 128)):
+        wl = small("empty", dtype=dtype, lengths=[0, 0], H=2, d_k=d, d_v=d, states=True, seed=21)
+        got = runner.backward(wl)
+        assert np.array_equal(got["dh0"], wl.dhT.astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 128)])
+def test_fresh_workspace_reuse_gives_identical_gradients(dtype, d):
+    wl = small("fresh", dtype=dtype, B=1, T=256, H=2, d_k=d, d_v=d, states=True, seed=15)
     a = runner.backward(wl)
     buf = runner.to_device(wl, want_o=True)
     runner.run_fwd(buf)
@@ -72,7 +98,7 @@ def test_fresh_workspace_reuse_gives_identical_gradients():
         assert np.array_equal(a[n], b[n]), n
 
 
-def test_bitwise_determinism_over_repeats():
+def test_bitwise_determinism_over_repeats(family):
     wl = small("determinism", dtype="bf16", lengths=[100, 260], H=4, d_k=128, d_v=128, states=True, seed=16)
     buf = runner.to_device(wl)
     runner.run_bwd(buf)
