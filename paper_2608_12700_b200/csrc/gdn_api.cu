@@ -66,8 +66,8 @@ gdn_status check_desc(const gdn_desc* d) {
 }
 
 WsLayout layout_for(const gdn_desc& d) {
-    // tcgen05 path: bf16 tile images for the factors and states, fp32 for the additive terms of the carries.
-    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 4, 0);
+    // tcgen05 path: every factor, state and additive term of the carries is a bf16 tile image.
+    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0);
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
     return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
 }
@@ -189,10 +189,10 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
     const int dk = desc->d_k, dv = desc->d_v;
     struct Q { const char* name; size_t off; int rows, cols; int kind; };  // kind 0: fp32 row-major always
     // kind 1: factor (fp32 row-major | bf16 tile image [rows][cols]); kind 2: factor stored transposed as an image
-    // [cols][rows] on the tcgen05 path; kind 3: additive term (fp32 row-major | fp32 column-chunk-major)
+    // [cols][rows] on the tcgen05 path
     const Q table[] = {{"gamma", L.gamma, 1, kC, 0}, {"T", L.Tm, kC, kC, 1},    {"W", L.W, kC, dk, 2},
-                       {"Ut", L.Ut, kC, dv, 2},      {"Nm", L.Nm, dk, dk, 1},   {"Bf", L.Bf, dk, dv, 3},
-                       {"hc", L.hc, dk, dv, 1},      {"E", L.E, dk, dv, 3},     {"dhn", L.dhn, dk, dv, 1}};
+                       {"Ut", L.Ut, kC, dv, 2},      {"Nm", L.Nm, dk, dk, 1},   {"Bf", L.Bf, dk, dv, 1},
+                       {"hc", L.hc, dk, dv, 1},      {"E", L.E, dk, dv, 1},     {"dhn", L.dhn, dk, dv, 1}};
     const Q* q = nullptr;
     for (const Q& t : table) if (strcmp(t.name, what) == 0) q = &t;
     if (!q) return GDN_ERR_BAD_SHAPE;
@@ -201,13 +201,6 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
     const char* base = static_cast<const char*>(workspace) + q->off;
     if (q->kind == 0 || !tcp) {
         return cudaMemcpy(host_out, base + ch * n * 4, n * 4, cudaMemcpyDeviceToHost) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
-    }
-    if (q->kind == 3) {
-        std::vector<float> tmp(n);
-        if (cudaMemcpy(tmp.data(), base + ch * n * 4, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GDN_ERR_CUDA;
-        for (int r = 0; r < q->rows; ++r)
-            for (int c = 0; c < q->cols; ++c) host_out[(size_t)r * q->cols + c] = tmp[((size_t)(c / 4) * q->rows + r) * 4 + (c % 4)];
-        return GDN_OK;
     }
     std::vector<uint16_t> img(n);
     if (cudaMemcpy(img.data(), base + ch * n * 2, n * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return GDN_ERR_CUDA;

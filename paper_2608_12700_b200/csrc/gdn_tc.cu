@@ -1,12 +1,13 @@
 // tcgen05 / TMEM / TMA kernels of the GDN backward for bf16 I/O, d_k = d_v = 128, chunk 64 (sm_100a).
 //
-// Three kernels follow the stage map of the chunked method (Section 4.2 of the paper):
+// Kernels follow the stage map of the chunked method (Section 4.2 of the paper):
 //   tc_prep  (one CTA per chunk-head)  gamma, A, T = (I + A)^-1, W, U~, Nm = Kb^T W, Bf = Kb^T U~ and, for the
 //                                      backward, E = scale (Diag(Gam) Q - P W)^T dO
-//   tc_scan  (one CTA per chain, direction and 64-column slice of the state)
+//   tc_scan  (one CTA per chain and direction)
 //                                      forward carry  h'  = Gam_e h  - Nm   h  + Bf   (stores h per chunk)
 //                                      reverse carry  dh  = Gam_e dh' - Nm^T dh' + E   (the paper's K#1; stores dh')
 //   tc_intra (one CTA per chunk-head)  every token gradient, including the VJP of the triangular solve (K#2)
+//   tc_out   (optional)                forward output o
 //
 // All dense products run on tcgen05.mma with fp32 accumulators in tensor memory; operands are bf16 tiles in
 // shared memory in the "blocked-64, 128-byte swizzle" format of tc_ptx.cuh, brought in by TMA (inputs) or by
@@ -15,17 +16,29 @@
 // The carried states stay fp32 in registers for the whole scan; tensor memory holds accumulators only and is
 // allocated once per CTA and released once.  Every wait is bounded; a wait that gives up records
 // GDN_ERR_DEVICE_TIMEOUT in the workspace header and the CTA leaves through its normal teardown.
+// Loops over accumulator columns are kept rolled (8 columns per trip): the kernels run each piece of code once
+// per chunk, so instruction-cache footprint matters more than loop overhead.
 #include "gdn_internal.cuh"
 #include "tc_ptx.cuh"
 #include "tc_tmap.cuh"
 
 namespace gdn {
+
+// Optional phase timing (compile with -DGDN_PHASE_TIMING): thread 0 of CTA 0 stamps clock64() at phase borders.
+#ifdef GDN_PHASE_TIMING
+__device__ long long g_ticks[4][32];
+#define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_ticks[kern][idx] = clock64(); } while (0)
+#else
+#define GDN_TICK(kern, idx) do { } while (0)
+#endif
+
 namespace {
 
 using namespace tc;
 
 constexpr int D = 128;          // d_k = d_v
 constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column half = warp / 4
+constexpr float kLog2e = 1.4426950408889634f;
 
 struct TcParams {
     Problem p;
@@ -44,7 +57,7 @@ __device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
     return p + ((1024u - (smem_u32(p) & 1023u)) & 1023u);
 }
 
-// 8 fp32 -> one 16-byte chunk of bf16
+// 8 fp32 <-> one 16-byte chunk of bf16
 __device__ __forceinline__ uint4 pack8(const float* v) {
     return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
 }
@@ -52,20 +65,21 @@ __device__ __forceinline__ void unpack8(const uint4& u, float* v) {
     v[0] = bf16_lo(u.x); v[1] = bf16_hi(u.x); v[2] = bf16_lo(u.y); v[3] = bf16_hi(u.y);
     v[4] = bf16_lo(u.z); v[5] = bf16_hi(u.z); v[6] = bf16_lo(u.w); v[7] = bf16_hi(u.w);
 }
-// Write 32 consecutive columns [c0, c0 + 32) of row r of a tile with R rows (c0 % 32 == 0).
-__device__ __forceinline__ void tile_store32(unsigned char* tile, int R, int r, int c0, const float* v) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(tile + tile_chunk_off(R, r, (c0 >> 3) + c)) = pack8(v + 8 * c);
+// Chunk `ch` (columns 8 ch .. 8 ch + 7) of row r of a tile with R rows.
+__device__ __forceinline__ void chunk_store(unsigned char* tile, int R, int r, int ch, const float* v) {
+    *reinterpret_cast<uint4*>(tile + tile_chunk_off(R, r, ch)) = pack8(v);
 }
-__device__ __forceinline__ void tile_load32(const unsigned char* tile, int R, int r, int c0, float* v) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) unpack8(*reinterpret_cast<const uint4*>(tile + tile_chunk_off(R, r, (c0 >> 3) + c)), v + 8 * c);
+__device__ __forceinline__ void chunk_load(const unsigned char* tile, int R, int r, int ch, float* v) {
+    unpack8(*reinterpret_cast<const uint4*>(tile + tile_chunk_off(R, r, ch)), v);
 }
 __device__ __forceinline__ float tile_get(const unsigned char* tile, int R, int r, int c) {
     return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + tile_off(R, r, c)));
 }
+__device__ __forceinline__ void tile_put(unsigned char* tile, int R, int r, int c, float x) {
+    *reinterpret_cast<__nv_bfloat16*>(tile + tile_off(R, r, c)) = __float2bfloat16_rn(x);
+}
 
-// Zero rows [len, 64) of a [rows0 .. rows0 + 64) window of a tile with R rows and 128 columns.
+// Zero rows [row0 + len, row0 + 64) of a tile with R rows and 128 columns.
 __device__ __forceinline__ void zero_tail_rows(unsigned char* tile, int R, int row0, int len) {
     for (int t = threadIdx.x; t < (kC - len) * 16; t += blockDim.x) {
         const int r = row0 + len + t / 16, ch = t % 16;
@@ -79,22 +93,99 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// Each lane holds 8 values (one per token of a group of 8); returns, on every lane, the sum over the 32 lanes of
+// the value belonging to token (lane % 8).  Fixed order: bit-identical from run to run.
+__device__ __forceinline__ float reduce8(float (&v)[8], int lane) {
+    bool up = (lane & 4) != 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float send = up ? v[k] : v[k + 4], keep = up ? v[k + 4] : v[k];
+        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    up = (lane & 2) != 0;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const float send = up ? v[k] : v[k + 2], keep = up ? v[k + 2] : v[k];
+        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    }
+    up = (lane & 1) != 0;
+    {
+        const float send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
+        v[0] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
+    }
+    float r = v[0];
+    r += __shfl_xor_sync(0xffffffffu, r, 8);
+    r += __shfl_xor_sync(0xffffffffu, r, 16);
+    return r;
+}
+
+// Copy a staged [64 tokens][128 features] bf16 tile to a [T, H, 128] tensor with 16-byte stores (rows < len only).
+__device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloat16* gbase, size_t row_pitch, int len) {
+    for (int t = threadIdx.x; t < kC * 16; t += blockDim.x) {
+        const int i = t >> 4, chk = t & 15;
+        if (i < len) *reinterpret_cast<uint4*>(gbase + (size_t)i * row_pitch + chk * 8) = *reinterpret_cast<const uint4*>(tile + tile_chunk_off(64, i, chk));
+    }
+}
+
+struct ChunkInfo { int c, hd, ch, tok0, len; };
+__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) {
+    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
+    x.c = blockIdx.x / p.d.H;
+    x.hd = blockIdx.x % p.d.H;
+    if (x.c >= hdr->n_chunks) return false;
+    x.ch = blockIdx.x;
+    x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
+    x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
+    return true;
+}
+
+// Wait for the MMAs committed to `bar`; on a timeout record it once.
+#define GDN_WAIT_MMA(where)                                                    \
+    if (ok) {                                                                  \
+        ok = mbar_wait(&bar_mma, mma_phase);                                   \
+        mma_phase ^= 1;                                                        \
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, where);              \
+    }                                                                          \
+    tc_fence_after();
+
+// One block diagonal (distance DIST below the main one) of the blocked inverse of I + A, 16 x 16 blocks:
+// T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc).  Af, Tf, Sf are fp32 [64][65] in shared memory.
+template <int DIST>
+__device__ __forceinline__ void inv_level(const float* Af, float* Tf, float* Sf) {
+    for (int o = threadIdx.x; o < (4 - DIST) * 256; o += blockDim.x) {
+        const int cb = (o >> 8) * 16, rb = cb + DIST * 16, ii = (o >> 4) & 15, jj = o & 15;
+        float s = 0.f;
+#pragma unroll
+        for (int m = 0; m < 16 * DIST; ++m) s = fmaf(Af[(rb + ii) * 65 + cb + m], Tf[(cb + m) * 65 + cb + jj], s);
+        Sf[(rb + ii) * 65 + cb + jj] = s;
+    }
+    __syncthreads();
+    for (int o = threadIdx.x; o < (4 - DIST) * 256; o += blockDim.x) {
+        const int cb = (o >> 8) * 16, rb = cb + DIST * 16, ii = (o >> 4) & 15, jj = o & 15;
+        float s = 0.f;
+#pragma unroll
+        for (int m = 0; m < 16; ++m) s = fmaf(Tf[(rb + ii) * 65 + rb + m], Sf[(rb + m) * 65 + cb + jj], s);   // T_rr is lower triangular: zeros above
+        Tf[(rb + ii) * 65 + cb + jj] = -s;
+    }
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------------------------------------
 // tc_prep
 // ------------------------------------------------------------------------------------------------
 namespace prep {
 constexpr uint32_t QK = 0;                    // [Q rows 0..63 ; K rows 64..127] x 128   32 KB (later: Nm image)
-constexpr uint32_t VO = 32768;                // [V ; dO] x 128                           32 KB
+constexpr uint32_t VO = 32768;                // [V ; dO] x 128                           32 KB (later: Bf image)
 constexpr uint32_t TT = 65536;                // T                      [64][64]           8 KB
 constexpr uint32_t TP = TT + 8192;            // T Diag(b Gam)
 constexpr uint32_t TPP = TP + 8192;           // T Diag(w)
 constexpr uint32_t PT = TPP + 8192;           // P = tril(Q K^T . D)
-constexpr uint32_t WT = PT + 8192;            // W^T   [128 dk][64 tokens]                16 KB
+constexpr uint32_t WT = PT + 8192;            // W^T   [128 dk][64 tokens]                16 KB (before: fp32 scratch S)
 constexpr uint32_t WET = WT + 16384;          // (Diag(e) W)^T
 constexpr uint32_t UTT = WET + 16384;         // U~^T  [128 dv][64]
 constexpr uint32_t UET = UTT + 16384;         // (Diag(e) U~)^T
-constexpr uint32_t X = UET + 16384;           // fp32 A and T during the inversion; later R = Diag(Gam) dO and (P^T dO)^T
-constexpr uint32_t XA = X, XT = X + 16640;
+constexpr uint32_t X = UET + 16384;           // fp32 A and T during the inversion; then R = Diag(Gam) dO and
+constexpr uint32_t XA = X, XT = X + 16640;    // (P^T dO)^T; finally the E image
 constexpr uint32_t XR = X, XPDO = X + 16384;
 constexpr uint32_t TILES_END = X + 34816;
 constexpr uint32_t SMEM_BYTES = TILES_END + 1024 /* alignment slack */;
@@ -106,22 +197,19 @@ constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF 
 __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
     using namespace prep;
     const Problem& p = P.p;
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    const int c = blockIdx.x / p.d.H, hd = blockIdx.x % p.d.H;
-    if (c >= hdr->n_chunks) return;
-    const int ch = blockIdx.x;
-    const int tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[c];
-    const int len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[c];
+    ChunkInfo x;
+    if (!chunk_info(p, x)) return;
     const int H = p.d.H;
     const bool bwd = P.with_bwd != 0;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gam[kC], Gam[kC], ee[kC], bb[kC], ww[kC];
+    __shared__ float gam[kC], gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC];
     __shared__ uint64_t bar_qk, bar_vo, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, half = warp >> 2;
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
         mbar_init(&bar_qk, 1); mbar_init(&bar_vo, 1); mbar_init(&bar_mma, 1);
@@ -134,25 +222,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     const uint32_t tmem = tmem_slot;
     bool ok = true;
     uint32_t mma_phase = 0;
+    GDN_TICK(0, 0);
 
     if (threadIdx.x == 0) {
         mbar_expect_tx(&bar_qk, 32768);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, hd * D + cb * 64, tok0, &bar_qk);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, hd * D + cb * 64, tok0, &bar_qk);
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_qk);
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_qk);
         }
         mbar_expect_tx(&bar_vo, bwd ? 32768 : 16384);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + VO + cb * 16384, &P.tm_v, hd * D + cb * 64, tok0, &bar_vo);
-            if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, hd * D + cb * 64, tok0, &bar_vo);
+            tma_load_2d(sm + VO + cb * 16384, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_vo);
+            if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_vo);
         }
     }
     // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
         float g = 0.f, b = 0.f;
-        if (i < len) {
-            const size_t idx = (size_t)(tok0 + i) * H + hd;
+        if (i < x.len) {
+            const size_t idx = (size_t)(x.tok0 + i) * H + x.hd;
             g = p.g[idx];
             b = p.beta[idx];
         }
@@ -166,83 +255,101 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     __syncthreads();
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
+        gl[i] = gam[i] * kLog2e;
         Gam[i] = expf(gam[i]);
         ee[i] = expf(gam[kC - 1] - gam[i]);
-        reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)ch * kC + i] = gam[i];
+        reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gam[i];
     }
     ok = mbar_wait(&bar_qk, 0) && mbar_wait(&bar_vo, 0);
     if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
-    if (ok && len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
-        zero_tail_rows(sm + QK, 128, 0, len);
-        zero_tail_rows(sm + QK, 128, 64, len);
-        zero_tail_rows(sm + VO, 128, 0, len);
-        if (bwd) zero_tail_rows(sm + VO, 128, 64, len);
+    if (ok && x.len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
+        zero_tail_rows(sm + QK, 128, 0, x.len);
+        zero_tail_rows(sm + QK, 128, 64, x.len);
+        zero_tail_rows(sm + VO, 128, 0, x.len);
+        if (bwd) zero_tail_rows(sm + VO, 128, 64, x.len);
         fence_async_smem();
     }
     __syncthreads();
+    GDN_TICK(0, 1);
 
     // ---- phase 1: S1 = [Q; K] K^T  (rows 0..63: Q K^T, rows 64..127: K K^T)
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), 128, 64, 128, false);
+        mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
         mma_commit(&bar_mma);
     }
-    if (ok) { ok = mbar_wait(&bar_mma, mma_phase); mma_phase ^= 1; if (!ok && threadIdx.x == 0) report_timeout(p.ws, 2); }
-    tc_fence_after();
-    float* Af = reinterpret_cast<float*>(sm + XA);   // [64][65]
-    float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][65]
+    float* Af = reinterpret_cast<float*>(sm + XA);   // [64][65]  strictly lower part of I + A
+    float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][65]  T
+    float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][65]  scratch of the blocked inversion
+    for (int t = threadIdx.x; t < kC * 65; t += blockDim.x) Tf[t] = 0.f;
+    GDN_WAIT_MMA(2)
+    GDN_TICK(0, 2);
     if (ok) {
-        float v[32];
-        tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_S1 + half * 32, v);
-        tmem_wait_ld();
-        const int i = (q4 & 1) * 32 + lane;
-        const int j0 = half * 32;
-        if (q4 < 2) {   // P_ij = (q_i . k_j) exp(gam_i - gam_j), j <= i (mask before exponentiating)
+        const int i = (q4 & 1) * 32 + lane, j0 = half * 32;
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            float v[8];
+            tmem_ld8(tmem + lane_base + C_S1 + j0 + part * 8, v);
+            tmem_wait_ld();
+            const int jb = j0 + part * 8;
+            if (q4 < 2) {   // P_ij = (q_i . k_j) exp(gam_i - gam_j), j <= i (mask before exponentiating)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (j0 + j <= i) ? v[j] * expf(gam[i] - gam[j0 + j]) : 0.f;
-            tile_store32(sm + PT, 64, i, j0, v);
-        } else {        // A_ij = b_i (k_i . k_j) exp(gam_i - gam_j), j < i
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= i) ? v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
+                chunk_store(sm + PT, 64, i, jb >> 3, v);
+            } else {        // A_ij = b_i (k_i . k_j) exp(gam_i - gam_j), j < i
 #pragma unroll
-            for (int j = 0; j < 32; ++j) Af[i * 65 + j0 + j] = (j0 + j < i) ? bb[i] * v[j] * expf(gam[i] - gam[j0 + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) Af[i * 65 + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
+            }
         }
     }
     tc_fence_before();
     __syncthreads();
-    // ---- T = (I + A)^-1: column j solves (I + A) x = e_j by forward substitution
-    if (threadIdx.x < kC) {
-        const int j = threadIdx.x;
-        for (int i = 0; i < kC; ++i) {
+    GDN_TICK(0, 3);
+    // ---- T = (I + A)^-1 by blocks of 16: diagonal blocks by forward substitution, then block row r of block
+    // column c from  T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc),  one block diagonal at a time.  All fp32.
+    if (threadIdx.x < kC) {   // column j of the inverse of diagonal block b0: t_i = [i == j] - sum_{m<i} A_im t_m
+        const int b0 = (threadIdx.x >> 4) * 16, j = threadIdx.x & 15;
+        float t[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
             float s = (i == j) ? 1.f : 0.f;
-            for (int m = j; m < i; ++m) s = fmaf(-Af[i * 65 + m], Tf[m * 65 + j], s);
-            Tf[i * 65 + j] = (i >= j) ? s : 0.f;
+#pragma unroll
+            for (int m = 0; m < i; ++m) s = fmaf(-Af[(b0 + i) * 65 + b0 + m], t[m], s);
+            t[i] = s;
+            Tf[(b0 + i) * 65 + b0 + j] = s;
         }
     }
     __syncthreads();
+    inv_level<1>(Af, Tf, Sf);
+    inv_level<2>(Af, Tf, Sf);
+    inv_level<3>(Af, Tf, Sf);
+    GDN_TICK(0, 4);
     for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
         const int i = t >> 3, cch = t & 7;
         float a[8], b[8], w8[8];
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
-            const int m = cch * 8 + x;
-            a[x] = Tf[i * 65 + m];
-            b[x] = a[x] * bb[m] * Gam[m];
-            w8[x] = a[x] * ww[m];
+        for (int k = 0; k < 8; ++k) {
+            const int m = cch * 8 + k;
+            a[k] = Tf[i * 65 + m];
+            b[k] = a[k] * bb[m] * Gam[m];
+            w8[k] = a[k] * ww[m];
         }
-        *reinterpret_cast<uint4*>(sm + TT + tile_chunk_off(64, i, cch)) = pack8(a);
-        *reinterpret_cast<uint4*>(sm + TP + tile_chunk_off(64, i, cch)) = pack8(b);
-        *reinterpret_cast<uint4*>(sm + TPP + tile_chunk_off(64, i, cch)) = pack8(w8);
+        chunk_store(sm + TT, 64, i, cch, a);
+        chunk_store(sm + TP, 64, i, cch, b);
+        chunk_store(sm + TPP, 64, i, cch, w8);
     }
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(0, 5);
 
     // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T ; (P^T dO)^T = dO^T P
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + C_W, op_mn_major(sm + QK, 128, 64), op_k_major(sm + TP, 64), 128, 64, 64, false);
-        mma_tile(tmem + C_U, op_mn_major(sm + VO, 128, 0), op_k_major(sm + TPP, 64), 128, 64, 64, false);
-        if (bwd) mma_tile(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), 128, 64, 64, false);
+        mma_tile<128, 64, 64>(tmem + C_W, op_mn_major(sm + QK, 128, 64), op_k_major(sm + TP, 64), false);
+        mma_tile<128, 64, 64>(tmem + C_U, op_mn_major(sm + VO, 128, 0), op_k_major(sm + TPP, 64), false);
+        if (bwd) mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
-        bulk_store(p.ws + p.L.Tm + (size_t)ch * 8192, sm + TT, 8192);
+        bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
         bulk_commit();
     }
     // R = Diag(Gam) dO (token-major tile), while the MMAs run.  The fp32 A / T scratch is dead by now.
@@ -250,84 +357,76 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
         for (int t = threadIdx.x; t < kC * 16; t += blockDim.x) {
             const int i = t >> 4, cch = t & 15;
             float v[8];
-            unpack8(*reinterpret_cast<const uint4*>(sm + VO + tile_chunk_off(128, 64 + i, cch)), v);
+            chunk_load(sm + VO, 128, 64 + i, cch, v);
 #pragma unroll
-            for (int x = 0; x < 8; ++x) v[x] *= Gam[i];
-            *reinterpret_cast<uint4*>(sm + XR + tile_chunk_off(64, i, cch)) = pack8(v);
+            for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
+            chunk_store(sm + XR, 64, i, cch, v);
         }
     }
-    if (ok) { ok = mbar_wait(&bar_mma, mma_phase); mma_phase ^= 1; if (!ok && threadIdx.x == 0) report_timeout(p.ws, 3); }
-    tc_fence_after();
+    GDN_WAIT_MMA(3)
     if (ok) {
         const int f = q4 * 32 + lane, i0 = half * 32;
-        float v[32], ve[32];
-        tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_W + i0, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) ve[i] = v[i] * ee[i0 + i];
-        tile_store32(sm + WT, 128, f, i0, v);
-        tile_store32(sm + WET, 128, f, i0, ve);
-        tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_U + i0, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) ve[i] = v[i] * ee[i0 + i];
-        tile_store32(sm + UTT, 128, f, i0, v);
-        tile_store32(sm + UET, 128, f, i0, ve);
-        if (bwd) {
-            tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_PDO + i0, v);
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            const int ib = i0 + part * 8;
+            float v[8], ve[8];
+            tmem_ld8(tmem + lane_base + C_W + ib, v);
             tmem_wait_ld();
-            tile_store32(sm + XPDO, 128, f, i0, v);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ve[i] = v[i] * ee[ib + i];
+            chunk_store(sm + WT, 128, f, ib >> 3, v);
+            chunk_store(sm + WET, 128, f, ib >> 3, ve);
+            tmem_ld8(tmem + lane_base + C_U + ib, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ve[i] = v[i] * ee[ib + i];
+            chunk_store(sm + UTT, 128, f, ib >> 3, v);
+            chunk_store(sm + UET, 128, f, ib >> 3, ve);
+            if (bwd) {
+                tmem_ld8(tmem + lane_base + C_PDO + ib, v);
+                tmem_wait_ld();
+                chunk_store(sm + XPDO, 128, f, ib >> 3, v);
+            }
         }
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(0, 6);
 
     // ---- phase 3: Nm = K^T (Diag(e) W) ; Bf = K^T (Diag(e) U~) ; E = Q^T R - W^T (P^T dO)
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), 128, 128, 64, false);
-        mma_tile(tmem + C_BF, op_mn_major(sm + QK, 128, 64), op_k_major(sm + UET, 128), 128, 128, 64, false);
-        if (bwd) {
-            mma_tile(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), 128, 128, 64, false);
-            mma_tile(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), 128, 128, 64, true, /*neg_a=*/true);
-        }
+        mma_tile<128, 128, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
+        mma_tile<128, 128, 64>(tmem + C_BF, op_mn_major(sm + QK, 128, 64), op_k_major(sm + UET, 128), false);
+        if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
+        if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
-        bulk_store(p.ws + p.L.W + (size_t)ch * 16384, sm + WT, 16384);
-        bulk_store(p.ws + p.L.Ut + (size_t)ch * 16384, sm + UTT, 16384);
+        bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
+        bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
         bulk_commit();
     }
-    if (ok) { ok = mbar_wait(&bar_mma, mma_phase); mma_phase ^= 1; if (!ok && threadIdx.x == 0) report_timeout(p.ws, 4); }
-    tc_fence_after();
-    if (ok) {
+    GDN_WAIT_MMA(4)
+    GDN_TICK(0, 7);
+    if (ok) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
         const int r = q4 * 32 + lane, c0 = half * 64;
-        float v[32];
-        // Nm -> bf16 tile image (reuses the Q/K tile, which no MMA reads any more)
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_NM + c0 + part * 32, v);
+        const float sc = p.d.scale;
+#pragma unroll 1
+        for (int part = 0; part < 8; ++part) {
+            const int cb = c0 + part * 8;
+            float v[8];
+            tmem_ld8(tmem + lane_base + C_NM + cb, v);
             tmem_wait_ld();
-            tile_store32(sm + QK, 128, r, c0 + part * 32, v);
-        }
-        // Bf and E -> fp32, column-chunk-major: float4 index (col / 4) * 128 + row
-        float4* gB = reinterpret_cast<float4*>(p.ws + p.L.Bf + (size_t)ch * D * D * 4);
-        float4* gE = reinterpret_cast<float4*>(p.ws + p.L.E + (size_t)ch * D * D * 4);
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_BF + c0 + part * 32, v);
+            chunk_store(sm + QK, 128, r, cb >> 3, v);
+            tmem_ld8(tmem + lane_base + C_BF + cb, v);
             tmem_wait_ld();
-#pragma unroll
-            for (int x = 0; x < 8; ++x) gB[(size_t)((c0 + part * 32) / 4 + x) * D + r] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
-        }
-        if (bwd) {
-            const float sc = p.d.scale;
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + C_E + c0 + part * 32, v);
+            chunk_store(sm + VO, 128, r, cb >> 3, v);
+            if (bwd) {
+                tmem_ld8(tmem + lane_base + C_E + cb, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    gE[(size_t)((c0 + part * 32) / 4 + x) * D + r] = make_float4(sc * v[4 * x], sc * v[4 * x + 1], sc * v[4 * x + 2], sc * v[4 * x + 3]);
+                for (int k = 0; k < 8; ++k) v[k] *= sc;
+                chunk_store(sm + X, 128, r, cb >> 3, v);
             }
         }
     }
@@ -336,56 +435,64 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     __syncthreads();
     if (threadIdx.x == 0) {
         if (ok) {
-            bulk_store(p.ws + p.L.Nm + (size_t)ch * 32768, sm + QK, 32768);
+            bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + QK, 32768);
+            bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + VO, 32768);
+            if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768);
             bulk_commit();
         }
         bulk_wait_all<0>();   // shared memory must stay valid until every bulk store has read it
     }
+    GDN_TICK(0, 8);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------------
-// tc_scan: forward and reverse inter-chunk carries.
-// blockIdx.x = ((chain * 2 + direction) * 2 + slice); a CTA owns 64 columns of the 128 x 128 state.
-// Per chunk: the fp32 state (registers) is rounded to a bf16 tile, one tcgen05.mma forms Nm h (forward) or
-// Nm^T dh (reverse), and the state is updated in fp32:  s <- Gam_e s - (Nm s) + add.  The bf16 tile that fed
-// the MMA is also what the chunk's gradient stage needs, so it is bulk-stored to the workspace as it is.
+// tc_scan: forward and reverse inter-chunk carries, one CTA per (chain, direction).
+// Per chunk: the fp32 state (registers; thread = one row, 64 columns) is rounded to a bf16 tile, one tcgen05.mma
+// forms Nm h (forward) or Nm^T dh (reverse), and the state is updated in fp32:  s <- Gam_e s - (Nm s) + add.
+// The bf16 tile that fed the MMA is also what the chunk's gradient stage needs, so each thread writes its part
+// of the tile image to the workspace as well.  Nm and the additive term (Bf or E) arrive through a two-stage
+// ring of bulk copies; the chunk decays exp(gamma_e) are fetched once per chain.
 // ------------------------------------------------------------------------------------------------
 namespace scan {
 constexpr int STAGES = 2;
-constexpr uint32_t NM = 0;                       // ring of Nm tile images, 32 KB each
-constexpr uint32_t HT = NM + STAGES * 32768;     // two state tiles [128 rows][64 columns], 16 KB each
-constexpr uint32_t SMEM_BYTES = HT + 2 * 16384 + 1024;
+constexpr int GE_CAP = 2048;                     // chunk decays cached per chain (longer chains read them from global)
+constexpr uint32_t NM = 0;                       // ring: Nm tile image (32 KB) + additive-term image (32 KB) per stage
+constexpr uint32_t ADD = 32768;
+constexpr uint32_t STAGE_BYTES = 65536;
+constexpr uint32_t HT = STAGES * STAGE_BYTES;    // state tile [128][128], 32 KB
+constexpr uint32_t SMEM_BYTES = HT + 32768 + 1024;
+static_assert(SMEM_BYTES + GE_CAP * 4 <= 227 * 1024, "shared memory budget");
 }  // namespace scan
 
-__global__ void __launch_bounds__(kThreads, 2) tc_scan_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_constant__ TcParams P) {
     using namespace scan;
     const Problem& p = P.p;
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
     if (hdr->status != GDN_OK) return;
-    const int slice = blockIdx.x & 1;
-    const int reverse = P.scan_dirs == 2 ? ((blockIdx.x >> 1) & 1) : P.scan_dirs;
-    const int chain = P.scan_dirs == 2 ? (blockIdx.x >> 2) : (blockIdx.x >> 1);
+    const int reverse = P.scan_dirs == 2 ? (blockIdx.x & 1) : P.scan_dirs;
+    const int chain = P.scan_dirs == 2 ? (blockIdx.x >> 1) : blockIdx.x;
     const int n = chain / p.d.H, hd = chain % p.d.H;
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
     const int c0 = seq_first[n], c1 = seq_first[n + 1], nsteps = c1 - c0;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
+    __shared__ float ge[GE_CAP];
     __shared__ uint64_t bar_full[STAGES], bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, hf = warp >> 2;
     const int r = q4 * 32 + lane;              // state row owned by this thread
-    const int lc0 = hf * 32;                   // first of its 32 columns inside the CTA's slice
-    const int gc0 = slice * 64 + lc0;          // ... and inside the full state
+    const int gc0 = hf * 64;                   // first of its 64 columns
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) mbar_init(&bar_full[s], 1);
         mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 64); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 128); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -396,82 +503,94 @@ __global__ void __launch_bounds__(kThreads, 2) tc_scan_kernel(const __grid_const
     const char* add_base = p.ws + (reverse ? p.L.E : p.L.Bf);
     char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES && s < nsteps; ++s) {
-            mbar_expect_tx(&bar_full[s], 32768);
-            bulk_load(sm + NM + s * 32768, nm_base + ((size_t)chunk_of(s) * p.d.H + hd) * 32768, 32768, &bar_full[s]);
-        }
-    }
+    auto fill = [&](int s) {   // thread 0: bring chunk step s into ring slot s % STAGES
+        const int stage = s % STAGES;
+        const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
+        mbar_expect_tx(&bar_full[stage], 65536);
+        bulk_load(sm + stage * STAGE_BYTES + NM, nm_base + ch * 32768, 32768, &bar_full[stage]);
+        bulk_load(sm + stage * STAGE_BYTES + ADD, add_base + ch * 32768, 32768, &bar_full[stage]);
+    };
+    if (threadIdx.x == 0)
+        for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
+    for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
+        ge[s] = expf(gamma[((size_t)chunk_of(s) * p.d.H + hd) * kC + kC - 1]);
     // initial state
-    float st[32];
+    float st[64];
     {
         const float* init = reverse ? p.dhT : p.h0;
         const size_t soff = ((size_t)n * p.d.H + hd) * D * D + (size_t)r * D + gc0;
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
-            float4 v = init ? *reinterpret_cast<const float4*>(init + soff + 4 * x) : make_float4(0.f, 0.f, 0.f, 0.f);
-            st[4 * x] = v.x; st[4 * x + 1] = v.y; st[4 * x + 2] = v.z; st[4 * x + 3] = v.w;
+        for (int k = 0; k < 16; ++k) {
+            float4 v = init ? *reinterpret_cast<const float4*>(init + soff + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            st[4 * k] = v.x; st[4 * k + 1] = v.y; st[4 * k + 2] = v.z; st[4 * k + 3] = v.w;
         }
     }
+    __syncthreads();
     bool ok = true;
     uint32_t mma_phase = 0;
+    unsigned char* Ht = sm + HT;
+#pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
         const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
-        const int stage = s % STAGES, hb = s & 1;
-        unsigned char* Ht = sm + HT + hb * 16384;
-        const float Ge = expf(gamma[ch * kC + kC - 1]);
-        float4 add[8];
-        const float4* ga = reinterpret_cast<const float4*>(add_base + ch * D * D * 4);
+        const int stage = s % STAGES;
+        const unsigned char* ring = sm + stage * STAGE_BYTES;
+        if (s < 4) GDN_TICK(1, s * 5 + 0);
+        const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
+        uint4 packed[8];   // state -> bf16: operand tile of the MMA and the stored per-chunk state
 #pragma unroll
-        for (int x = 0; x < 8; ++x) add[x] = ga[(size_t)(gc0 / 4 + x) * D + r];
-        tile_store32(Ht, 128, r, lc0, st);
+        for (int k = 0; k < 8; ++k) {
+            packed[k] = pack8(st + 8 * k);
+            *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, hf * 8 + k)) = packed[k];
+        }
         fence_async_smem();
         __syncthreads();
+        if (s < 4) GDN_TICK(1, s * 5 + 1);
         if (threadIdx.x == 0) {
+            // every thread has finished step s - 1, so its ring slot can take step s - 1 + STAGES
+            if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
             ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
             if (ok) {
                 tc_fence_after();
-                const Operand a = reverse ? op_mn_major(sm + NM + stage * 32768, 128) : op_k_major(sm + NM + stage * 32768, 128);
-                mma_tile(tmem, a, op_mn_major(Ht, 128), 128, 64, 128, false);
+                const Operand a = reverse ? op_mn_major(ring + NM, 128) : op_k_major(ring + NM, 128);
+                mma_tile<128, 128, 128>(tmem, a, op_mn_major(Ht, 128), false);
             } else {
                 report_timeout(p.ws, 10);
             }
-            bulk_store(keep_base + ch * 32768 + slice * 16384, Ht, 16384);
-            bulk_commit();
-            bulk_wait_read<1>();   // the store issued one step ago has finished reading the other state tile
             mma_commit(&bar_mma);
         }
-        ok = mbar_wait(&bar_mma, mma_phase);
+        {   // the same bytes go to the workspace while the MMA runs (after the fence: it would wait for these stores)
+            char* keep = keep_base + ch * 32768;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(keep + tile_chunk_off(128, r, hf * 8 + k)) = packed[k];
+        }
+        if (s < 4) GDN_TICK(1, s * 5 + 2);
+        ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);   // the additive term of this step is in shared memory
+        if (ok) ok = mbar_wait(&bar_mma, mma_phase);
         mma_phase ^= 1;
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 11); break; }
         tc_fence_after();
-        float dl[32];
-        tmem_ld32(tmem + ((uint32_t)(q4 * 32) << 16) + lc0, dl);
-        tmem_wait_ld();
+        if (s < 4) GDN_TICK(1, s * 5 + 3);
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
-            st[4 * x + 0] = fmaf(Ge, st[4 * x + 0], add[x].x - dl[4 * x + 0]);
-            st[4 * x + 1] = fmaf(Ge, st[4 * x + 1], add[x].y - dl[4 * x + 1]);
-            st[4 * x + 2] = fmaf(Ge, st[4 * x + 2], add[x].z - dl[4 * x + 2]);
-            st[4 * x + 3] = fmaf(Ge, st[4 * x + 3], add[x].w - dl[4 * x + 3]);
+        for (int k = 0; k < 8; ++k) {
+            float dl[8], ad[8];
+            tmem_ld8(tmem + lane_base + gc0 + 8 * k, dl);
+            chunk_load(ring + ADD, 128, r, hf * 8 + k, ad);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) st[8 * k + j] = fmaf(Ge, st[8 * k + j], ad[j] - dl[j]);
         }
+        if (s < 4) GDN_TICK(1, s * 5 + 4);
         tc_fence_before();
-        if (threadIdx.x == 0 && s + STAGES < nsteps) {   // the MMA that read this ring slot has completed
-            mbar_expect_tx(&bar_full[stage], 32768);
-            bulk_load(sm + NM + stage * 32768, nm_base + ((size_t)chunk_of(s + STAGES) * p.d.H + hd) * 32768, 32768, &bar_full[stage]);
-        }
     }
     float* fin = reverse ? p.dh0 : p.hT;
     if (fin && ok) {
         const size_t soff = ((size_t)n * p.d.H + hd) * D * D + (size_t)r * D + gc0;
 #pragma unroll
-        for (int x = 0; x < 8; ++x) *reinterpret_cast<float4*>(fin + soff + 4 * x) = make_float4(st[4 * x], st[4 * x + 1], st[4 * x + 2], st[4 * x + 3]);
+        for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
     }
-    if (threadIdx.x == 0) bulk_wait_all<0>();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 64);
+    if (warp == 0) tmem_dealloc(tmem, 128);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -489,57 +608,40 @@ __global__ void __launch_bounds__(kThreads, 2) tc_scan_kernel(const __grid_const
 // The decay gradient uses the identities  rowsum(dP.P) + scale Gam <q, dO h^T> = <q, dq>  and its analogues for
 // k:  dgamma_i = <q_i, dq_i> + <k_i, dk_i^row> - <k_i, dk_i^col>, where dk^row = Diag(b)(G K + Diag(Gam) dXk)
 // collects the terms in which k_i enters with exp(+gamma_i) and dk^col those with exp(-gamma_i); the last row
-// of the chunk adds sum_j r_j + Gam_e <dh', h> (r_j = <(Kb dh')_j, U_j>).
+// of the chunk adds sum_j r_j + Gam_e <dh', h> (r_j = <(Kb dh')_j, U_j>).  Outputs are staged in shared memory
+// as token-major tiles and written with 16-byte stores.
 // ------------------------------------------------------------------------------------------------
 namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
 constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB
-constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
+constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64], then staged dq / dk
 constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
 constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk^T, dXv^T [128][64] each
 constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
-constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G, Diag(b) G [64][64] each
+constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later staged dv, then G and Diag(b) G
 constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DO, DXKT = HH, DXVT = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
+constexpr uint32_t DWT = DO, DXKT = HH, DXVT = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192, STG_QK = DO, STG_V = UT;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-__host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns in 512 TMEM columns
+__host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
-
-// Sum v[t] over the 32 lanes of a warp for 32 values at once; lane l ends with the total of index l in v[0].
-__device__ __forceinline__ void butterfly32(float (&v)[32], int lane) {
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const bool up = (lane & off) != 0;
-#pragma unroll
-        for (int k = 0; k < off; ++k) {
-            const float send = up ? v[k] : v[k + off];
-            const float keep = up ? v[k + off] : v[k];
-            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-    }
-}
 
 __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
     using namespace intra;
     const Problem& p = P.p;
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    const int c = blockIdx.x / p.d.H, hd = blockIdx.x % p.d.H;
-    if (c >= hdr->n_chunks) return;
-    const int ch = blockIdx.x;
-    const int tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[c];
-    const int len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[c];
+    ChunkInfo x;
+    if (!chunk_info(p, x)) return;
     const int H = p.d.H;
     const float sc = p.d.scale;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gam[kC], Gam[kC], ee[kC], bb[kC];
-    __shared__ float red1[2][4][32], red2[2][4][32], red3[2][4][32];
-    __shared__ float dws[kC], dgam[kC], scal[2][kThreads / 32];
+    __shared__ float gl[kC], Gam[kC], ee[kC], bb[kC];
+    __shared__ float red[4][2][4][32];       // four token-wise reductions: [which][column half][lane quadrant][token]
+    __shared__ float dgam[kC], scal[2][kThreads / 32];
     __shared__ uint64_t bar_in0, bar_in1, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -557,266 +659,283 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     const uint32_t tmem = tmem_slot;
     bool ok = true;
     uint32_t mma_phase = 0;
+    GDN_TICK(2, 0);
 
     if (threadIdx.x == 0) {
         mbar_expect_tx(&bar_in0, 32768 + 16384 + 32768 + 32768);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, hd * D + cb * 64, tok0, &bar_in0);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, hd * D + cb * 64, tok0, &bar_in0);
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_in0);
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in0);
         }
-        bulk_load(sm + WT, p.ws + p.L.W + (size_t)ch * 16384, 16384, &bar_in0);
-        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)ch * 32768, 32768, &bar_in0);
-        bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)ch * 32768, 32768, &bar_in0);
+        bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in0);
+        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in0);
+        bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)x.ch * 32768, 32768, &bar_in0);
         mbar_expect_tx(&bar_in1, 16384 + 16384 + 16384 + 8192);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + VT + cb * 8192, &P.tm_v, hd * D + cb * 64, tok0, &bar_in1);
-            tma_load_2d(sm + DO + cb * 8192, &P.tm_do, hd * D + cb * 64, tok0, &bar_in1);
+            tma_load_2d(sm + VT + cb * 8192, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_in1);
+            tma_load_2d(sm + DO + cb * 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_in1);
         }
-        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)ch * 16384, 16384, &bar_in1);
-        bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)ch * 8192, 8192, &bar_in1);
+        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in1);
+        bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)x.ch * 8192, 8192, &bar_in1);
     }
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
-        const float g = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)ch * kC + i];
-        gam[i] = g;
+        const float* gsrc = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC;
+        const float g = gsrc[i], gend = gsrc[kC - 1];
+        gl[i] = g * kLog2e;
         Gam[i] = expf(g);
-        bb[i] = (i < len) ? p.beta[(size_t)(tok0 + i) * H + hd] : 0.f;
+        ee[i] = expf(gend - g);
+        bb[i] = (i < x.len) ? p.beta[(size_t)(x.tok0 + i) * H + x.hd] : 0.f;
     }
-    __syncthreads();
-    if (threadIdx.x < kC) ee[threadIdx.x] = expf(gam[kC - 1] - gam[threadIdx.x]);
     ok = mbar_wait(&bar_in0, 0) && mbar_wait(&bar_in1, 0);
     if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
-    if (ok && len < kC) {
-        zero_tail_rows(sm + QK, 128, 0, len);
-        zero_tail_rows(sm + QK, 128, 64, len);
-        zero_tail_rows(sm + VT, 64, 0, len);
-        zero_tail_rows(sm + DO, 64, 0, len);
+    if (ok && x.len < kC) {
+        zero_tail_rows(sm + QK, 128, 0, x.len);
+        zero_tail_rows(sm + QK, 128, 64, x.len);
+        zero_tail_rows(sm + VT, 64, 0, x.len);
+        zero_tail_rows(sm + DO, 64, 0, x.len);
         fence_async_smem();
     }
     __syncthreads();
-    auto Dij = [&](int i, int j) -> float { return expf(gam[i] - gam[j]); };   // only for j <= i
-#define GDN_WAIT_MMA(where)                                                                         \
-    if (ok) {                                                                                       \
-        ok = mbar_wait(&bar_mma, mma_phase);                                                        \
-        mma_phase ^= 1;                                                                             \
-        if (!ok && threadIdx.x == 0) report_timeout(p.ws, where);                                   \
-    }                                                                                               \
-    tc_fence_after();
+    GDN_TICK(2, 1);
 
     // ---- phase 1
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(0), op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), 64, 64, 128, false);
-        mma_tile(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), 128, 64, 128, false);
-        mma_tile(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), 128, 64, 128, false);
+        mma_tile<64, 64, 128>(tmem + slot(0), op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
+        mma_tile<128, 64, 128>(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
+        mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
         mma_commit(&bar_mma);
     }
     // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up)
     float hh = 0.f;
+#pragma unroll 1
     for (int t = threadIdx.x; t < 2048; t += blockDim.x) {
         float a[8], b[8];
         unpack8(*reinterpret_cast<const uint4*>(sm + HH + t * 16), a);
         unpack8(*reinterpret_cast<const uint4*>(sm + DH + t * 16), b);
 #pragma unroll
-        for (int x = 0; x < 8; ++x) hh = fmaf(a[x], b[x], hh);
+        for (int k = 0; k < 8; ++k) hh = fmaf(a[k], b[k], hh);
     }
+    GDN_TICK(2, 2);
     GDN_WAIT_MMA(21)
-    if (ok) {   // P_ij = (q_i . k_j) D_ij for j <= i   (M = 64 accumulator: row i on lane (i % 16) + 32 (i / 16))
-        float v[32];
-        tmem_ld32(tmem + lane_base + slot(0) + half * 32, v);
-        tmem_wait_ld();
-        const int i = q4 * 16 + lane, j0 = half * 32;
-        if (lane < 16) {
+    GDN_TICK(2, 3);
+    const int mi = q4 * 16 + lane;     // row of an M = 64 accumulator held by this lane (lanes 0..15 only)
+    const int j0 = half * 32;
+    if (ok) {   // P_ij = (q_i . k_j) D_ij for j <= i
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            float v[8];
+            const int jb = j0 + part * 8;
+            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
+            tmem_wait_ld();
+            if (lane < 16) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (j0 + j <= i) ? v[j] * Dij(i, j0 + j) : 0.f;
-            tile_store32(sm + PT, 64, i, j0, v);
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                chunk_store(sm + PT, 64, mi, jb >> 3, v);
+            }
         }
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(2, 4);
 
     // ---- phase 2
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(3), op_mn_major(sm + DO, 64), op_mn_major(sm + PT, 64), 128, 64, 64, false);
+        mma_tile<128, 64, 64>(tmem + slot(3), op_mn_major(sm + DO, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
     }
+    GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
     const int f = q4 * 32 + lane;      // feature (lane of the transposed accumulators)
     const int i0 = half * 32;          // first of this thread's 32 tokens
     float rs = 0.f;
     if (ok) {
-        float u[32], t[32];
-        tile_load32(sm + UTT, 128, f, i0, u);
-        tmem_ld32(tmem + lane_base + slot(1) + i0, t);
-        tmem_wait_ld();
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            const int ib = i0 + part * 8;
+            float u[8], t[8], kb[8], pd[8];
+            chunk_load(sm + UTT, 128, f, ib >> 3, u);
+            tmem_ld8(tmem + lane_base + slot(1) + ib, t);
+            tmem_ld8(tmem + lane_base + slot(2) + ib, kb);
+            tmem_ld8(tmem + lane_base + slot(3) + ib, pd);
+            tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) u[i] -= t[i];                       // U = U~ - W h
-        tile_store32(sm + UT, 128, f, i0, u);
-        float kb[32];
-        tmem_ld32(tmem + lane_base + slot(2) + i0, kb);
-        tmem_ld32(tmem + lane_base + slot(3) + i0, t);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const float kbe = ee[i0 + i] * kb[i];
-            rs = fmaf(kbe, u[i], rs);                                     // sum_j r_j
-            t[i] = fmaf(sc, t[i], kbe);                                   // dU = scale P^T dO + Diag(e) K dh'
+            for (int i = 0; i < 8; ++i) {
+                u[i] -= t[i];                                       // U = U~ - W h
+                const float kbe = ee[ib + i] * kb[i];
+                rs = fmaf(kbe, u[i], rs);                           // sum_j r_j
+                pd[i] = fmaf(sc, pd[i], kbe);                       // dU = scale P^T dO + Diag(e) K dh'
+            }
+            chunk_store(sm + UT, 128, f, ib >> 3, u);
+            chunk_store(sm + DUT, 128, f, ib >> 3, pd);
         }
-        tile_store32(sm + DUT, 128, f, i0, t);
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(2, 6);
 
     // ---- phase 3
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(0), op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), 64, 64, 128, false);
-        mma_tile(tmem + slot(4), op_k_major(sm + HH, 128), op_k_major(sm + DO, 64), 128, 64, 128, false);
-        mma_tile(tmem + slot(5), op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), 128, 64, 128, false, /*neg_a=*/true);
+        mma_tile<64, 64, 128>(tmem + slot(0), op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);
+        mma_tile<128, 64, 128>(tmem + slot(4), op_k_major(sm + HH, 128), op_k_major(sm + DO, 64), false);
+        mma_tile<128, 64, 128>(tmem + slot(5), op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
         mma_commit(&bar_mma);
     }
+    GDN_TICK(2, 7);
     GDN_WAIT_MMA(23)
     if (ok) {
-        float v[32];
-        tmem_ld32(tmem + lane_base + slot(0) + half * 32, v);
-        tmem_wait_ld();
-        const int i = q4 * 16 + lane, j0 = half * 32;
-        if (lane < 16) {   // dPD = scale tril(dO U^T) . D
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            float v[8], w[8];
+            const int jb = j0 + part * 8, ib = i0 + part * 8;
+            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
+            tmem_ld8(tmem + lane_base + slot(5) + ib, w);
+            tmem_wait_ld();
+            if (lane < 16) {   // dPD = scale tril(dO U^T) . D
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (j0 + j <= i) ? sc * v[j] * Dij(i, j0 + j) : 0.f;
-            tile_store32(sm + DPD, 64, i, j0, v);
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? sc * v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                chunk_store(sm + DPD, 64, mi, jb >> 3, v);
+            }
+            chunk_store(sm + DWT, 128, f, ib >> 3, w);              // dW^T = -(dU h^T)^T
         }
-        tmem_ld32(tmem + lane_base + slot(5) + i0, v);
-        tmem_wait_ld();
-        tile_store32(sm + DWT, 128, f, i0, v);                            // dW^T = -(dU h^T)^T
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(2, 8);
 
     // ---- phase 4
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(1), op_mn_major(sm + QK, 128, 64), op_k_major(sm + DPD, 64), 128, 64, 64, false);
-        mma_tile(tmem + slot(2), op_k_major(sm + DWT, 128), op_mn_major(sm + TT, 64), 128, 64, 64, false);
-        mma_tile(tmem + slot(3), op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), 128, 64, 64, false);
-        mma_tile(tmem + slot(6), op_mn_major(sm + QK, 128, 0), op_mn_major(sm + DPD, 64), 128, 64, 64, false);
-        mma_tile(tmem + slot(7), op_k_major(sm + DH, 128), op_mn_major(sm + UT, 128), 128, 64, 128, false);
+        mma_tile<128, 64, 64>(tmem + slot(1), op_mn_major(sm + QK, 128, 64), op_k_major(sm + DPD, 64), false);
+        mma_tile<128, 64, 64>(tmem + slot(2), op_k_major(sm + DWT, 128), op_mn_major(sm + TT, 64), false);
+        mma_tile<128, 64, 64>(tmem + slot(3), op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), false);
+        mma_tile<128, 64, 64>(tmem + slot(6), op_mn_major(sm + QK, 128, 0), op_mn_major(sm + DPD, 64), false);
+        mma_tile<128, 64, 128>(tmem + slot(7), op_k_major(sm + DH, 128), op_mn_major(sm + UT, 128), false);
         mma_commit(&bar_mma);
     }
+    GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
-    float acc1[32];   // <q, dq> - <k, dk^col> per token, this thread's feature only
-#pragma unroll
-    for (int i = 0; i < 32; ++i) acc1[i] = 0.f;
-    __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((size_t)tok0 * H + hd) * D + f;
-    __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + ((size_t)tok0 * H + hd) * D + f;
-    __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + ((size_t)tok0 * H + hd) * D + f;
+    __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((size_t)x.tok0 * H + x.hd) * D;
+    __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + ((size_t)x.tok0 * H + x.hd) * D;
+    __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + ((size_t)x.tok0 * H + x.hd) * D;
     const size_t rowp = (size_t)H * D;
     if (ok) {
-        float a[32], b[32];
-        tmem_ld32(tmem + lane_base + slot(4) + i0, a);
-        tmem_ld32(tmem + lane_base + slot(1) + i0, b);
-        tmem_wait_ld();
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            const int ib = i0 + part * 8;
+            float a[8], b[8], xk[8], xv[8];
+            tmem_ld8(tmem + lane_base + slot(4) + ib, a);
+            tmem_ld8(tmem + lane_base + slot(1) + ib, b);
+            tmem_ld8(tmem + lane_base + slot(2) + ib, xk);
+            tmem_ld8(tmem + lane_base + slot(3) + ib, xv);
+            tmem_wait_ld();
+            chunk_store(sm + DXKT, 128, f, ib >> 3, xk);
+            chunk_store(sm + DXVT, 128, f, ib >> 3, xv);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const float dq = fmaf(sc * Gam[i0 + i], a[i], b[i]);          // dq = scale Gam (dO h^T) + dPD K
-            acc1[i] = tile_get(sm + QK, 128, i0 + i, f) * dq;
-            if (i0 + i < len) gdq[(size_t)(i0 + i) * rowp] = __float2bfloat16_rn(dq);
+            for (int i = 0; i < 8; ++i) {
+                const float dq = fmaf(sc * Gam[ib + i], a[i], b[i]);   // dq = scale Gam (dO h^T) + dPD K
+                tile_put(sm + STG_QK, 64, ib + i, f, dq);
+                a[i] = tile_get(sm + QK, 128, ib + i, f) * dq;          // <q, dq> partial
+                tile_put(sm + STG_V, 64, ib + i, f, bb[ib + i] * xv[i]);  // dv = w dXv
+                xv[i] *= tile_get(sm + VT, 64, ib + i, f);              // dw partial
+            }
+            const float s0 = reduce8(a, lane), s1 = reduce8(xv, lane);
+            if (lane < 8) { red[0][half][q4][part * 8 + lane] = s0; red[1][half][q4][part * 8 + lane] = s1; }
         }
-        tmem_ld32(tmem + lane_base + slot(2) + i0, a);
-        tmem_ld32(tmem + lane_base + slot(3) + i0, b);
-        tmem_wait_ld();
-        tile_store32(sm + DXKT, 128, f, i0, a);
-        tile_store32(sm + DXVT, 128, f, i0, b);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            if (i0 + i < len) gdv[(size_t)(i0 + i) * rowp] = __float2bfloat16_rn(bb[i0 + i] * b[i]);   // dv = w dXv
-            b[i] *= tile_get(sm + VT, 64, i0 + i, f);                                             // dw partial
-        }
-        butterfly32(b, lane);
-        red1[half][q4][lane] = b[0];
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
-    if (threadIdx.x < kC) {
-        const int hf = threadIdx.x >> 5, l = threadIdx.x & 31;
-        dws[threadIdx.x] = (red1[hf][0][l] + red1[hf][1][l]) + (red1[hf][2][l] + red1[hf][3][l]);
-    }
+    GDN_TICK(2, 10);
 
-    // ---- phase 5
+    // ---- phase 5 (the staged dq and dv leave while the MMAs run)
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(0), op_mn_major(sm + DXKT, 128), op_mn_major(sm + WT, 128), 64, 64, 128, false);
-        mma_tile(tmem + slot(0), op_mn_major(sm + DXVT, 128), op_mn_major(sm + UTT, 128), 64, 64, 128, true);
+        mma_tile<64, 64, 128>(tmem + slot(0), op_mn_major(sm + DXKT, 128), op_mn_major(sm + WT, 128), false);
+        mma_tile<64, 64, 128>(tmem + slot(0), op_mn_major(sm + DXVT, 128), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
     }
+    if (ok) {
+        flush_rows(sm + STG_QK, gdq, rowp, x.len);
+        flush_rows(sm + STG_V, gdv, rowp, x.len);
+    }
+    __syncthreads();   // the staging tiles are rewritten below
+    GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
     if (ok) {
-        float v[32], w[32];
-        tmem_ld32(tmem + lane_base + slot(0) + half * 32, v);
-        tmem_wait_ld();
-        const int i = q4 * 16 + lane, j0 = half * 32;
-        if (lane < 16) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            float v[8], w[8];
+            const int jb = j0 + part * 8;
+            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
+            tmem_wait_ld();
+            if (lane < 16) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                v[j] = (j0 + j < i) ? -v[j] * Dij(i, j0 + j) : 0.f;
-                w[j] = bb[i] * v[j];
+                for (int j = 0; j < 8; ++j) {
+                    v[j] = (jb + j < mi) ? -v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                    w[j] = bb[mi] * v[j];
+                }
+                chunk_store(sm + GT, 64, mi, jb >> 3, v);
+                chunk_store(sm + BGT, 64, mi, jb >> 3, w);
             }
-            tile_store32(sm + GT, 64, i, j0, v);
-            tile_store32(sm + BGT, 64, i, j0, w);
         }
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    GDN_TICK(2, 12);
 
     // ---- phase 6
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + slot(4), op_mn_major(sm + QK, 128, 64), op_k_major(sm + GT, 64), 128, 64, 64, false);
-        mma_tile(tmem + slot(6), op_mn_major(sm + QK, 128, 64), op_mn_major(sm + BGT, 64), 128, 64, 64, true);
+        mma_tile<128, 64, 64>(tmem + slot(4), op_mn_major(sm + QK, 128, 64), op_k_major(sm + GT, 64), false);
+        mma_tile<128, 64, 64>(tmem + slot(6), op_mn_major(sm + QK, 128, 64), op_mn_major(sm + BGT, 64), true);
         mma_commit(&bar_mma);
     }
+    GDN_TICK(2, 13);
     GDN_WAIT_MMA(26)
     if (ok) {
-        float y[32], t[32];
-        tmem_ld32(tmem + lane_base + slot(4) + i0, y);
-        tmem_ld32(tmem + lane_base + slot(2) + i0, t);
-        tmem_wait_ld();
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            const int ib = i0 + part * 8;
+            float y[8], t[8], c1[8], c2[8];
+            tmem_ld8(tmem + lane_base + slot(4) + ib, y);
+            tmem_ld8(tmem + lane_base + slot(2) + ib, t);
+            tmem_ld8(tmem + lane_base + slot(6) + ib, c1);
+            tmem_ld8(tmem + lane_base + slot(7) + ib, c2);
+            tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) y[i] = fmaf(Gam[i0 + i], t[i], y[i]);     // Y = G K + Diag(Gam) dXk ; dk^row = Diag(b) Y
-        float c2[32];
-        tmem_ld32(tmem + lane_base + slot(6) + i0, t);
-        tmem_ld32(tmem + lane_base + slot(7) + i0, c2);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const float kcol = fmaf(ee[i0 + i], c2[i], t[i]);                   // dk^col
-            const float kk = tile_get(sm + QK, 128, 64 + i0 + i, f);
-            if (i0 + i < len) gdk[(size_t)(i0 + i) * rowp] = __float2bfloat16_rn(fmaf(bb[i0 + i], y[i], kcol));
-            acc1[i] = fmaf(-kk, kcol, acc1[i]);
-            y[i] *= kk;                                                         // db partial
+            for (int i = 0; i < 8; ++i) {
+                const float yy = fmaf(Gam[ib + i], t[i], y[i]);        // Y = G K + Diag(Gam) dXk ; dk^row = Diag(b) Y
+                const float kcol = fmaf(ee[ib + i], c2[i], c1[i]);      // dk^col
+                const float kk = tile_get(sm + QK, 128, 64 + ib + i, f);
+                tile_put(sm + STG_QK, 64, ib + i, f, fmaf(bb[ib + i], yy, kcol));
+                y[i] = kk * yy;                                         // db partial
+                c1[i] = kk * kcol;                                      // <k, dk^col> partial
+            }
+            const float s2 = reduce8(y, lane), s3 = reduce8(c1, lane);
+            if (lane < 8) { red[2][half][q4][part * 8 + lane] = s2; red[3][half][q4][part * 8 + lane] = s3; }
         }
-        butterfly32(y, lane);
-        butterfly32(acc1, lane);
-        red2[half][q4][lane] = y[0];
-        red3[half][q4][lane] = acc1[0];
     }
     // block totals of sum_j r_j and <dh', h>
     rs = warp_sum(rs);
     hh = warp_sum(hh);
     if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
     __syncthreads();
+    GDN_TICK(2, 14);
+    if (ok) flush_rows(sm + STG_QK, gdk, rowp, x.len);
     if (threadIdx.x < kC) {
         const int i = threadIdx.x, hf = i >> 5, l = i & 31;
-        const float db = (red2[hf][0][l] + red2[hf][1][l]) + (red2[hf][2][l] + red2[hf][3][l]);
-        const float d1 = (red3[hf][0][l] + red3[hf][1][l]) + (red3[hf][2][l] + red3[hf][3][l]);
-        if (i < len) p.dbeta[(size_t)(tok0 + i) * H + hd] = db + dws[i];
-        dgam[i] = fmaf(bb[i], db, d1);
+        auto tot = [&](int w) { return (red[w][hf][0][l] + red[w][hf][1][l]) + (red[w][hf][2][l] + red[w][hf][3][l]); };
+        const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
+        if (i < x.len) p.dbeta[(size_t)(x.tok0 + i) * H + x.hd] = db + dw;
+        dgam[i] = fmaf(bb[i], db, qdq - kcol);
     }
     __syncthreads();
     if (threadIdx.x == 0 && ok) {
@@ -826,36 +945,32 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
         float run = 0.f;   // gam_i = sum_{j<=i} g_j  =>  dg_j = sum_{i>=j} dgam_i
         for (int i = kC - 1; i >= 0; --i) {
             run += dgam[i];
-            if (i < len) p.dg[(size_t)(tok0 + i) * H + hd] = run;
+            if (i < x.len) p.dg[(size_t)(x.tok0 + i) * H + x.hd] = run;
         }
     }
     tc_fence_before();
     __syncthreads();
+    GDN_TICK(2, 15);
     if (warp == 0) tmem_dealloc(tmem, 512);
-#undef GDN_WAIT_MMA
 }
 
 // ------------------------------------------------------------------------------------------------
 // tc_out (optional forward output): o = scale (Diag(Gam) Q h + P (U~ - W h))
 // ------------------------------------------------------------------------------------------------
 namespace outk {
-constexpr uint32_t QK = 0, WT = 32768, UTT = WT + 16384, HH = UTT + 16384, PT = HH + 32768, UT = PT + 8192;
-constexpr uint32_t SMEM_BYTES = UT + 16384 + 1024;
+constexpr uint32_t QK = 0, WT = 32768, UTT = WT + 16384, HH = UTT + 16384, PT = HH + 32768, UT = PT + 8192, STG = UT + 16384;
+constexpr uint32_t SMEM_BYTES = STG + 16384 + 1024;
 }  // namespace outk
 
 __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_constant__ TcParams P) {
     using namespace outk;
     const Problem& p = P.p;
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    const int c = blockIdx.x / p.d.H, hd = blockIdx.x % p.d.H;
-    if (c >= hdr->n_chunks) return;
-    const int ch = blockIdx.x;
-    const int tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[c];
-    const int len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[c];
+    ChunkInfo x;
+    if (!chunk_info(p, x)) return;
     const int H = p.d.H;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gam[kC];
+    __shared__ float gl[kC], Gam[kC];
     __shared__ uint64_t bar_in, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -870,74 +985,84 @@ __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_consta
     if (threadIdx.x == 0) {
         mbar_expect_tx(&bar_in, 32768 + 16384 + 16384 + 32768);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, hd * D + cb * 64, tok0, &bar_in);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, hd * D + cb * 64, tok0, &bar_in);
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_in);
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in);
         }
-        bulk_load(sm + WT, p.ws + p.L.W + (size_t)ch * 16384, 16384, &bar_in);
-        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)ch * 16384, 16384, &bar_in);
-        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)ch * 32768, 32768, &bar_in);
+        bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in);
+        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in);
+        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in);
     }
-    if (threadIdx.x < kC) gam[threadIdx.x] = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)ch * kC + threadIdx.x];
+    if (threadIdx.x < kC) {
+        const float g = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + threadIdx.x];
+        gl[threadIdx.x] = g * kLog2e;
+        Gam[threadIdx.x] = expf(g);
+    }
     bool ok = mbar_wait(&bar_in, 0);
+    uint32_t mma_phase = 0;
     if (!ok && threadIdx.x == 0) report_timeout(p.ws, 30);
-    if (ok && len < kC) {
-        zero_tail_rows(sm + QK, 128, 0, len);
-        zero_tail_rows(sm + QK, 128, 64, len);
+    if (ok && x.len < kC) {
+        zero_tail_rows(sm + QK, 128, 0, x.len);
+        zero_tail_rows(sm + QK, 128, 64, x.len);
         fence_async_smem();
     }
     __syncthreads();
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + 0, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), 64, 64, 128, false);
-        mma_tile(tmem + 64, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), 128, 64, 128, false);
-        mma_tile(tmem + 128, op_mn_major(sm + HH, 128), op_k_major(sm + QK, 128, 0), 128, 64, 128, false);
+        mma_tile<64, 64, 128>(tmem + 0, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
+        mma_tile<128, 64, 128>(tmem + 64, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
+        mma_tile<128, 64, 128>(tmem + 128, op_mn_major(sm + HH, 128), op_k_major(sm + QK, 128, 0), false);
         mma_commit(&bar_mma);
     }
-    if (ok) { ok = mbar_wait(&bar_mma, 0); if (!ok && threadIdx.x == 0) report_timeout(p.ws, 31); }
-    tc_fence_after();
-    const int f = q4 * 32 + lane, i0 = half * 32;
+    GDN_WAIT_MMA(31)
+    const int f = q4 * 32 + lane, i0 = half * 32, mi = q4 * 16 + lane, j0 = half * 32;
     if (ok) {
-        float v[32], u[32];
-        tmem_ld32(tmem + lane_base + 0 + half * 32, v);
-        tmem_wait_ld();
-        const int i = q4 * 16 + lane, j0 = half * 32;
-        if (lane < 16) {
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            float v[8], u[8], t[8];
+            const int jb = j0 + part * 8, ib = i0 + part * 8;
+            tmem_ld8(tmem + lane_base + 0 + jb, v);
+            tmem_ld8(tmem + lane_base + 64 + ib, t);
+            chunk_load(sm + UTT, 128, f, ib >> 3, u);
+            tmem_wait_ld();
+            if (lane < 16) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (j0 + j <= i) ? v[j] * expf(gam[i] - gam[j0 + j]) : 0.f;
-            tile_store32(sm + PT, 64, i, j0, v);
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                chunk_store(sm + PT, 64, mi, jb >> 3, v);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) u[i] -= t[i];
+            chunk_store(sm + UT, 128, f, ib >> 3, u);
         }
-        tile_load32(sm + UTT, 128, f, i0, u);
-        tmem_ld32(tmem + lane_base + 64 + i0, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i2 = 0; i2 < 32; ++i2) u[i2] -= v[i2];
-        tile_store32(sm + UT, 128, f, i0, u);
     }
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile(tmem + 192, op_k_major(sm + UT, 128), op_k_major(sm + PT, 64), 128, 64, 64, false);
+        mma_tile<128, 64, 64>(tmem + 192, op_k_major(sm + UT, 128), op_k_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
     }
-    if (ok) { ok = mbar_wait(&bar_mma, 1); if (!ok && threadIdx.x == 0) report_timeout(p.ws, 32); }
-    tc_fence_after();
+    GDN_WAIT_MMA(32)
     if (ok) {
-        float a[32], b[32];
-        tmem_ld32(tmem + lane_base + 128 + i0, a);
-        tmem_ld32(tmem + lane_base + 192 + i0, b);
-        tmem_wait_ld();
-        __nv_bfloat16* go = reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)tok0 * H + hd) * D + f;
         const float sc = p.d.scale;
+#pragma unroll 1
+        for (int part = 0; part < 4; ++part) {
+            const int ib = i0 + part * 8;
+            float a[8], b[8];
+            tmem_ld8(tmem + lane_base + 128 + ib, a);
+            tmem_ld8(tmem + lane_base + 192 + ib, b);
+            tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            if (i0 + i < len) go[(size_t)(i0 + i) * H * D] = __float2bfloat16_rn(sc * fmaf(expf(gam[i0 + i]), a[i], b[i]));
+            for (int i = 0; i < 8; ++i) tile_put(sm + STG, 64, ib + i, f, sc * fmaf(Gam[ib + i], a[i], b[i]));
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (ok) flush_rows(sm + STG, reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)x.tok0 * H + x.hd) * D, (size_t)H * D, x.len);
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
+
+#undef GDN_WAIT_MMA
 
 }  // namespace
 
@@ -960,65 +1085,37 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
     return true;
 }
 
+template <class Kernel>
+static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t smem, Stage stage, int grid, const TcParams& P,
+                                       cudaStream_t st) {
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    if (grid > 0) {
+        StageScope t(stage, st);
+        kernel<<<grid, kThreads, smem, st>>>(P);
+    }
+    return cudaGetLastError();
+}
+
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(tc_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prep::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    const int CH = P.p.L.max_chunks * P.p.d.H;
-    if (CH > 0) {
-        StageScope t(ST_PREP, st);
-        tc_prep_kernel<<<CH, kThreads, prep::SMEM_BYTES, st>>>(P);
-    }
-    return cudaGetLastError();
+    static bool done = false;
+    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, P.p.L.max_chunks * P.p.d.H, P, st);
 }
-
-// which: 0 = forward carry only, 1 = reverse only, 2 = both (one launch; forward and reverse CTAs interleave)
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(tc_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)scan::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static bool done = false;
     const int chains = P.p.d.N * P.p.d.H;
-    if (chains > 0) {
-        StageScope t(ST_SCANS, st);
-        tc_scan_kernel<<<chains * (P.scan_dirs == 2 ? 4 : 2), kThreads, scan::SMEM_BYTES, st>>>(P);
-    }
-    return cudaGetLastError();
+    return launch_chunk_kernel(tc_scan_kernel, done, scan::SMEM_BYTES, ST_SCANS, chains * (P.scan_dirs == 2 ? 2 : 1), P, st);
 }
-
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(tc_intra_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)intra::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    const int CH = P.p.L.max_chunks * P.p.d.H;
-    if (CH > 0) {
-        StageScope t(ST_INTRA, st);
-        tc_intra_kernel<<<CH, kThreads, intra::SMEM_BYTES, st>>>(P);
-    }
-    return cudaGetLastError();
+    static bool done = false;
+    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, P.p.L.max_chunks * P.p.d.H, P, st);
 }
-
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)outk::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    const int CH = P.p.L.max_chunks * P.p.d.H;
-    if (CH > 0) {
-        StageScope t(ST_OUT, st);
-        tc_out_kernel<<<CH, kThreads, outk::SMEM_BYTES, st>>>(P);
-    }
-    return cudaGetLastError();
+    static bool done = false;
+    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, P, st);
 }
 
 // A call with no tokens still owes the pass-through of the states.
@@ -1055,3 +1152,9 @@ cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st
 }
 
 }  // namespace gdn
+
+#ifdef GDN_PHASE_TIMING
+extern "C" int gdn_debug_ticks(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks, sizeof(long long) * 4 * 32);
+}
+#endif

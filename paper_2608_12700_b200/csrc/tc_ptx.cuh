@@ -126,6 +126,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Same for 8 consecutive columns.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 // ---------------------------------------------------------------- tcgen05.mma (bf16 x bf16 -> fp32)
 // Instruction descriptor: dense, fp32 accumulate, bf16 A and B.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn_major, bool b_mn_major, bool neg_a = false) {
@@ -145,41 +156,46 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint
            | (2ull << 61);  // 128-byte swizzle
 }
 
-// Operand view of a tile (or of a row/column window of it) for one MMA with contraction length Kt.
+// Operand view of a tile (or of a row/column window of it).  The descriptor of the k-th K=16 slice is
+// base + k * step + (k / 4) * jump in units of 16 bytes, so that issuing a product costs a few integer adds.
 struct Operand {
-    uint32_t base;     // shared address of element (row0, col0) of the window (row0 % 8 == 0, col0 % 64 == 0)
-    uint32_t R;        // rows of the underlying tile (block stride = R * 128 bytes)
+    uint32_t lo, hi;   // descriptor of slice 0
+    uint32_t step;     // added to lo per K=16 slice
+    uint32_t jump;     // added to lo on top of that after every fourth slice
     bool mn_major;     // false: contraction runs over tile columns; true: over tile rows
 };
-// Window whose MN index runs over tile rows starting at row0 and whose K index runs over columns from col0.
+// Window whose MN index runs over tile rows starting at row0 and whose K index runs over columns from col0
+// (row0 % 8 == 0, col0 % 64 == 0).  16 columns = 32 bytes inside a 128-byte row; every fourth slice moves on to
+// the next 64-column block, R * 128 bytes further.
 __device__ __forceinline__ Operand op_k_major(const void* tile, int R, int row0 = 0, int col0 = 0) {
-    return Operand{smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), (uint32_t)R, false};
+    const uint64_t d = make_desc(smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), 16, 1024);
+    return Operand{(uint32_t)d, (uint32_t)(d >> 32), 2u, (uint32_t)(R * 8 - 8), false};
 }
 // Window whose MN index runs over tile columns starting at col0 and whose K index runs over rows from row0.
+// 16 rows = 2048 bytes; LBO = distance between 64-column blocks, SBO = distance between 8-row groups.
 __device__ __forceinline__ Operand op_mn_major(const void* tile, int R, int row0 = 0, int col0 = 0) {
-    return Operand{smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), (uint32_t)R, true};
-}
-// Descriptor of the k-th K=16 slice.
-__device__ __forceinline__ uint64_t op_desc(const Operand& o, int ks) {
-    if (!o.mn_major)   // 16 columns = 32 bytes inside a 128-byte row; every 4th step moves to the next column block
-        return make_desc(o.base + (uint32_t)((ks >> 2) * o.R * 128 + (ks & 3) * 32), 16, 1024);
-    // 16 rows = 2048 bytes; LBO = distance between 64-column blocks, SBO = distance between 8-row groups
-    return make_desc(o.base + (uint32_t)ks * 2048, o.R * 128, 1024);
+    const uint64_t d = make_desc(smem_u32(tile) + (uint32_t)((col0 >> 6) * R * 128 + row0 * 128), (uint32_t)R * 128, 1024);
+    return Operand{(uint32_t)d, (uint32_t)(d >> 32), 128u, 0u, true};
 }
 
-__device__ __forceinline__ void mma_issue(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+__device__ __forceinline__ void mma_issue(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// D[M x N] (+)= A[M x Kt] * B[Kt x N]; one thread issues Kt/16 instructions.
-__device__ __forceinline__ void mma_tile(uint32_t tmem_d, const Operand& a, const Operand& b, int M, int N, int Kt, bool accumulate,
-                                         bool neg_a = false) {
+// D[M x N] (+)= A[M x Kt] * B[Kt x N]: one thread issues Kt / 16 instructions, fully unrolled so that each costs two
+// integer adds besides the tcgen05.mma itself (the tensor pipe accepts one such instruction every ~50-60 cycles).
+template <int M, int N, int Kt>
+__device__ __forceinline__ void mma_tile(uint32_t tmem_d, const Operand& a, const Operand& b, bool accumulate, bool neg_a = false) {
     const uint32_t idesc = make_idesc(M, N, a.mn_major, b.mn_major, neg_a);
-    for (int ks = 0; ks < Kt / 16; ++ks) mma_issue(tmem_d, op_desc(a, ks), op_desc(b, ks), idesc, accumulate || ks > 0);
+#pragma unroll
+    for (int ks = 0; ks < Kt / 16; ++ks) {
+        const uint32_t al = a.lo + ks * a.step + (ks >> 2) * a.jump, bl = b.lo + ks * b.step + (ks >> 2) * b.jump;
+        mma_issue(tmem_d, ((uint64_t)a.hi << 32) | al, ((uint64_t)b.hi << 32) | bl, idesc, (accumulate || ks > 0) ? 1u : 0u);
+    }
 }
 // Arrive on `bar` when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
@@ -187,6 +203,12 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 }
 
 // ---------------------------------------------------------------- small conversions
+// 2^x, hardware approximation (about 2 ulp); callers pass non-positive arguments only.
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&t);
