@@ -114,6 +114,33 @@ const char* gdn_status_string(gdn_status s);
  * or NULL for an unsupported descriptor.  Diagnostic only. */
 const char* gdn_kernel_path(const gdn_desc* desc);
 
+/* ---- backward without a caller-provided workspace (the paper has no counterpart) ----------------
+ * Some callers may not allocate device memory at the point where they need the gradients: code running
+ * under a memory pool that is frozen for the duration of a training step, plug-ins that are handed
+ * input and output buffers by a host framework and nothing else, or processes whose memory budget was
+ * fixed at start-up.  gdn_bwd_noalloc is gdn_bwd for them: same arguments without the workspace, same
+ * results.  Its scratch is an array of GDN_NOALLOC_WORKSPACE_BYTES that lives inside the library on every
+ * GPU that loads it, for the life of the process.  The call allocates and frees nothing.
+ *   - Problems whose gdn_workspace_bytes() backward size exceeds GDN_NOALLOC_WORKSPACE_BYTES are refused
+ *     with GDN_ERR_WORKSPACE_TOO_SMALL before anything is launched (at bf16, d_k = d_v = 128 the limit is
+ *     about 160 chunk-heads, e.g. H = 4 and 2560 tokens).
+ *   - The first call on a device looks up the array's device address (one-time set-up on the host); make
+ *     that first call outside of any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  The call
+ *     clears the part that must start from zero itself.  Two calls that overlap on the GPU (different
+ *     streams, or a second call enqueued before the first has finished on another stream) race on it:
+ *     keep such calls on one stream or synchronise between them.
+ *   - Conditions that only the device can see (malformed cu_seqlens) are not reported by this variant;
+ *     use gdn_bwd with gdn_last_device_status where that matters. */
+#define GDN_NOALLOC_WORKSPACE_BYTES (32u * 1024u * 1024u)
+gdn_status gdn_bwd_noalloc(const gdn_desc* desc,
+                           const void* q, const void* k, const void* v,
+                           const float* g, const float* beta, const float* h0,
+                           const void* dO, const float* dhT,
+                           const int32_t* cu_seqlens_dev,
+                           void* dq, void* dk, void* dv, float* dg, float* dbeta, float* dh0,
+                           void* cuda_stream);
+
 /* ---- measurement hooks (not part of the method; the paper has no counterpart) -------------------
  * gdn_launch_count: number of kernels this library has launched in this process.
  * gdn_stage_timing_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events

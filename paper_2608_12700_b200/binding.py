@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
-           "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family"]
+           "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -69,6 +69,8 @@ def lib():
         L.gdn_stage_timing_enable.argtypes = [I]
         L.gdn_stage_timing_read.restype = I
         L.gdn_stage_timing_read.argtypes = [I, P, P, P, P]
+        L.gdn_bwd_noalloc.restype = I
+        L.gdn_bwd_noalloc.argtypes = [D] + [P] * 15 + [P]
         L.gdn_debug_read.restype = I
         L.gdn_debug_read.argtypes = [D, P, ctypes.c_char_p, I, I, P]
         L.gdn_debug_force_family.restype = I
@@ -182,3 +184,16 @@ def gdn_debug_read(desc: gdn_desc, workspace, what: str, chunk: int, head: int):
     if s != GDN_OK:
         raise GdnError(s, "gdn_debug_read")
     return out
+
+
+GDN_NOALLOC_WORKSPACE_BYTES = 32 * 1024 * 1024
+
+
+def gdn_bwd_noalloc(desc, q, k, v, g, beta, h0, dO, dhT, cu_seqlens, dq, dk, dv, dg, dbeta, dh0, stream=None,
+                    check=True) -> int:
+    """gdn_bwd with the library's built-in scratch instead of a caller workspace (nothing is allocated)."""
+    s = lib().gdn_bwd_noalloc(ctypes.byref(desc), _p(q), _p(k), _p(v), _p(g), _p(beta), _p(h0), _p(dO), _p(dhT),
+                              _p(cu_seqlens), _p(dq), _p(dk), _p(dv), _p(dg), _p(dbeta), _p(dh0), _stream(stream))
+    if check and s != GDN_OK:
+        raise GdnError(s, "gdn_bwd_noalloc")
+    return s
