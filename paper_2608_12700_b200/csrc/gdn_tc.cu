@@ -37,7 +37,12 @@ namespace {
 using namespace tc;
 
 constexpr int D = 128;          // d_k = d_v
-constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column half = warp / 4
+constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column half = warp / 4 (scan, out)
+// The chunk kernels run 16 warps: four warps share a TMEM lane quadrant and split the 64 token columns four ways,
+// which shortens every thread's serial readout chain and gives the scheduler more warps to hide latencies with.
+constexpr int kWideThreads = 512;
+constexpr int kGroups = kWideThreads / 128;   // column groups
+constexpr int kTG = kC / kGroups;             // token columns per group (16)
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct TcParams {
@@ -194,7 +199,7 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF = 384, C_E = 0;
 }  // namespace prep
 
-__global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
     using namespace prep;
     const Problem& p = P.p;
     ChunkInfo x;
@@ -208,7 +213,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     __shared__ uint64_t bar_qk, bar_vo, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q4 = warp & 3, half = warp >> 2;
+    const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
@@ -285,9 +290,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     GDN_WAIT_MMA(2)
     GDN_TICK(0, 2);
     if (ok) {
-        const int i = (q4 & 1) * 32 + lane, j0 = half * 32;
+        const int i = (q4 & 1) * 32 + lane, j0 = grp * kTG;
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             float v[8];
             tmem_ld8(tmem + lane_base + C_S1 + j0 + part * 8, v);
             tmem_wait_ld();
@@ -365,9 +370,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     }
     GDN_WAIT_MMA(3)
     if (ok) {
-        const int f = q4 * 32 + lane, i0 = half * 32;
+        const int f = q4 * 32 + lane, i0 = grp * kTG;
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             const int ib = i0 + part * 8;
             float v[8], ve[8];
             tmem_ld8(tmem + lane_base + C_W + ib, v);
@@ -409,10 +414,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_prep_kernel(const __grid_const
     GDN_WAIT_MMA(4)
     GDN_TICK(0, 7);
     if (ok) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
-        const int r = q4 * 32 + lane, c0 = half * 64;
+        const int r = q4 * 32 + lane, c0 = grp * (D / kGroups);
         const float sc = p.d.scale;
 #pragma unroll 1
-        for (int part = 0; part < 8; ++part) {
+        for (int part = 0; part < D / kGroups / 8; ++part) {
             const int cb = c0 + part * 8;
             float v[8];
             tmem_ld8(tmem + lane_base + C_NM + cb, v);
@@ -629,7 +634,7 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
 
-__global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
     using namespace intra;
     const Problem& p = P.p;
     ChunkInfo x;
@@ -640,12 +645,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
     __shared__ float gl[kC], Gam[kC], ee[kC], bb[kC];
-    __shared__ float red[4][2][4][32];       // four token-wise reductions: [which][column half][lane quadrant][token]
-    __shared__ float dgam[kC], scal[2][kThreads / 32];
+    __shared__ float red[4][kGroups][4][kTG];   // four token-wise reductions: [which][column group][lane quadrant][token]
+    __shared__ float dgam[kC], scal[2][kWideThreads / 32];
     __shared__ uint64_t bar_in0, bar_in1, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q4 = warp & 3, half = warp >> 2;
+    const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
@@ -721,10 +726,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     GDN_WAIT_MMA(21)
     GDN_TICK(2, 3);
     const int mi = q4 * 16 + lane;     // row of an M = 64 accumulator held by this lane (lanes 0..15 only)
-    const int j0 = half * 32;
+    const int j0 = grp * kTG;
     if (ok) {   // P_ij = (q_i . k_j) D_ij for j <= i
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             float v[8];
             const int jb = j0 + part * 8;
             tmem_ld8(tmem + lane_base + slot(0) + jb, v);
@@ -750,11 +755,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
     const int f = q4 * 32 + lane;      // feature (lane of the transposed accumulators)
-    const int i0 = half * 32;          // first of this thread's 32 tokens
+    const int i0 = grp * kTG;          // first of this thread's 32 tokens
     float rs = 0.f;
     if (ok) {
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             const int ib = i0 + part * 8;
             float u[8], t[8], kb[8], pd[8];
             chunk_load(sm + UTT, 128, f, ib >> 3, u);
@@ -790,7 +795,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     GDN_WAIT_MMA(23)
     if (ok) {
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
             const int jb = j0 + part * 8, ib = i0 + part * 8;
             tmem_ld8(tmem + lane_base + slot(0) + jb, v);
@@ -827,7 +832,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     const size_t rowp = (size_t)H * D;
     if (ok) {
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             const int ib = i0 + part * 8;
             float a[8], b[8], xk[8], xv[8];
             tmem_ld8(tmem + lane_base + slot(4) + ib, a);
@@ -846,11 +851,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
                 xv[i] *= tile_get(sm + VT, 64, ib + i, f);              // dw partial
             }
             const float s0 = reduce8(a, lane), s1 = reduce8(xv, lane);
-            if (lane < 8) { red[0][half][q4][part * 8 + lane] = s0; red[1][half][q4][part * 8 + lane] = s1; }
+            if (lane < 8) { red[0][grp][q4][part * 8 + lane] = s0; red[1][grp][q4][part * 8 + lane] = s1; }
+            GDN_TICK(2, 16 + part);
         }
     }
     tc_fence_before();
     fence_async_smem();
+    GDN_TICK(2, 20);
     __syncthreads();
     GDN_TICK(2, 10);
 
@@ -861,16 +868,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
         mma_tile<64, 64, 128>(tmem + slot(0), op_mn_major(sm + DXVT, 128), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
     }
+    GDN_TICK(2, 21);
     if (ok) {
         flush_rows(sm + STG_QK, gdq, rowp, x.len);
         flush_rows(sm + STG_V, gdv, rowp, x.len);
     }
+    GDN_TICK(2, 22);
     __syncthreads();   // the staging tiles are rewritten below
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
+    GDN_TICK(2, 23);
     if (ok) {
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
             const int jb = j0 + part * 8;
             tmem_ld8(tmem + lane_base + slot(0) + jb, v);
@@ -884,8 +894,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
                 chunk_store(sm + GT, 64, mi, jb >> 3, v);
                 chunk_store(sm + BGT, 64, mi, jb >> 3, w);
             }
+            GDN_TICK(2, 24 + part);
         }
     }
+    GDN_TICK(2, 28);
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
@@ -902,7 +914,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     GDN_WAIT_MMA(26)
     if (ok) {
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
+        for (int part = 0; part < kTG / 8; ++part) {
             const int ib = i0 + part * 8;
             float y[8], t[8], c1[8], c2[8];
             tmem_ld8(tmem + lane_base + slot(4) + ib, y);
@@ -920,7 +932,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
                 c1[i] = kk * kcol;                                      // <k, dk^col> partial
             }
             const float s2 = reduce8(y, lane), s3 = reduce8(c1, lane);
-            if (lane < 8) { red[2][half][q4][part * 8 + lane] = s2; red[3][half][q4][part * 8 + lane] = s3; }
+            if (lane < 8) { red[2][grp][q4][part * 8 + lane] = s2; red[3][grp][q4][part * 8 + lane] = s3; }
         }
     }
     // block totals of sum_j r_j and <dh', h>
@@ -931,7 +943,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     GDN_TICK(2, 14);
     if (ok) flush_rows(sm + STG_QK, gdk, rowp, x.len);
     if (threadIdx.x < kC) {
-        const int i = threadIdx.x, hf = i >> 5, l = i & 31;
+        const int i = threadIdx.x, hf = i / kTG, l = i % kTG;
         auto tot = [&](int w) { return (red[w][hf][0][l] + red[w][hf][1][l]) + (red[w][hf][2][l] + red[w][hf][3][l]); };
         const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
         if (i < x.len) p.dbeta[(size_t)(x.tok0 + i) * H + x.hd] = db + dw;
@@ -940,7 +952,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_intra_kernel(const __grid_cons
     __syncthreads();
     if (threadIdx.x == 0 && ok) {
         float rsum = 0.f, hsum = 0.f;
-        for (int w = 0; w < kThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
+        for (int w = 0; w < kWideThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
         dgam[kC - 1] += rsum + Gam[kC - 1] * hsum;
         float run = 0.f;   // gam_i = sum_{j<=i} g_j  =>  dg_j = sum_{i>=j} dgam_i
         for (int i = kC - 1; i >= 0; --i) {
@@ -1086,8 +1098,8 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
 }
 
 template <class Kernel>
-static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t smem, Stage stage, int grid, const TcParams& P,
-                                       cudaStream_t st) {
+static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t smem, Stage stage, int grid, int threads,
+                                       const TcParams& P, cudaStream_t st) {
     if (!attr_done) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -1095,27 +1107,27 @@ static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t 
     }
     if (grid > 0) {
         StageScope t(stage, st);
-        kernel<<<grid, kThreads, smem, st>>>(P);
+        kernel<<<grid, threads, smem, st>>>(P);
     }
     return cudaGetLastError();
 }
 
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
     static bool done = false;
-    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, P.p.L.max_chunks * P.p.d.H, P, st);
+    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, P.p.L.max_chunks * P.p.d.H, kWideThreads, P, st);
 }
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int chains = P.p.d.N * P.p.d.H;
-    return launch_chunk_kernel(tc_scan_kernel, done, scan::SMEM_BYTES, ST_SCANS, chains * (P.scan_dirs == 2 ? 2 : 1), P, st);
+    return launch_chunk_kernel(tc_scan_kernel, done, scan::SMEM_BYTES, ST_SCANS, chains * (P.scan_dirs == 2 ? 2 : 1), kThreads, P, st);
 }
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
     static bool done = false;
-    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, P.p.L.max_chunks * P.p.d.H, P, st);
+    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, P.p.L.max_chunks * P.p.d.H, kWideThreads, P, st);
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static bool done = false;
-    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, P, st);
+    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, kThreads, P, st);
 }
 
 // A call with no tokens still owes the pass-through of the states.
