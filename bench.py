@@ -194,7 +194,7 @@ def run_ours(args):
     # The dominant kernel is charged with the whole path's algorithmic work when it is the kernel that
     # streams the inputs and writes the gradients (the intra / fused gradient stage); a scan stage is
     # charged with the state traffic it cannot avoid.  Stated per stage in the design doc.
-    dom_bytes, dom_flops = stage_algorithmic_work(dom, wl, io_bytes)
+    dom_bytes, dom_flops = stage_algorithmic_work(dom, wl, io_bytes, binding.gdn_kernel_path(desc))
     d_hbm, d_tc = benchutil.roofline_times(dom_bytes, dom_flops, peaks, sustained=False)
     dom_s = stage_ms[dom] * 1e-3
     if d_hbm >= d_tc:
@@ -230,13 +230,23 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def stage_algorithmic_work(stage, wl, io_bytes):
+def stage_algorithmic_work(stage, wl, io_bytes, family=""):
     """(bytes, flops) the named stage must move / multiply per launch (one launch covers the whole batch)."""
     from paper_2608_12700_b200 import benchutil
     th, chains, chd = wl.T_total * wl.H, wl.N * wl.H, wl.n_chunks() * wl.H
     dk, dv = wl.d_k, wl.d_v
     tri_k, tri_v, dense = 64 * 64 * dk, 64 * 64 * dv, 2 * 64 * dk * dv
     gates = 2 if wl.delta_rule else 1
+    if family == "tcgen05_bf16_scalar_gate":
+        # two fused passes per chain: the forward pass reads k, v, g; the backward pass streams every input and
+        # writes every gradient (the whole path's algorithmic traffic) and runs 5 triangular + 4 dense products
+        if stage == "fscan":
+            return th * ((dk + dv) * io_bytes + 4), chd * dense
+        if stage == "rscan":
+            byts = benchutil.path_alg_bytes(token_heads=th, chains=chains, d_k=dk, d_v=dv, io_bytes=io_bytes, delta_rule=0,
+                                            has_h0=False, has_dhT=wl.dhT is not None)
+            return byts, chd * (3 * tri_k + 2 * tri_v + 4 * dense)
+        return th * 4, 0.0
     if stage in ("fscan", "rscan"):
         # a carry stage must at least read its chunk-local operator and write one state per chunk
         return chd * (dk * dk + 2 * dk * dv) * io_bytes, chd * 2.0 * dk * dk * dv

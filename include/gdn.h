@@ -110,7 +110,8 @@ gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream);
 /* Static, NUL-terminated description of a status code. */
 const char* gdn_status_string(gdn_status s);
 
-/* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16"),
+/* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16",
+ * "tcgen05_bf16_scalar_gate"),
  * or NULL for an unsupported descriptor.  Diagnostic only. */
 const char* gdn_kernel_path(const gdn_desc* desc);
 

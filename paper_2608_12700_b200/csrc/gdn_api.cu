@@ -44,13 +44,18 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-enum class Path { None, SimtF32, SimtBf16, TcBf16 };
+enum class Path { None, SimtF32, SimtBf16, TcBf16, Tc64Bf16 };
 
 int g_force_family = 0;
 
 Path pick_path(const gdn_desc& d) {
     if (d.dtype == GDN_F32) return Path::SimtF32;
-    if (d.dtype == GDN_BF16) return (tc_supported(d) && g_force_family != 1) ? Path::TcBf16 : Path::SimtBf16;
+    if (d.dtype == GDN_BF16) {
+        if (g_force_family == 1) return Path::SimtBf16;
+        if (tc_supported(d)) return Path::TcBf16;
+        if (tc64_supported(d)) return Path::Tc64Bf16;
+        return Path::SimtBf16;
+    }
     return Path::None;
 }
 
@@ -67,7 +72,7 @@ gdn_status check_desc(const gdn_desc* d) {
 
 WsLayout layout_for(const gdn_desc& d) {
     // tcgen05 path: every factor, state and additive term of the carries is a bf16 tile image.
-    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0);
+    if (pick_path(d) == Path::TcBf16 || pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
     return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
 }
@@ -115,7 +120,8 @@ gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k,
     p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.h0 = h0; p.cu = cu; p.o = o; p.hT = hT;
     p.ws = static_cast<char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-    const cudaError_t e = pick_path(*desc) == Path::TcBf16 ? tc_launch_fwd(p, st) : simt_launch_fwd(p, st);
+    const Path path = pick_path(*desc);
+    const cudaError_t e = path == Path::TcBf16 ? tc_launch_fwd(p, st) : path == Path::Tc64Bf16 ? tc64_launch_fwd(p, st) : simt_launch_fwd(p, st);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
@@ -142,7 +148,9 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     p.ws = static_cast<char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const bool fresh = workspace_is_fresh_from_fwd != 0;
-    const cudaError_t e = pick_path(*desc) == Path::TcBf16 ? tc_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
+    const Path path = pick_path(*desc);
+    const cudaError_t e = path == Path::TcBf16 ? tc_launch_bwd(p, fresh, st)
+                          : path == Path::Tc64Bf16 ? tc64_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
@@ -184,7 +192,7 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
     if (!workspace || !what || !host_out) return GDN_ERR_NULL_ARG;
     const WsLayout L = layout_for(*desc);
     if (chunk < 0 || chunk >= L.max_chunks || head < 0 || head >= desc->H) return GDN_ERR_BAD_SHAPE;
-    const bool tcp = pick_path(*desc) == Path::TcBf16;
+    const bool tcp = pick_path(*desc) == Path::TcBf16 || pick_path(*desc) == Path::Tc64Bf16;
     const size_t ch = (size_t)chunk * desc->H + head;
     const int dk = desc->d_k, dv = desc->d_v;
     struct Q { const char* name; size_t off; int rows, cols; int kind; };  // kind 0: fp32 row-major always
@@ -251,6 +259,7 @@ const char* gdn_kernel_path(const gdn_desc* desc) {
         case Path::SimtF32: return "simt_f32";
         case Path::SimtBf16: return "simt_bf16";
         case Path::TcBf16: return "tcgen05_bf16";
+        case Path::Tc64Bf16: return "tcgen05_bf16_scalar_gate";
         default: return nullptr;
     }
 }

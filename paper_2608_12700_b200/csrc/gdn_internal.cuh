@@ -109,4 +109,10 @@ bool tc_supported(const gdn_desc& d);
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 
+
+// tcgen05 family for the scalar-gate recurrence (bf16 I/O, d_k = d_v = 64, delta rule off).
+bool tc64_supported(const gdn_desc& d);
+cudaError_t tc64_launch_fwd(const Problem& p, cudaStream_t st);
+cudaError_t tc64_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
+
 }  // namespace gdn

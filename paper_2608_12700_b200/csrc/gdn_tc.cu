@@ -18,9 +18,7 @@
 // GDN_ERR_DEVICE_TIMEOUT in the workspace header and the CTA leaves through its normal teardown.
 // Loops over accumulator columns are kept rolled (8 columns per trip): the kernels run each piece of code once
 // per chunk, so instruction-cache footprint matters more than loop overhead.
-#include "gdn_internal.cuh"
-#include "tc_ptx.cuh"
-#include "tc_tmap.cuh"
+#include "tc_common.cuh"
 
 namespace gdn {
 
@@ -34,8 +32,6 @@ __device__ long long g_ticks[4][32];
 
 namespace {
 
-using namespace tc;
-
 constexpr int D = 128;          // d_k = d_v
 constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column half = warp / 4 (scan, out)
 // The chunk kernels run 16 warps: four warps share a TMEM lane quadrant and split the 64 token columns four ways,
@@ -43,115 +39,12 @@ constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column hal
 constexpr int kWideThreads = 512;
 constexpr int kGroups = kWideThreads / 128;   // column groups
 constexpr int kTG = kC / kGroups;             // token columns per group (16)
-constexpr float kLog2e = 1.4426950408889634f;
-
 struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
     int with_bwd;                          // prep: also produce E
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
 };
-
-__device__ __forceinline__ void report_timeout(char* ws, int where) {
-    WsHeader* h = reinterpret_cast<WsHeader*>(ws);
-    h->status = GDN_ERR_DEVICE_TIMEOUT;
-    h->detail = where;
-}
-
-__device__ __forceinline__ unsigned char* align1024(unsigned char* p) {
-    return p + ((1024u - (smem_u32(p) & 1023u)) & 1023u);
-}
-
-// 8 fp32 <-> one 16-byte chunk of bf16
-__device__ __forceinline__ uint4 pack8(const float* v) {
-    return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-}
-__device__ __forceinline__ void unpack8(const uint4& u, float* v) {
-    v[0] = bf16_lo(u.x); v[1] = bf16_hi(u.x); v[2] = bf16_lo(u.y); v[3] = bf16_hi(u.y);
-    v[4] = bf16_lo(u.z); v[5] = bf16_hi(u.z); v[6] = bf16_lo(u.w); v[7] = bf16_hi(u.w);
-}
-// Chunk `ch` (columns 8 ch .. 8 ch + 7) of row r of a tile with R rows.
-__device__ __forceinline__ void chunk_store(unsigned char* tile, int R, int r, int ch, const float* v) {
-    *reinterpret_cast<uint4*>(tile + tile_chunk_off(R, r, ch)) = pack8(v);
-}
-__device__ __forceinline__ void chunk_load(const unsigned char* tile, int R, int r, int ch, float* v) {
-    unpack8(*reinterpret_cast<const uint4*>(tile + tile_chunk_off(R, r, ch)), v);
-}
-__device__ __forceinline__ float tile_get(const unsigned char* tile, int R, int r, int c) {
-    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + tile_off(R, r, c)));
-}
-__device__ __forceinline__ void tile_put(unsigned char* tile, int R, int r, int c, float x) {
-    *reinterpret_cast<__nv_bfloat16*>(tile + tile_off(R, r, c)) = __float2bfloat16_rn(x);
-}
-
-// Zero rows [row0 + len, row0 + 64) of a tile with R rows and 128 columns.
-__device__ __forceinline__ void zero_tail_rows(unsigned char* tile, int R, int row0, int len) {
-    for (int t = threadIdx.x; t < (kC - len) * 16; t += blockDim.x) {
-        const int r = row0 + len + t / 16, ch = t % 16;
-        *reinterpret_cast<uint4*>(tile + tile_chunk_off(R, r, ch)) = make_uint4(0, 0, 0, 0);
-    }
-}
-
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// Each lane holds 8 values (one per token of a group of 8); returns, on every lane, the sum over the 32 lanes of
-// the value belonging to token (lane % 8).  Fixed order: bit-identical from run to run.
-__device__ __forceinline__ float reduce8(float (&v)[8], int lane) {
-    bool up = (lane & 4) != 0;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const float send = up ? v[k] : v[k + 4], keep = up ? v[k + 4] : v[k];
-        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-    }
-    up = (lane & 2) != 0;
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        const float send = up ? v[k] : v[k + 2], keep = up ? v[k + 2] : v[k];
-        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-    }
-    up = (lane & 1) != 0;
-    {
-        const float send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
-        v[0] = keep + __shfl_xor_sync(0xffffffffu, send, 1);
-    }
-    float r = v[0];
-    r += __shfl_xor_sync(0xffffffffu, r, 8);
-    r += __shfl_xor_sync(0xffffffffu, r, 16);
-    return r;
-}
-
-// Copy a staged [64 tokens][128 features] bf16 tile to a [T, H, 128] tensor with 16-byte stores (rows < len only).
-__device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloat16* gbase, size_t row_pitch, int len) {
-    for (int t = threadIdx.x; t < kC * 16; t += blockDim.x) {
-        const int i = t >> 4, chk = t & 15;
-        if (i < len) *reinterpret_cast<uint4*>(gbase + (size_t)i * row_pitch + chk * 8) = *reinterpret_cast<const uint4*>(tile + tile_chunk_off(64, i, chk));
-    }
-}
-
-struct ChunkInfo { int c, hd, ch, tok0, len; };
-__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) {
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    x.c = blockIdx.x / p.d.H;
-    x.hd = blockIdx.x % p.d.H;
-    if (x.c >= hdr->n_chunks) return false;
-    x.ch = blockIdx.x;
-    x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
-    x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
-    return true;
-}
-
-// Wait for the MMAs committed to `bar`; on a timeout record it once.
-#define GDN_WAIT_MMA(where)                                                    \
-    if (ok) {                                                                  \
-        ok = mbar_wait(&bar_mma, mma_phase);                                   \
-        mma_phase ^= 1;                                                        \
-        if (!ok && threadIdx.x == 0) report_timeout(p.ws, where);              \
-    }                                                                          \
-    tc_fence_after();
 
 // One block diagonal (distance DIST below the main one) of the blocked inverse of I + A, 16 x 16 blocks:
 // T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc).  Af, Tf, Sf are fp32 [64][65] in shared memory.

@@ -49,10 +49,30 @@ def test_ragged_varlen_and_empty_sequence(dtype, family):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_scalar_gate_recurrence_delta_rule_off(dtype):
+def test_scalar_gate_recurrence_delta_rule_off(dtype, family):
     wl = small("beta_off_" + dtype, dtype=dtype, B=2, T=200, H=2, d_k=64, d_v=64, delta_rule=0, g_scale=0.05,
                seed=12)
     check_against_oracle(wl, runner.backward(wl))
+
+
+def test_scalar_gate_recurrence_ragged_with_states(family):
+    wl = small("beta_off_ragged", dtype="bf16", lengths=[65, 128, 0, 37, 300, 1], H=3, d_k=64, d_v=64, delta_rule=0,
+               g_scale=0.05, states=True, scale=0.5, seed=22)
+    got = runner.backward(wl)
+    check_against_oracle(wl, got)
+    assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))
+
+
+def test_scalar_gate_forward_outputs(family):
+    wl = small("beta_off_fwd", dtype="bf16", lengths=[70, 130], H=2, d_k=64, d_v=64, delta_rule=0, states=True, seed=23)
+    buf = runner.to_device(wl, want_o=True)
+    runner.run_fwd(buf)
+    got = runner.fetch(buf)
+    ref = oracle_grads(wl)
+    assert rel(got["o"], ref["o"]) < TOL["bf16"]
+    assert rel(got["hT"], ref["hT"]) < TOL["bf16"]
+    runner.run_bwd(buf, fresh=1)
+    check_against_oracle(wl, runner.fetch(buf))
 
 
 def test_scale_argument():
@@ -77,6 +97,7 @@ def test_kernel_family_dispatch():
     assert binding.gdn_kernel_path(mk(dtype="f32")) == "simt_f32"
     assert binding.gdn_kernel_path(mk(d_k=64, d_v=64)) == "simt_bf16"
     assert binding.gdn_kernel_path(mk(delta_rule=0)) == "simt_bf16"
+    assert binding.gdn_kernel_path(mk(d_k=64, d_v=64, delta_rule=0)) == "tcgen05_bf16_scalar_gate"
 
 
 def test_zero_tokens_passes_the_state_gradient_through():
