@@ -247,9 +247,11 @@ def stage_algorithmic_work(stage, wl, io_bytes, family=""):
                                             has_h0=False, has_dhT=wl.dhT is not None)
             return byts, chd * (3 * tri_k + 2 * tri_v + 4 * dense)
         return th * 4, 0.0
-    if stage in ("fscan", "rscan"):
-        # a carry stage must at least read its chunk-local operator and write one state per chunk
-        return chd * (dk * dk + 2 * dk * dv) * io_bytes, chd * 2.0 * dk * dk * dv
+    if stage in ("fscan", "rscan", "scans"):
+        # a carry stage must at least read its chunk-local operator and additive term and write one state per chunk;
+        # "scans" is the launch that runs the forward and the reverse carry together
+        ndir = 2 if stage == "scans" else 1
+        return ndir * chd * (dk * dk + 2 * dk * dv) * io_bytes, ndir * chd * 2.0 * dk * dk * dv
     if stage == "prep":
         return th * ((dk + dv) * io_bytes + 4 * gates), chd * (2 * tri_k + tri_v + 2 * dense + 2 * 64 ** 3 / 3)
     if stage == "eprep":

@@ -25,9 +25,13 @@ namespace gdn {
 // Optional phase timing (compile with -DGDN_PHASE_TIMING): thread 0 of CTA 0 stamps clock64() at phase borders.
 #ifdef GDN_PHASE_TIMING
 __device__ long long g_ticks[4][32];
-#define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_ticks[kern][idx] = clock64(); } while (0)
+__device__ int g_tick_trip = 0;   // which trip of a persistent CTA is stamped
+__device__ int g_trip_now = 0;
+#define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (kern != 2 || g_trip_now == g_tick_trip)) g_ticks[kern][idx] = clock64(); } while (0)
+#define GDN_TICKT(tid, kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == (tid)) g_ticks[kern][idx] = clock64(); } while (0)
 #else
 #define GDN_TICK(kern, idx) do { } while (0)
+#define GDN_TICKT(tid, kern, idx) do { } while (0)
 #endif
 
 namespace {
@@ -95,9 +99,11 @@ constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF 
 __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
     using namespace prep;
     const Problem& p = P.p;
-    ChunkInfo x;
-    if (!chunk_info(p, x)) return;
+    // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ... and pulls the inputs of its
+    // next one into L2 while it works on the current one.
     const int H = p.d.H;
+    const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
+    if ((int)blockIdx.x >= n_items) return;
     const bool bwd = P.with_bwd != 0;
 
     extern __shared__ unsigned char smem_raw[];
@@ -119,7 +125,11 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     bool ok = true;
-    uint32_t mma_phase = 0;
+    uint32_t mma_phase = 0, in_phase = 0;
+#pragma unroll 1
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
+    ChunkInfo x;
+    chunk_info(p, x, item);
     GDN_TICK(0, 0);
 
     if (threadIdx.x == 0) {
@@ -132,6 +142,15 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         for (int cb = 0; cb < 2; ++cb) {
             tma_load_2d(sm + VO + cb * 16384, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_vo);
             if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_vo);
+        }
+        ChunkInfo nx;
+        if (item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x)) {   // next trip's inputs -> L2
+            for (int cb = 0; cb < 2; ++cb) {
+                prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
+                prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
+                prefetch_l2_tma_2d(&P.tm_v, nx.hd * D + cb * 64, nx.tok0);
+                if (bwd) prefetch_l2_tma_2d(&P.tm_do, nx.hd * D + cb * 64, nx.tok0);
+            }
         }
     }
     // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
@@ -158,8 +177,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         ee[i] = expf(gam[kC - 1] - gam[i]);
         reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gam[i];
     }
-    ok = mbar_wait(&bar_qk, 0) && mbar_wait(&bar_vo, 0);
-    if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
+    if (ok) {
+        ok = mbar_wait(&bar_qk, in_phase) && mbar_wait(&bar_vo, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
+    }
     if (ok && x.len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
         zero_tail_rows(sm + QK, 128, 0, x.len);
         zero_tail_rows(sm + QK, 128, 64, x.len);
@@ -338,9 +359,13 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
             if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768);
             bulk_commit();
         }
-        bulk_wait_all<0>();   // shared memory must stay valid until every bulk store has read it
+        bulk_wait_read<0>();  // shared memory must stay valid until every bulk store has read it
     }
+    tc_fence_before();
+    __syncthreads();          // the next trip overwrites the tiles
     GDN_TICK(0, 8);
+    if (!ok) break;
+    }
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -354,12 +379,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 namespace scan {
 constexpr int STAGES = 2;
+constexpr int PREFETCH_AHEAD = 3;                // steps by which L2 prefetches run ahead of the ring loads
 constexpr int GE_CAP = 2048;                     // chunk decays cached per chain (longer chains read them from global)
 constexpr uint32_t NM = 0;                       // ring: Nm tile image (32 KB) + additive-term image (32 KB) per stage
 constexpr uint32_t ADD = 32768;
 constexpr uint32_t STAGE_BYTES = 65536;
-constexpr uint32_t HT = STAGES * STAGE_BYTES;    // state tile [128][128], 32 KB
-constexpr uint32_t SMEM_BYTES = HT + 32768 + 1024;
+constexpr uint32_t HT = STAGES * STAGE_BYTES;    // two state tiles [128][128], 32 KB each (one feeds the MMA and the
+                                                 // bulk store of this step while the next step's is being written)
+constexpr uint32_t SMEM_BYTES = HT + 2 * 32768 + 1024;
 static_assert(SMEM_BYTES + GE_CAP * 4 <= 227 * 1024, "shared memory budget");
 }  // namespace scan
 
@@ -407,9 +434,21 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
         mbar_expect_tx(&bar_full[stage], 65536);
         bulk_load(sm + stage * STAGE_BYTES + NM, nm_base + ch * 32768, 32768, &bar_full[stage]);
         bulk_load(sm + stage * STAGE_BYTES + ADD, add_base + ch * 32768, 32768, &bar_full[stage]);
+        // The ring gives a load one step of lead, less than an HBM round trip; pull the step after next into L2 now.
+        if (s + PREFETCH_AHEAD < nsteps) {
+            const size_t chn = (size_t)chunk_of(s + PREFETCH_AHEAD) * p.d.H + hd;
+            prefetch_l2_bulk(nm_base + chn * 32768, 32768);
+            prefetch_l2_bulk(add_base + chn * 32768, 32768);
+        }
     };
-    if (threadIdx.x == 0)
+    if (threadIdx.x == 32) {
+        for (int s = STAGES; s < STAGES + PREFETCH_AHEAD && s < nsteps; ++s) {
+            const size_t chn = (size_t)chunk_of(s) * p.d.H + hd;
+            prefetch_l2_bulk(nm_base + chn * 32768, 32768);
+            prefetch_l2_bulk(add_base + chn * 32768, 32768);
+        }
         for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
+    }
     for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
         ge[s] = expf(gamma[((size_t)chunk_of(s) * p.d.H + hd) * kC + kC - 1]);
     // initial state
@@ -426,26 +465,21 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     __syncthreads();
     bool ok = true;
     uint32_t mma_phase = 0;
-    unsigned char* Ht = sm + HT;
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
+        unsigned char* Ht = sm + HT + (s & 1) * 32768;
         const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
         const int stage = s % STAGES;
         const unsigned char* ring = sm + stage * STAGE_BYTES;
         if (s < 4) GDN_TICK(1, s * 5 + 0);
         const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
-        uint4 packed[8];   // state -> bf16: operand tile of the MMA and the stored per-chunk state
+        // state -> bf16: operand tile of the MMA; the same bytes are the per-chunk state the gradient stage reads
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            packed[k] = pack8(st + 8 * k);
-            *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, hf * 8 + k)) = packed[k];
-        }
+        for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, hf * 8 + k)) = pack8(st + 8 * k);
         fence_async_smem();
         __syncthreads();
         if (s < 4) GDN_TICK(1, s * 5 + 1);
         if (threadIdx.x == 0) {
-            // every thread has finished step s - 1, so its ring slot can take step s - 1 + STAGES
-            if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
             ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
             if (ok) {
                 tc_fence_after();
@@ -454,12 +488,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
             } else {
                 report_timeout(p.ws, 10);
             }
+            // The tile leaves through the async proxy: generic global stores here would stall the next step's proxy
+            // fence until they drain.  Waiting for the previous step's store to have read its tile before committing the
+            // MMA orders that read before the overwrite of the tile two steps later.
+            bulk_store(keep_base + ch * 32768, Ht, 32768);
+            bulk_commit();
+            bulk_wait_read<1>();
             mma_commit(&bar_mma);
-        }
-        {   // the same bytes go to the workspace while the MMA runs (after the fence: it would wait for these stores)
-            char* keep = keep_base + ch * 32768;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(keep + tile_chunk_off(128, r, hf * 8 + k)) = packed[k];
+        } else if (threadIdx.x == 32) {
+            // every thread has finished step s - 1, so its ring slot can take step s - 1 + STAGES.  Bulk copies are slow
+            // to issue; a thread of another warp does it so that the MMA issue is not delayed.
+            if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
         }
         if (s < 4) GDN_TICK(1, s * 5 + 2);
         ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);   // the additive term of this step is in shared memory
@@ -486,6 +525,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 #pragma unroll
         for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
     }
+    if (threadIdx.x == 0) bulk_wait_read<0>();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 128);
@@ -506,23 +546,25 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 // The decay gradient uses the identities  rowsum(dP.P) + scale Gam <q, dO h^T> = <q, dq>  and its analogues for
 // k:  dgamma_i = <q_i, dq_i> + <k_i, dk_i^row> - <k_i, dk_i^col>, where dk^row = Diag(b)(G K + Diag(Gam) dXk)
 // collects the terms in which k_i enters with exp(+gamma_i) and dk^col those with exp(-gamma_i); the last row
-// of the chunk adds sum_j r_j + Gam_e <dh', h> (r_j = <(Kb dh')_j, U_j>).  Outputs are staged in shared memory
-// as token-major tiles and written with 16-byte stores.
+// of the chunk adds sum_j r_j + Gam_e <dh', h> (r_j = <(Kb dh')_j, U_j>).  Phases 1-2 produce transposed
+// accumulators (features on TMEM lanes) because their results feed later products; from phase 3 on every
+// accumulator that becomes a gradient is token-major.
 // ------------------------------------------------------------------------------------------------
 namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
 constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB
-constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64], then staged dq / dk
+constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
 constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
-constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk^T, dXv^T [128][64] each
+constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each
 constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
-constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later staged dv, then G and Diag(b) G
-constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB
+constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later staged dq, then G and Diag(b) G [64][64] each
+constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dv, then staged dk
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DO, DXKT = HH, DXVT = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192, STG_QK = DO, STG_V = UT;
+constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
+constexpr uint32_t STG_A = UT, STG_B = DUT;   // token-major staging of dq | dv and dk (free once phase 4 has read U^T, dU^T)
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
@@ -530,15 +572,17 @@ __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eigh
 __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
     using namespace intra;
     const Problem& p = P.p;
-    ChunkInfo x;
-    if (!chunk_info(p, x)) return;
+    // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
+    // tiles of its next one are pulled into L2, so that the loads at the top of the next trip do not wait for HBM.
     const int H = p.d.H;
+    const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
+    if ((int)blockIdx.x >= n_items) return;
     const float sc = p.d.scale;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
     __shared__ float gl[kC], Gam[kC], ee[kC], bb[kC];
-    __shared__ float red[4][kGroups][4][kTG];   // four token-wise reductions: [which][column group][lane quadrant][token]
+    __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kWideThreads / 32];
     __shared__ uint64_t bar_in0, bar_in1, bar_mma;
     __shared__ uint32_t tmem_slot;
@@ -556,7 +600,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     bool ok = true;
-    uint32_t mma_phase = 0;
+    uint32_t mma_phase = 0, in_phase = 0;
+#pragma unroll 1
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
+    ChunkInfo x;
+    chunk_info(p, x, item);
+#ifdef GDN_PHASE_TIMING
+    if (blockIdx.x == 0 && threadIdx.x == 0) g_trip_now = (item - (int)blockIdx.x) / (int)gridDim.x;
+#endif
     GDN_TICK(2, 0);
 
     if (threadIdx.x == 0) {
@@ -575,6 +626,20 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
         }
         bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in1);
         bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)x.ch * 8192, 8192, &bar_in1);
+        ChunkInfo nx;
+        if (item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x)) {   // next trip's tiles -> L2
+            for (int cb = 0; cb < 2; ++cb) {
+                prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
+                prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
+                prefetch_l2_tma_2d(&P.tm_v, nx.hd * D + cb * 64, nx.tok0);
+                prefetch_l2_tma_2d(&P.tm_do, nx.hd * D + cb * 64, nx.tok0);
+            }
+            prefetch_l2_bulk(p.ws + p.L.W + (size_t)nx.ch * 16384, 16384);
+            prefetch_l2_bulk(p.ws + p.L.Ut + (size_t)nx.ch * 16384, 16384);
+            prefetch_l2_bulk(p.ws + p.L.Tm + (size_t)nx.ch * 8192, 8192);
+            prefetch_l2_bulk(p.ws + p.L.hc + (size_t)nx.ch * 32768, 32768);
+            prefetch_l2_bulk(p.ws + p.L.dhn + (size_t)nx.ch * 32768, 32768);
+        }
     }
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
@@ -585,8 +650,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
         ee[i] = expf(gend - g);
         bb[i] = (i < x.len) ? p.beta[(size_t)(x.tok0 + i) * H + x.hd] : 0.f;
     }
-    ok = mbar_wait(&bar_in0, 0) && mbar_wait(&bar_in1, 0);
-    if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
+    if (ok) {
+        ok = mbar_wait(&bar_in0, in_phase) && mbar_wait(&bar_in1, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
+    }
     if (ok && x.len < kC) {
         zero_tail_rows(sm + QK, 128, 0, x.len);
         zero_tail_rows(sm + QK, 128, 64, x.len);
@@ -676,12 +743,27 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     __syncthreads();
     GDN_TICK(2, 6);
 
+    // From here on the accumulators that become gradients are produced token-major (64 token rows x 128 features,
+    // M = 64): a thread owns a token row, so row dots are thread-local and rows leave with 16-byte stores.  A 64-row
+    // accumulator occupies lanes 0..15 of each quadrant ("group A"); a second one sits in lanes 16..31 of the same
+    // columns ("group B", address + 16 lanes), and one tcgen05.ld serves both groups.
+    //   columns   group A                               group B
+    //   0..127    dO h^T (ph 3) -> (bG) K (ph 6)        dP (ph 3, 64 cols) -> dXk (ph 4)
+    //   128..255  (dP.D) K (ph 4) -> dXk again (ph 6)   dXv (ph 4)
+    //   256..383  dW^T (ph 3, all lanes) -> dk^col      G K (ph 6)
+    //   384..511  U dh'^T (ph 4)                        dA (ph 5, 64 cols)
+    constexpr uint32_t LB = 16u << 16;
+    const bool ga = lane < 16;
+    const int tr = q4 * 16 + (lane & 15);   // token row of this lane in token-major accumulators
+    const int cb0 = grp * 32;               // first of this thread's 32 feature columns
+    const int j0b = grp * kTG;              // first of its 16 columns in 64-column accumulators
+
     // ---- phase 3
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile<64, 64, 128>(tmem + slot(0), op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);
-        mma_tile<128, 64, 128>(tmem + slot(4), op_k_major(sm + HH, 128), op_k_major(sm + DO, 64), false);
-        mma_tile<128, 64, 128>(tmem + slot(5), op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
+        mma_tile<64, 64, 128>(tmem + 0 + LB, op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);           // dO U^T
+        mma_tile<64, 128, 128>(tmem + 0, op_k_major(sm + DO, 64), op_k_major(sm + HH, 128), false);                 // dO h^T
+        mma_tile<128, 64, 128>(tmem + 256, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
         mma_commit(&bar_mma);
     }
     GDN_TICK(2, 7);
@@ -690,14 +772,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
-            const int jb = j0 + part * 8, ib = i0 + part * 8;
-            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
-            tmem_ld8(tmem + lane_base + slot(5) + ib, w);
+            const int jb = j0b + part * 8, ib = i0 + part * 8;
+            tmem_ld8(tmem + lane_base + 0 + jb, v);       // group B: dO U^T
+            tmem_ld8(tmem + lane_base + 256 + ib, w);     // all lanes: dW^T
             tmem_wait_ld();
-            if (lane < 16) {   // dPD = scale tril(dO U^T) . D
+            if (!ga) {   // dPD = scale tril(dO U^T) . D
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? sc * v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
-                chunk_store(sm + DPD, 64, mi, jb >> 3, v);
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? sc * v[j] * ex2(gl[tr] - gl[jb + j]) : 0.f;
+                chunk_store(sm + DPD, 64, tr, jb >> 3, v);
             }
             chunk_store(sm + DWT, 128, f, ib >> 3, w);              // dW^T = -(dU h^T)^T
         }
@@ -710,87 +792,88 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     // ---- phase 4
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile<128, 64, 64>(tmem + slot(1), op_mn_major(sm + QK, 128, 64), op_k_major(sm + DPD, 64), false);
-        mma_tile<128, 64, 64>(tmem + slot(2), op_k_major(sm + DWT, 128), op_mn_major(sm + TT, 64), false);
-        mma_tile<128, 64, 64>(tmem + slot(3), op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), false);
-        mma_tile<128, 64, 64>(tmem + slot(6), op_mn_major(sm + QK, 128, 0), op_mn_major(sm + DPD, 64), false);
-        mma_tile<128, 64, 128>(tmem + slot(7), op_k_major(sm + DH, 128), op_mn_major(sm + UT, 128), false);
+        mma_tile<64, 128, 64>(tmem + 128, op_k_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 64), false);           // (dP.D) K
+        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
+        mma_tile<64, 128, 128>(tmem + 384, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);              // U dh'^T
+        mma_tile<64, 128, 64>(tmem + 0 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);            // T^T dW
+        mma_tile<64, 128, 64>(tmem + 128 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DUT, 128), false);          // T^T dU
         mma_commit(&bar_mma);
     }
     GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
-    __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + ((size_t)x.tok0 * H + x.hd) * D;
-    __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + ((size_t)x.tok0 * H + x.hd) * D;
-    __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + ((size_t)x.tok0 * H + x.hd) * D;
     const size_t rowp = (size_t)H * D;
+    const size_t gbase = ((size_t)x.tok0 * H + x.hd) * D;
+    __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + gbase;
+    __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + gbase;
+    __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + gbase;
     if (ok) {
+        float acc = 0.f;   // group A: <q, dq> ; group B: <v, dXv> over this thread's columns
 #pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
-            const int ib = i0 + part * 8;
-            float a[8], b[8], xk[8], xv[8];
-            tmem_ld8(tmem + lane_base + slot(4) + ib, a);
-            tmem_ld8(tmem + lane_base + slot(1) + ib, b);
-            tmem_ld8(tmem + lane_base + slot(2) + ib, xk);
-            tmem_ld8(tmem + lane_base + slot(3) + ib, xv);
+        for (int part = 0; part < 4; ++part) {
+            const int cb = cb0 + part * 8;
+            float a[8], b[8], t8[8];
+            tmem_ld8(tmem + lane_base + 0 + cb, a);       // A: dO h^T      B: dXk
+            tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: (dP.D) K    B: dXv
             tmem_wait_ld();
-            chunk_store(sm + DXKT, 128, f, ib >> 3, xk);
-            chunk_store(sm + DXVT, 128, f, ib >> 3, xv);
+            if (ga) {
+                chunk_load(sm + QK, 128, tr, cb >> 3, t8);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float dq = fmaf(sc * Gam[ib + i], a[i], b[i]);   // dq = scale Gam (dO h^T) + dPD K
-                tile_put(sm + STG_QK, 64, ib + i, f, dq);
-                a[i] = tile_get(sm + QK, 128, ib + i, f) * dq;          // <q, dq> partial
-                tile_put(sm + STG_V, 64, ib + i, f, bb[ib + i] * xv[i]);  // dv = w dXv
-                xv[i] *= tile_get(sm + VT, 64, ib + i, f);              // dw partial
+                for (int j = 0; j < 8; ++j) {
+                    a[j] = fmaf(sc * Gam[tr], a[j], b[j]);              // dq = scale Gam (dO h^T) + (dP.D) K
+                    acc = fmaf(t8[j], a[j], acc);
+                }
+                chunk_store(sm + STG_A, 64, tr, cb >> 3, a);
+            } else {
+                chunk_store(sm + DXK, 64, tr, cb >> 3, a);
+                chunk_store(sm + DXV, 64, tr, cb >> 3, b);
+                chunk_load(sm + VT, 64, tr, cb >> 3, t8);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    acc = fmaf(t8[j], b[j], acc);                       // dw partial
+                    b[j] *= bb[tr];                                     // dv = w dXv
+                }
+                chunk_store(sm + STG_B, 64, tr, cb >> 3, b);
             }
-            const float s0 = reduce8(a, lane), s1 = reduce8(xv, lane);
-            if (lane < 8) { red[0][grp][q4][part * 8 + lane] = s0; red[1][grp][q4][part * 8 + lane] = s1; }
-            GDN_TICK(2, 16 + part);
         }
+        red[ga ? 0 : 1][grp][tr] = acc;
     }
     tc_fence_before();
     fence_async_smem();
-    GDN_TICK(2, 20);
     __syncthreads();
     GDN_TICK(2, 10);
 
-    // ---- phase 5 (the staged dq and dv leave while the MMAs run)
+    // ---- phase 5
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile<64, 64, 128>(tmem + slot(0), op_mn_major(sm + DXKT, 128), op_mn_major(sm + WT, 128), false);
-        mma_tile<64, 64, 128>(tmem + slot(0), op_mn_major(sm + DXVT, 128), op_mn_major(sm + UTT, 128), true);
+        mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
+        mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
     }
-    GDN_TICK(2, 21);
-    if (ok) {
-        flush_rows(sm + STG_QK, gdq, rowp, x.len);
-        flush_rows(sm + STG_V, gdv, rowp, x.len);
+    if (ok) {   // the staged dq and dv rows leave with coalesced 16-byte stores while the MMAs run
+        flush_rows(sm + STG_A, gdq, rowp, x.len);
+        flush_rows(sm + STG_B, gdv, rowp, x.len);
     }
-    GDN_TICK(2, 22);
     __syncthreads();   // the staging tiles are rewritten below
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
-    GDN_TICK(2, 23);
     if (ok) {
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
-            const int jb = j0 + part * 8;
-            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
+            const int jb = j0b + part * 8;
+            tmem_ld8(tmem + lane_base + 384 + jb, v);
             tmem_wait_ld();
-            if (lane < 16) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
+            if (!ga) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    v[j] = (jb + j < mi) ? -v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
-                    w[j] = bb[mi] * v[j];
+                    v[j] = (jb + j < tr) ? -v[j] * ex2(gl[tr] - gl[jb + j]) : 0.f;
+                    w[j] = bb[tr] * v[j];
                 }
-                chunk_store(sm + GT, 64, mi, jb >> 3, v);
-                chunk_store(sm + BGT, 64, mi, jb >> 3, w);
+                chunk_store(sm + GT, 64, tr, jb >> 3, v);
+                chunk_store(sm + BGT, 64, tr, jb >> 3, w);
             }
-            GDN_TICK(2, 24 + part);
         }
     }
-    GDN_TICK(2, 28);
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
@@ -799,34 +882,40 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     // ---- phase 6
     if (ok && threadIdx.x == 0) {
         tc_fence_after();
-        mma_tile<128, 64, 64>(tmem + slot(4), op_mn_major(sm + QK, 128, 64), op_k_major(sm + GT, 64), false);
-        mma_tile<128, 64, 64>(tmem + slot(6), op_mn_major(sm + QK, 128, 64), op_mn_major(sm + BGT, 64), true);
+        mma_tile<64, 128, 64>(tmem + 256 + LB, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);       // G K
+        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), true);           // += (bG)^T K
+        mma_tile<64, 128, 64>(tmem + 0, op_k_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), false);             // (bG) K
+        mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);               // T^T dW again, group A
         mma_commit(&bar_mma);
     }
     GDN_TICK(2, 13);
     GDN_WAIT_MMA(26)
     if (ok) {
+        float acc = 0.f;   // group A: <k, dk^col> ; group B: db = <k, G K + Gam dXk>
 #pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
-            const int ib = i0 + part * 8;
-            float y[8], t[8], c1[8], c2[8];
-            tmem_ld8(tmem + lane_base + slot(4) + ib, y);
-            tmem_ld8(tmem + lane_base + slot(2) + ib, t);
-            tmem_ld8(tmem + lane_base + slot(6) + ib, c1);
-            tmem_ld8(tmem + lane_base + slot(7) + ib, c2);
+        for (int part = 0; part < 4; ++part) {
+            const int cb = cb0 + part * 8;
+            float a[8], b[8], c8[8], d8[8], kk[8];
+            tmem_ld8(tmem + lane_base + 0 + cb, a);       // A: (bG) K        B: dXk
+            tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: dXk
+            tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: dk^col part   B: G K
+            tmem_ld8(tmem + lane_base + 384 + cb, d8);    // A: U dh'^T
             tmem_wait_ld();
+            chunk_load(sm + QK, 128, 64 + tr, cb >> 3, kk);
+            if (ga) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float yy = fmaf(Gam[ib + i], t[i], y[i]);        // Y = G K + Diag(Gam) dXk ; dk^row = Diag(b) Y
-                const float kcol = fmaf(ee[ib + i], c2[i], c1[i]);      // dk^col
-                const float kk = tile_get(sm + QK, 128, 64 + ib + i, f);
-                tile_put(sm + STG_QK, 64, ib + i, f, fmaf(bb[ib + i], yy, kcol));
-                y[i] = kk * yy;                                         // db partial
-                c1[i] = kk * kcol;                                      // <k, dk^col> partial
+                for (int j = 0; j < 8; ++j) {
+                    const float kcol = fmaf(ee[tr], d8[j], c8[j]);                     // dk^col
+                    acc = fmaf(kk[j], kcol, acc);
+                    a[j] = a[j] + bb[tr] * Gam[tr] * b[j] + kcol;                      // dk = Diag(b)(G K + Gam dXk) + dk^col
+                }
+                chunk_store(sm + STG_B, 64, tr, cb >> 3, a);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], a[j], c8[j]), acc);
             }
-            const float s2 = reduce8(y, lane), s3 = reduce8(c1, lane);
-            if (lane < 8) { red[2][grp][q4][part * 8 + lane] = s2; red[3][grp][q4][part * 8 + lane] = s3; }
         }
+        red[ga ? 3 : 2][grp][tr] = acc;
     }
     // block totals of sum_j r_j and <dh', h>
     rs = warp_sum(rs);
@@ -834,10 +923,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
     __syncthreads();
     GDN_TICK(2, 14);
-    if (ok) flush_rows(sm + STG_QK, gdk, rowp, x.len);
+    if (ok) flush_rows(sm + STG_B, gdk, rowp, x.len);
     if (threadIdx.x < kC) {
-        const int i = threadIdx.x, hf = i / kTG, l = i % kTG;
-        auto tot = [&](int w) { return (red[w][hf][0][l] + red[w][hf][1][l]) + (red[w][hf][2][l] + red[w][hf][3][l]); };
+        const int i = threadIdx.x;
+        auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
         const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
         if (i < x.len) p.dbeta[(size_t)(x.tok0 + i) * H + x.hd] = db + dw;
         dgam[i] = fmaf(bb[i], db, qdq - kcol);
@@ -854,8 +943,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
         }
     }
     tc_fence_before();
-    __syncthreads();
+    __syncthreads();   // every reader of this trip's tiles and scratch is done
     GDN_TICK(2, 15);
+    if (!ok) break;
+    }
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -1005,18 +1096,33 @@ static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t 
     return cudaGetLastError();
 }
 
+static int sm_count();
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
     static bool done = false;
-    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, P.p.L.max_chunks * P.p.d.H, kWideThreads, P, st);
+    const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
+    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kWideThreads, P, st);
 }
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int chains = P.p.d.N * P.p.d.H;
     return launch_chunk_kernel(tc_scan_kernel, done, scan::SMEM_BYTES, ST_SCANS, chains * (P.scan_dirs == 2 ? 2 : 1), kThreads, P, st);
 }
+// Number of SMs of the current device (persistent kernels launch one CTA per SM).
+static int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!cached[dev]) {
+        int n = 0;
+        cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    }
+    return cached[dev];
+}
+
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
     static bool done = false;
-    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, P.p.L.max_chunks * P.p.d.H, kWideThreads, P, st);
+    const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
+    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kWideThreads, P, st);
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static bool done = false;
@@ -1059,6 +1165,9 @@ cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st
 }  // namespace gdn
 
 #ifdef GDN_PHASE_TIMING
+extern "C" int gdn_debug_tick_trip(int trip) {
+    return (int)cudaMemcpyToSymbol(gdn::g_tick_trip, &trip, sizeof(int));
+}
 extern "C" int gdn_debug_ticks(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks, sizeof(long long) * 4 * 32);
 }

@@ -93,16 +93,17 @@ __device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloa
 }
 
 struct ChunkInfo { int c, hd, ch, tok0, len; };
-__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) {
+__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int item) {
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    x.c = blockIdx.x / p.d.H;
-    x.hd = blockIdx.x % p.d.H;
+    x.c = item / p.d.H;
+    x.hd = item % p.d.H;
     if (x.c >= hdr->n_chunks) return false;
-    x.ch = blockIdx.x;
+    x.ch = item;
     x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
     x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
     return true;
 }
+__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) { return chunk_info(p, x, (int)blockIdx.x); }
 
 // Wait for the MMAs committed to `bar`; on a timeout record it once.
 #define GDN_WAIT_MMA(where)                                                    \
