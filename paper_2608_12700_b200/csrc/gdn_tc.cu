@@ -46,6 +46,7 @@ constexpr int kTG = kC / kGroups;             // token columns per group (16)
 struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
+    CUtensorMap tm_dq, tm_dk, tm_dv;       // same geometry, for the gradient stores of full chunks
     int with_bwd;                          // prep: also produce E
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
 };
@@ -557,14 +558,16 @@ constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      
 constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
-constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each
-constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
+constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each, then staged dk
+constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB   later staged dq, dv
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
-constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later staged dq, then G and Diag(b) G [64][64] each
-constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dv, then staged dk
+constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each
+constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
 constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
-constexpr uint32_t STG_A = UT, STG_B = DUT;   // token-major staging of dq | dv and dk (free once phase 4 has read U^T, dU^T)
+// token-major staging of dq, dv (over dh', which phase 4 reads last) and of dk (over dXk, dXv, which phase 5 reads last):
+// nothing else reuses these regions within a trip, so the asynchronous stores need no wait before the trip ends
+constexpr uint32_t STG_A = DH, STG_B = DH + 16384, STG_K = HH;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
@@ -801,6 +804,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     }
     GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
+    const bool full = x.len == kC;
     const size_t rowp = (size_t)H * D;
     const size_t gbase = ((size_t)x.tok0 * H + x.hd) * D;
     __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + gbase;
@@ -848,12 +852,19 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
+    } else if (ok && full && threadIdx.x == 32) {
+        // staged dq, dv leave through the async proxy (generic global stores would stall the next proxy fence); a
+        // thread of another warp issues them so that the MMA issue is not delayed
+        for (int cb = 0; cb < 2; ++cb) {
+            tma_store_2d(&P.tm_dq, x.hd * D + cb * 64, x.tok0, sm + STG_A + cb * 8192);
+            tma_store_2d(&P.tm_dv, x.hd * D + cb * 64, x.tok0, sm + STG_B + cb * 8192);
+        }
+        bulk_commit();
     }
-    if (ok) {   // the staged dq and dv rows leave with coalesced 16-byte stores while the MMAs run
+    if (ok && !full) {   // ragged tail: rows beyond the sequence must not be written
         flush_rows(sm + STG_A, gdq, rowp, x.len);
         flush_rows(sm + STG_B, gdv, rowp, x.len);
     }
-    __syncthreads();   // the staging tiles are rewritten below
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
     if (ok) {
@@ -909,7 +920,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
                     acc = fmaf(kk[j], kcol, acc);
                     a[j] = a[j] + bb[tr] * Gam[tr] * b[j] + kcol;                      // dk = Diag(b)(G K + Gam dXk) + dk^col
                 }
-                chunk_store(sm + STG_B, 64, tr, cb >> 3, a);
+                chunk_store(sm + STG_K, 64, tr, cb >> 3, a);
             } else {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], a[j], c8[j]), acc);
@@ -921,9 +932,18 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     rs = warp_sum(rs);
     hh = warp_sum(hh);
     if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
+    fence_async_smem();
     __syncthreads();
     GDN_TICK(2, 14);
-    if (ok) flush_rows(sm + STG_B, gdk, rowp, x.len);
+    if (ok && full) {
+        if (threadIdx.x == 32) {
+            for (int cb = 0; cb < 2; ++cb) tma_store_2d(&P.tm_dk, x.hd * D + cb * 64, x.tok0, sm + STG_K + cb * 8192);
+            bulk_commit();
+            bulk_wait_read<0>();   // all staged gradients of this trip have left shared memory
+        }
+    } else if (ok) {
+        flush_rows(sm + STG_K, gdk, rowp, x.len);
+    }
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
         auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
@@ -1078,6 +1098,11 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_v, p.v, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_do, with_bwd ? p.dO : p.v, rows, cols, pitch, 64)) return false;
+    if (with_bwd) {
+        if (!tc::make_tmap_bf16_2d(&P.tm_dq, p.dq, rows, cols, pitch, 64)) return false;
+        if (!tc::make_tmap_bf16_2d(&P.tm_dk, p.dk, rows, cols, pitch, 64)) return false;
+        if (!tc::make_tmap_bf16_2d(&P.tm_dv, p.dv, rows, cols, pitch, 64)) return false;
+    }
     return true;
 }
 
