@@ -952,15 +952,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
         dgam[i] = fmaf(bb[i], db, qdq - kcol);
     }
     __syncthreads();
-    if (threadIdx.x == 0 && ok) {
+    if (warp == 0 && ok) {
         float rsum = 0.f, hsum = 0.f;
         for (int w = 0; w < kWideThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
-        dgam[kC - 1] += rsum + Gam[kC - 1] * hsum;
-        float run = 0.f;   // gam_i = sum_{j<=i} g_j  =>  dg_j = sum_{i>=j} dgam_i
-        for (int i = kC - 1; i >= 0; --i) {
-            run += dgam[i];
-            if (i < x.len) p.dg[(size_t)(x.tok0 + i) * H + x.hd] = run;
-        }
+        write_dg_suffix(dgam, nullptr, rsum + Gam[kC - 1] * hsum, p.dg + (size_t)x.tok0 * H + x.hd, (size_t)H, x.len, lane);
     }
     tc_fence_before();
     __syncthreads();   // every reader of this trip's tiles and scratch is done

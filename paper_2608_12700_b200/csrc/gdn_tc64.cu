@@ -23,6 +23,7 @@ constexpr int kThreads64 = 256;   // 8 warps: lane quadrant = warp % 4 (rows 16 
 struct Tc64Params {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 64] bf16, boxes of 64 rows x 64 columns
+    CUtensorMap tm_dq, tm_dk, tm_dv;       // same geometry, for the gradient stores of full chunks
 };
 
 // chunk-local cumulative log decay, one warp per chunk-head (lane l owns tokens l and l + 32)
@@ -401,44 +402,39 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         GDN_WAIT_MMA(52)
         if (!ok) break;
         float dot = 0.f;   // group B: <q_r, dq_r> - <k_r, dk_r> over this thread's columns
-        {
-            const size_t grow = ((size_t)(tok0 + r) * H + hd) * D6;
-            __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + grow;
-            __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + grow;
-            __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + grow;
-            const bool wr = r < len;
+        // Gradient rows are staged token-major over tiles that phase 2 has finished with (dv over P, dk over dP.D, dq
+        // over Diag(Gam) dO) and leave by TMA stores; generic global stores here would be one 16-byte piece per row.
 #pragma unroll 1
-            for (int part = 0; part < 4; ++part) {
-                float a[8], b[8], x[8];
-                const int jb = cb0 + part * 8;
-                tmem_ld8(tmem + lane_base + C3 + jb, a);     // A: P^T dO        B: (dP.D)^T Q
-                tmem_ld8(tmem + lane_base + C2 + jb, b);     // A: K dh'         B: V dh'^T
-                tmem_wait_ld();
-                if (ga) {
+        for (int part = 0; part < 4; ++part) {
+            float a[8], b[8], x[8];
+            const int jb = cb0 + part * 8;
+            tmem_ld8(tmem + lane_base + C3 + jb, a);     // A: P^T dO        B: (dP.D)^T Q
+            tmem_ld8(tmem + lane_base + C2 + jb, b);     // A: K dh'         B: V dh'^T
+            tmem_wait_ld();
+            if (ga) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) a[j] = fmaf(sc, a[j], ee[r] * b[j]);      // dv = scale P^T dO + Diag(e) K dh'
-                    if (wr) *reinterpret_cast<uint4*>(gdv + jb) = pack8(a);
-                } else {
-                    chunk_load(tiles + KT, 64, r, jb >> 3, x);
+                for (int j = 0; j < 8; ++j) a[j] = fmaf(sc, a[j], ee[r] * b[j]);      // dv = scale P^T dO + Diag(e) K dh'
+                chunk_store(sm + PX, 64, r, jb >> 3, a);
+            } else {
+                chunk_load(tiles + KT, 64, r, jb >> 3, x);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        a[j] = fmaf(ee[r], b[j], a[j]);                                    // dk = (dP.D)^T Q + Diag(e) V dh'^T
-                        dot = fmaf(-x[j], a[j], dot);
-                    }
-                    if (wr) *reinterpret_cast<uint4*>(gdk + jb) = pack8(a);
+                for (int j = 0; j < 8; ++j) {
+                    a[j] = fmaf(ee[r], b[j], a[j]);                                    // dk = (dP.D)^T Q + Diag(e) V dh'^T
+                    dot = fmaf(-x[j], a[j], dot);
                 }
-                tmem_ld8(tmem + lane_base + C0 + jb, a);     //                  B: dO h^T
-                tmem_ld8(tmem + lane_base + C1 + jb, b);     //                  B: (dP.D) K
-                tmem_wait_ld();
-                if (!ga) {
-                    chunk_load(tiles + QT, 64, r, jb >> 3, x);
+                chunk_store(sm + DPD, 64, r, jb >> 3, a);
+            }
+            tmem_ld8(tmem + lane_base + C0 + jb, a);     //                  B: dO h^T
+            tmem_ld8(tmem + lane_base + C1 + jb, b);     //                  B: (dP.D) K
+            tmem_wait_ld();
+            if (!ga) {
+                chunk_load(tiles + QT, 64, r, jb >> 3, x);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        a[j] = fmaf(sc * Gam[r], a[j], b[j]);                              // dq = scale Gam dO h^T + (dP.D) K
-                        dot = fmaf(x[j], a[j], dot);
-                    }
-                    if (wr) *reinterpret_cast<uint4*>(gdq + jb) = pack8(a);
+                for (int j = 0; j < 8; ++j) {
+                    a[j] = fmaf(sc * Gam[r], a[j], b[j]);                              // dq = scale Gam dO h^T + (dP.D) K
+                    dot = fmaf(x[j], a[j], dot);
                 }
+                chunk_store(sm + DH, 64, r, jb >> 3, a);
             }
         }
         if (!ga) dgp[half][r] = dot;
@@ -455,16 +451,34 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         hh = warp_sum(ga ? hh : 0.f);
         if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
         tc_fence_before();
-        __syncthreads();   // every reader of this stage's tiles is done; partial sums are visible
-        if (threadIdx.x == 0) {
-            if (s + STAGES < nsteps) fill(s + STAGES);
+        fence_async_smem();
+        __syncthreads();   // every reader of this stage's tiles is done; partial sums and staged rows are visible
+        if (len == kC) {
+            if (threadIdx.x == 32) {
+                tma_store_2d(&P.tm_dv, hd * D6, tok0, sm + PX);
+                tma_store_2d(&P.tm_dk, hd * D6, tok0, sm + DPD);
+                tma_store_2d(&P.tm_dq, hd * D6, tok0, sm + DH);
+                bulk_commit();
+                if (s + STAGES < nsteps) fill(s + STAGES);
+                bulk_wait_read<0>();   // the staging tiles are rewritten right after the next barrier
+            }
+        } else {   // ragged tail: rows beyond the sequence must not be written
+            const size_t gbase = ((size_t)tok0 * H + hd) * D6;
+            for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
+                const int i = t >> 3, chk = t & 7;
+                if (i < len) {
+                    const size_t o = gbase + (size_t)i * H * D6 + chk * 8;
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dv) + o) = *reinterpret_cast<const uint4*>(sm + PX + tile_chunk_off(64, i, chk));
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dk) + o) = *reinterpret_cast<const uint4*>(sm + DPD + tile_chunk_off(64, i, chk));
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dq) + o) = *reinterpret_cast<const uint4*>(sm + DH + tile_chunk_off(64, i, chk));
+                }
+            }
+            if (threadIdx.x == 32 && s + STAGES < nsteps) fill(s + STAGES);
+        }
+        if (warp == 0) {
             float rsum = 0.f, hsum = 0.f;
             for (int w = 0; w < kThreads64 / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
-            float run = 0.f;   // gam_i = sum_{j<=i} g_j  =>  dg_j = sum_{i>=j} dgam_i
-            for (int i = kC - 1; i >= 0; --i) {
-                run += dgp[0][i] + dgp[1][i] + (i == kC - 1 ? rsum + Ge * hsum : 0.f);
-                if (i < len) p.dg[(size_t)(tok0 + i) * H + hd] = run;
-            }
+            write_dg_suffix(dgp[0], dgp[1], rsum + Ge * hsum, p.dg + (size_t)tok0 * H + hd, (size_t)H, len, lane);
         }
     }
     if (p.dh0 && ok && ga) {
@@ -492,6 +506,11 @@ static bool fill_params64(Tc64Params& P, const Problem& p, bool with_bwd) {
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_v, p.v, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_do, with_bwd ? p.dO : p.v, rows, cols, pitch, 64)) return false;
+    if (with_bwd) {
+        if (!tc::make_tmap_bf16_2d(&P.tm_dq, p.dq, rows, cols, pitch, 64)) return false;
+        if (!tc::make_tmap_bf16_2d(&P.tm_dk, p.dk, rows, cols, pitch, 64)) return false;
+        if (!tc::make_tmap_bf16_2d(&P.tm_dv, p.dv, rows, cols, pitch, 64)) return false;
+    }
     return true;
 }
 

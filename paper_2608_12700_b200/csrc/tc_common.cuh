@@ -92,6 +92,22 @@ __device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloa
     }
 }
 
+// dg_j = sum_{i >= j} dgam_i inside a chunk (gam_i = sum_{j <= i} g_j), by one warp: lane l owns tokens l and l + 32.
+// v0 + v1 (two partial arrays, v1 may be null) are the 64 values of dgam; `last_extra` is added to the last one.
+__device__ __forceinline__ void write_dg_suffix(const float* v0, const float* v1, float last_extra, float* dg, size_t stride,
+                                                int len, int lane) {
+    float a = v0[lane] + (v1 ? v1[lane] : 0.f);
+    float b = v0[lane + 32] + (v1 ? v1[lane + 32] : 0.f) + (lane == 31 ? last_extra : 0.f);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float ta = __shfl_down_sync(0xffffffffu, a, o), tb = __shfl_down_sync(0xffffffffu, b, o);
+        if (lane + o < 32) { a += ta; b += tb; }
+    }
+    a += __shfl_sync(0xffffffffu, b, 0);
+    if (lane < len) dg[(size_t)lane * stride] = a;
+    if (lane + 32 < len) dg[(size_t)(lane + 32) * stride] = b;
+}
+
 struct ChunkInfo { int c, hd, ch, tok0, len; };
 __device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int item) {
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
