@@ -166,9 +166,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         gam[i] = g; bb[i] = b; ww[i] = b;
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int i = 0; i < kC; ++i) { s += gam[i]; gam[i] = s; }
+    if (warp == 0) {   // inclusive prefix sum of the 64 log decays: lane l owns tokens l and l + 32
+        float a = gam[lane], b = gam[lane + 32];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
+            if (lane >= o) { a += ua; b += ub; }
+        }
+        b += __shfl_sync(0xffffffffu, a, 31);
+        gam[lane] = a;
+        gam[lane + 32] = b;
     }
     __syncthreads();
     if (threadIdx.x < kC) {
@@ -240,8 +247,11 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         }
     }
     __syncthreads();
+    GDN_TICK(0, 16);
     inv_level<1>(Af, Tf, Sf);
+    GDN_TICK(0, 17);
     inv_level<2>(Af, Tf, Sf);
+    GDN_TICK(0, 18);
     inv_level<3>(Af, Tf, Sf);
     GDN_TICK(0, 4);
     for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
@@ -353,14 +363,17 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     tc_fence_before();
     fence_async_smem();
     __syncthreads();
+    // one bulk store per image, issued by threads of three different warps (bulk copies are slow to issue); each waits
+    // until its store has read shared memory, which the next trip overwrites
     if (threadIdx.x == 0) {
-        if (ok) {
-            bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + QK, 32768);
-            bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + VO, 32768);
-            if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768);
-            bulk_commit();
-        }
-        bulk_wait_read<0>();  // shared memory must stay valid until every bulk store has read it
+        if (ok) { bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + QK, 32768); bulk_commit(); }
+        bulk_wait_read<0>();   // also covers the T, W^T and U~^T stores issued earlier by this thread
+    } else if (threadIdx.x == 32) {
+        if (ok) { bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + VO, 32768); bulk_commit(); }
+        bulk_wait_read<0>();
+    } else if (threadIdx.x == 64 && bwd) {
+        if (ok) { bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768); bulk_commit(); }
+        bulk_wait_read<0>();
     }
     tc_fence_before();
     __syncthreads();          // the next trip overwrites the tiles

@@ -91,6 +91,31 @@ def test_forward_outputs_match_oracle(dtype, dk, dv):
     assert rel(got["hT"], ref["hT"]) < TOL[dtype]
 
 
+def test_erase_gate_zero_makes_the_solve_vanish_bitwise(family):
+    """Paper, Section 4.1: b = 0 gives M = 0 and T = I exactly; checked on the stored chunk factors."""
+    wl = small("beta_zero", dtype="bf16", B=1, T=192, H=2, d_k=128, d_v=128, states=True, seed=24)
+    wl.beta[:] = 0.0
+    buf = runner.to_device(wl)
+    runner.run_bwd(buf)
+    assert binding.gdn_last_device_status(buf.workspace) == 0
+    for c in range(3):
+        for hd in range(2):
+            T = binding.gdn_debug_read(buf.desc, buf.workspace, "T", c, hd)
+            W = binding.gdn_debug_read(buf.desc, buf.workspace, "W", c, hd)
+            assert np.array_equal(T, np.eye(64, dtype=np.float32))
+            assert not np.any(W)
+    check_against_oracle(wl, runner.fetch(buf))
+
+
+def test_nan_propagates_on_the_tensor_core_path():
+    wl = small("nan_tc", dtype="bf16", B=2, T=192, H=2, d_k=128, d_v=128, seed=25)
+    wl.v[70, 1, 3] = np.nan        # batch row 0, token 70, head 1
+    got = runner.backward(wl)
+    assert np.isnan(got["dk"][:192, 1]).any() and np.isnan(got["dbeta"][:192, 1]).any()
+    assert np.isfinite(got["dk"][:, 0]).all() and np.isfinite(got["dq"][:, 0]).all()   # other head
+    assert np.isfinite(got["dk"][192:]).all()                                          # other batch row
+
+
 def test_kernel_family_dispatch():
     mk = lambda **kw: binding.make_desc(**dict(dict(B=1, T=64, H=1, d_k=128, d_v=128, N=1, dtype="bf16"), **kw))
     assert binding.gdn_kernel_path(mk()) == "tcgen05_bf16"
