@@ -51,24 +51,38 @@ struct TcParams {
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
 };
 
-// One block diagonal (distance DIST below the main one) of the blocked inverse of I + A, 16 x 16 blocks:
-// T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc).  Af, Tf, Sf are fp32 [64][65] in shared memory.
-template <int DIST>
-__device__ __forceinline__ void inv_level(const float* Af, float* Tf, float* Sf) {
-    for (int o = threadIdx.x; o < (4 - DIST) * 256; o += blockDim.x) {
-        const int cb = (o >> 8) * 16, rb = cb + DIST * 16, ii = (o >> 4) & 15, jj = o & 15;
-        float s = 0.f;
+// Blocked inverse of I + A (unit lower triangular, 16 x 16 blocks), fp32 in shared memory, rows of kLdi floats:
+//   T_rr = (I + A_rr)^-1 ;  At_rk = T_rr A_rk (r > k) ;  T_rc = -sum_{k=c}^{r-1} At_rk T_kc, one block diagonal at a time.
+// These steps are bound by shared-memory load issue, so a thread produces four adjacent outputs of a row: one scalar
+// (broadcast) and one 16-byte load feed four FMAs.  inv_premul forms every At_rk; inv_level fills block diagonal DIST.
+constexpr int kLdi = 68;   // row pitch: 16-byte aligned rows, conflict-free for the access patterns below
+__device__ __forceinline__ void inv_premul(const float* Af, const float* Tf, float* Sf) {
+    // six blocks below the diagonal: (1,0) (2,0) (2,1) (3,0) (3,1) (3,2)
+    for (int o = threadIdx.x; o < 6 * 64; o += blockDim.x) {
+        const int blk = o >> 6, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
+        const int rb = (blk == 0 ? 1 : blk < 3 ? 2 : 3) * 16, cb = (blk == 0 ? 0 : blk < 3 ? blk - 1 : blk - 3) * 16;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int m = 0; m < 16 * DIST; ++m) s = fmaf(Af[(rb + ii) * 65 + cb + m], Tf[(cb + m) * 65 + cb + jj], s);
-        Sf[(rb + ii) * 65 + cb + jj] = s;
+        for (int m = 0; m < 16; ++m) {   // T_rr is lower triangular: zeros above the diagonal
+            const float a = Tf[(rb + ii) * kLdi + rb + m];
+            const float4 v = *reinterpret_cast<const float4*>(Af + (rb + m) * kLdi + cb + j4);
+            s.x = fmaf(a, v.x, s.x); s.y = fmaf(a, v.y, s.y); s.z = fmaf(a, v.z, s.z); s.w = fmaf(a, v.w, s.w);
+        }
+        *reinterpret_cast<float4*>(Sf + (rb + ii) * kLdi + cb + j4) = s;
     }
-    __syncthreads();
-    for (int o = threadIdx.x; o < (4 - DIST) * 256; o += blockDim.x) {
-        const int cb = (o >> 8) * 16, rb = cb + DIST * 16, ii = (o >> 4) & 15, jj = o & 15;
-        float s = 0.f;
+}
+template <int DIST>
+__device__ __forceinline__ void inv_level(const float* At, float* Tf) {
+    for (int o = threadIdx.x; o < (4 - DIST) * 64; o += blockDim.x) {
+        const int cb = (o >> 6) * 16, rb = cb + DIST * 16, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int m = 0; m < 16; ++m) s = fmaf(Tf[(rb + ii) * 65 + rb + m], Sf[(rb + m) * 65 + cb + jj], s);   // T_rr is lower triangular: zeros above
-        Tf[(rb + ii) * 65 + cb + jj] = -s;
+        for (int m = 0; m < 16 * DIST; ++m) {
+            const float a = At[(rb + ii) * kLdi + cb + m];
+            const float4 v = *reinterpret_cast<const float4*>(Tf + (cb + m) * kLdi + cb + j4);
+            s.x = fmaf(a, v.x, s.x); s.y = fmaf(a, v.y, s.y); s.z = fmaf(a, v.z, s.z); s.w = fmaf(a, v.w, s.w);
+        }
+        *reinterpret_cast<float4*>(Tf + (rb + ii) * kLdi + cb + j4) = make_float4(-s.x, -s.y, -s.z, -s.w);
     }
     __syncthreads();
 }
@@ -88,7 +102,7 @@ constexpr uint32_t WET = WT + 16384;          // (Diag(e) W)^T
 constexpr uint32_t UTT = WET + 16384;         // U~^T  [128 dv][64]
 constexpr uint32_t UET = UTT + 16384;         // (Diag(e) U~)^T
 constexpr uint32_t X = UET + 16384;           // fp32 A and T during the inversion; then R = Diag(Gam) dO and
-constexpr uint32_t XA = X, XT = X + 16640;    // (P^T dO)^T; finally the E image
+constexpr uint32_t XA = X, XT = X + 17408;    // (P^T dO)^T; finally the E image
 constexpr uint32_t XR = X, XPDO = X + 16384;
 constexpr uint32_t TILES_END = X + 34816;
 constexpr uint32_t SMEM_BYTES = TILES_END + 1024 /* alignment slack */;
@@ -109,7 +123,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gam[kC], gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC];
+    __shared__ __align__(16) float gam[kC], gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC], bgam[kC];
     __shared__ uint64_t bar_qk, bar_vo, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -182,6 +196,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         const int i = threadIdx.x;
         gl[i] = gam[i] * kLog2e;
         Gam[i] = expf(gam[i]);
+        bgam[i] = bb[i] * Gam[i];
         ee[i] = expf(gam[kC - 1] - gam[i]);
         reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gam[i];
     }
@@ -205,10 +220,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
         mma_commit(&bar_mma);
     }
-    float* Af = reinterpret_cast<float*>(sm + XA);   // [64][65]  strictly lower part of I + A
-    float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][65]  T
-    float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][65]  scratch of the blocked inversion
-    for (int t = threadIdx.x; t < kC * 65; t += blockDim.x) Tf[t] = 0.f;
+    float* Af = reinterpret_cast<float*>(sm + XA);   // [64][kLdi]  strictly lower part of I + A
+    float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][kLdi]  T
+    float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
+    for (int t = threadIdx.x; t < kC * kLdi; t += blockDim.x) Tf[t] = 0.f;
     GDN_WAIT_MMA(2)
     GDN_TICK(0, 2);
     if (ok) {
@@ -225,7 +240,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
                 chunk_store(sm + PT, 64, i, jb >> 3, v);
             } else {        // A_ij = b_i (k_i . k_j) exp(gam_i - gam_j), j < i
 #pragma unroll
-                for (int j = 0; j < 8; ++j) Af[i * 65 + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) Af[i * kLdi + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
             }
         }
     }
@@ -241,29 +256,32 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         for (int i = 0; i < 16; ++i) {
             float s = (i == j) ? 1.f : 0.f;
 #pragma unroll
-            for (int m = 0; m < i; ++m) s = fmaf(-Af[(b0 + i) * 65 + b0 + m], t[m], s);
+            for (int m = 0; m < i; ++m) s = fmaf(-Af[(b0 + i) * kLdi + b0 + m], t[m], s);
             t[i] = s;
-            Tf[(b0 + i) * 65 + b0 + j] = s;
+            Tf[(b0 + i) * kLdi + b0 + j] = s;
         }
     }
     __syncthreads();
     GDN_TICK(0, 16);
-    inv_level<1>(Af, Tf, Sf);
+    inv_premul(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
+    __syncthreads();
+    inv_level<1>(Sf, Tf);
     GDN_TICK(0, 17);
-    inv_level<2>(Af, Tf, Sf);
+    inv_level<2>(Sf, Tf);
     GDN_TICK(0, 18);
-    inv_level<3>(Af, Tf, Sf);
+    inv_level<3>(Sf, Tf);
     GDN_TICK(0, 4);
     for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
         const int i = t >> 3, cch = t & 7;
         float a[8], b[8], w8[8];
+        *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8);
+        *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8 + 4);
+        *reinterpret_cast<float4*>(b) = *reinterpret_cast<const float4*>(bgam + cch * 8);
+        *reinterpret_cast<float4*>(b + 4) = *reinterpret_cast<const float4*>(bgam + cch * 8 + 4);
+        *reinterpret_cast<float4*>(w8) = *reinterpret_cast<const float4*>(ww + cch * 8);
+        *reinterpret_cast<float4*>(w8 + 4) = *reinterpret_cast<const float4*>(ww + cch * 8 + 4);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int m = cch * 8 + k;
-            a[k] = Tf[i * 65 + m];
-            b[k] = a[k] * bb[m] * Gam[m];
-            w8[k] = a[k] * ww[m];
-        }
+        for (int k = 0; k < 8; ++k) { b[k] *= a[k]; w8[k] *= a[k]; }
         chunk_store(sm + TT, 64, i, cch, a);
         chunk_store(sm + TP, 64, i, cch, b);
         chunk_store(sm + TPP, 64, i, cch, w8);
