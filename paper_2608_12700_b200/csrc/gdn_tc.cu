@@ -235,12 +235,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
             tmem_wait_ld();
             const int jb = j0 + part * 8;
             if (q4 < 2) {   // P_ij = (q_i . k_j) exp(gam_i - gam_j), j <= i (mask before exponentiating)
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= i) ? v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= i) ? v[j] * ex2(gl[i] - g8[j]) : 0.f;
                 chunk_store(sm + PT, 64, i, jb >> 3, v);
             } else {        // A_ij = b_i (k_i . k_j) exp(gam_i - gam_j), j < i
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) Af[i * kLdi + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) Af[i * kLdi + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - g8[j]) : 0.f;
             }
         }
     }
@@ -320,14 +324,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
             float v[8], ve[8];
             tmem_ld8(tmem + lane_base + C_W + ib, v);
             tmem_wait_ld();
+            float e8[8];
+            ld8s(ee + ib, e8);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ve[i] = v[i] * ee[ib + i];
+            for (int i = 0; i < 8; ++i) ve[i] = v[i] * e8[i];
             chunk_store(sm + WT, 128, f, ib >> 3, v);
             chunk_store(sm + WET, 128, f, ib >> 3, ve);
             tmem_ld8(tmem + lane_base + C_U + ib, v);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ve[i] = v[i] * ee[ib + i];
+            for (int i = 0; i < 8; ++i) ve[i] = v[i] * e8[i];
             chunk_store(sm + UTT, 128, f, ib >> 3, v);
             chunk_store(sm + UET, 128, f, ib >> 3, ve);
             if (bwd) {
@@ -615,7 +621,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gl[kC], Gam[kC], ee[kC], bb[kC];
+    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC];
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kWideThreads / 32];
     __shared__ uint64_t bar_in0, bar_in1, bar_mma;
@@ -729,8 +735,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
             tmem_ld8(tmem + lane_base + slot(0) + jb, v);
             tmem_wait_ld();
             if (lane < 16) {
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - g8[j]) : 0.f;
                 chunk_store(sm + PT, 64, mi, jb >> 3, v);
             }
         }
@@ -760,11 +768,13 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
             tmem_ld8(tmem + lane_base + slot(1) + ib, t);
             tmem_ld8(tmem + lane_base + slot(2) + ib, kb);
             tmem_ld8(tmem + lane_base + slot(3) + ib, pd);
+            float e8[8];
+            ld8s(ee + ib, e8);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 u[i] -= t[i];                                       // U = U~ - W h
-                const float kbe = ee[ib + i] * kb[i];
+                const float kbe = e8[i] * kb[i];
                 rs = fmaf(kbe, u[i], rs);                           // sum_j r_j
                 pd[i] = fmaf(sc, pd[i], kbe);                       // dU = scale P^T dO + Diag(e) K dh'
             }
@@ -811,8 +821,10 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
             tmem_ld8(tmem + lane_base + 256 + ib, w);     // all lanes: dW^T
             tmem_wait_ld();
             if (!ga) {   // dPD = scale tril(dO U^T) . D
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? sc * v[j] * ex2(gl[tr] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? sc * v[j] * ex2(gl[tr] - g8[j]) : 0.f;
                 chunk_store(sm + DPD, 64, tr, jb >> 3, v);
             }
             chunk_store(sm + DWT, 128, f, ib >> 3, w);              // dW^T = -(dU h^T)^T
@@ -906,9 +918,11 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
             tmem_ld8(tmem + lane_base + 384 + jb, v);
             tmem_wait_ld();
             if (!ga) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    v[j] = (jb + j < tr) ? -v[j] * ex2(gl[tr] - gl[jb + j]) : 0.f;
+                    v[j] = (jb + j < tr) ? -v[j] * ex2(gl[tr] - g8[j]) : 0.f;
                     w[j] = bb[tr] * v[j];
                 }
                 chunk_store(sm + GT, 64, tr, jb >> 3, v);
@@ -1012,7 +1026,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_consta
     const int H = p.d.H;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gl[kC], Gam[kC];
+    __shared__ __align__(16) float gl[kC], Gam[kC];
     __shared__ uint64_t bar_in, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1067,8 +1081,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_consta
             chunk_load(sm + UTT, 128, f, ib >> 3, u);
             tmem_wait_ld();
             if (lane < 16) {
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - gl[jb + j]) : 0.f;
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - g8[j]) : 0.f;
                 chunk_store(sm + PT, 64, mi, jb >> 3, v);
             }
 #pragma unroll

@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gl[kC], Gam[kC], ee[kC];
+    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC];
     __shared__ uint64_t bar_full[STAGES], bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -183,8 +183,10 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
                 tmem_ld8(tmem + lane_base + 64 + jb, v);
                 tmem_wait_ld();
                 if (act) {
+                    float g8[8];
+                    ld8s(gl + jb, g8);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) v[j] = (jb + j <= r) ? v[j] * ex2(gl[r] - gl[jb + j]) : 0.f;
+                    for (int j = 0; j < 8; ++j) v[j] = (jb + j <= r) ? v[j] * ex2(gl[r] - g8[j]) : 0.f;
                     chunk_store(sm + PT, 64, r, jb >> 3, v);
                 }
             }
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float gl[kC], Gam[kC], ee[kC], dgp[2][kC], scal[2][kThreads64 / 32];
+    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], dgp[2][kC], scal[2][kThreads64 / 32];
     __shared__ uint64_t bar_full[STAGES], bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -375,9 +377,11 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             tmem_wait_ld();
             if (ga) {
                 chunk_load(tiles + VT, 64, r, jb >> 3, vv);
+                float g8[8];
+                ld8s(gl + jb, g8);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const float dcy = (jb + j <= r) ? ex2(gl[r] - gl[jb + j]) : 0.f;   // masked first: the exponent is never positive
+                    const float dcy = (jb + j <= r) ? ex2(gl[r] - g8[j]) : 0.f;   // masked first: the exponent is never positive
                     s8[j] *= dcy;                   // P
                     p8[j] *= sc * dcy;              // dP . D
                     rs = fmaf(kd[j], vv[j], rs);

@@ -37,6 +37,11 @@ __device__ __forceinline__ void chunk_store(unsigned char* tile, int R, int r, i
 __device__ __forceinline__ void chunk_load(const unsigned char* tile, int R, int r, int ch, float* v) {
     unpack8(*reinterpret_cast<const uint4*>(tile + tile_chunk_off(R, r, ch)), v);
 }
+// Eight consecutive floats from a 16-byte aligned shared array (two vector loads instead of eight scalar ones).
+__device__ __forceinline__ void ld8s(const float* p, float* v) {
+    *reinterpret_cast<float4*>(v) = *reinterpret_cast<const float4*>(p);
+    *reinterpret_cast<float4*>(v + 4) = *reinterpret_cast<const float4*>(p + 4);
+}
 __device__ __forceinline__ float tile_get(const unsigned char* tile, int R, int r, int c) {
     return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(tile + tile_off(R, r, c)));
 }
