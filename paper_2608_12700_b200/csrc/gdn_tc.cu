@@ -43,6 +43,7 @@ constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column hal
 constexpr int kWideThreads = 512;
 constexpr int kGroups = kWideThreads / 128;   // column groups
 constexpr int kTG = kC / kGroups;             // token columns per group (16)
+constexpr int kIntraThreads = kWideThreads + 32;   // the gradient kernel adds one warp that only issues MMAs and copies
 struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
@@ -590,26 +591,28 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 // ------------------------------------------------------------------------------------------------
 namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
-constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB
+constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB   later staged dv
 constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
 constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
 constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each, then staged dk
-constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB   later staged dq, dv
+constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
 constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each
-constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB
+constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dq
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
 constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
-// token-major staging of dq, dv (over dh', which phase 4 reads last) and of dk (over dXk, dXv, which phase 5 reads last):
-// nothing else reuses these regions within a trip, so the asynchronous stores need no wait before the trip ends
-constexpr uint32_t STG_A = DH, STG_B = DH + 16384, STG_K = HH;
+// token-major staging of dq (over dU^T, last read by the early products of phase 4), of dv (in place over V: a thread
+// overwrites exactly the chunk it has just read) and of dk (over dXk, dXv, last read by phase 5).  None of these is
+// read by the late products of phase 4 or rewritten within the trip, so the asynchronous stores need no wait before
+// the trip ends.
+constexpr uint32_t STG_A = DUT, STG_B = VT, STG_K = HH;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
 
-__global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
     using namespace intra;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
@@ -623,12 +626,18 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     unsigned char* sm = align1024(smem_raw);
     __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC];
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
-    __shared__ float dgam[kC], scal[2][kWideThreads / 32];
+    __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
     __shared__ uint64_t bar_in0, bar_in1, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    // Warps 0..15 read accumulators; warp 16 only issues: its first lane feeds the tensor pipe, and the warp spreads the
+    // bulk loads of a trip over its lanes (each such instruction costs its issuer hundreds of cycles).  Because the
+    // issuer has no readout duties, a phase can commit the products the next readout needs first and keep issuing the
+    // ones that are only needed later while the readout already runs.
+    const bool worker = warp < 16;
+    const bool issuer = threadIdx.x == kWideThreads;
 
     if (threadIdx.x == 0) {
         mbar_init(&bar_in0, 1); mbar_init(&bar_in1, 1); mbar_init(&bar_mma, 1);
@@ -650,35 +659,39 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
 #endif
     GDN_TICK(2, 0);
 
-    if (threadIdx.x == 0) {
+    if (issuer) {
         mbar_expect_tx(&bar_in0, 32768 + 16384 + 32768 + 32768);
-        for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_in0);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in0);
-        }
-        bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in0);
-        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in0);
-        bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)x.ch * 32768, 32768, &bar_in0);
         mbar_expect_tx(&bar_in1, 16384 + 16384 + 16384 + 8192);
-        for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + VT + cb * 8192, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_in1);
-            tma_load_2d(sm + DO + cb * 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_in1);
+    }
+    if (lane == 0 && worker) {   // one bulk / TMA load and one L2 prefetch per warp: their issue cost runs in parallel
+        const int cb = warp & 1, xq = x.hd * D + cb * 64;
+        switch (warp) {
+            case 0: case 1: tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_in0); break;
+            case 2: case 3: tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_in0); break;
+            case 4: bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in0); break;
+            case 5: bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in0); break;
+            case 6: bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)x.ch * 32768, 32768, &bar_in0); break;
+            case 8: case 9: tma_load_2d(sm + VT + cb * 8192, &P.tm_v, xq, x.tok0, &bar_in1); break;
+            case 10: case 11: tma_load_2d(sm + DO + cb * 8192, &P.tm_do, xq, x.tok0, &bar_in1); break;
+            case 12: bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in1); break;
+            case 13: bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)x.ch * 8192, 8192, &bar_in1); break;
+            default: break;
         }
-        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in1);
-        bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)x.ch * 8192, 8192, &bar_in1);
         ChunkInfo nx;
         if (item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x)) {   // next trip's tiles -> L2
-            for (int cb = 0; cb < 2; ++cb) {
-                prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
-                prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
-                prefetch_l2_tma_2d(&P.tm_v, nx.hd * D + cb * 64, nx.tok0);
-                prefetch_l2_tma_2d(&P.tm_do, nx.hd * D + cb * 64, nx.tok0);
+            const int xn = nx.hd * D + cb * 64;
+            switch (warp) {
+                case 0: case 1: prefetch_l2_tma_2d(&P.tm_q, xn, nx.tok0); break;
+                case 2: case 3: prefetch_l2_tma_2d(&P.tm_k, xn, nx.tok0); break;
+                case 4: prefetch_l2_bulk(p.ws + p.L.W + (size_t)nx.ch * 16384, 16384); break;
+                case 5: prefetch_l2_bulk(p.ws + p.L.hc + (size_t)nx.ch * 32768, 32768); break;
+                case 6: prefetch_l2_bulk(p.ws + p.L.dhn + (size_t)nx.ch * 32768, 32768); break;
+                case 8: case 9: prefetch_l2_tma_2d(&P.tm_v, xn, nx.tok0); break;
+                case 10: case 11: prefetch_l2_tma_2d(&P.tm_do, xn, nx.tok0); break;
+                case 12: prefetch_l2_bulk(p.ws + p.L.Ut + (size_t)nx.ch * 16384, 16384); break;
+                case 13: prefetch_l2_bulk(p.ws + p.L.Tm + (size_t)nx.ch * 8192, 8192); break;
+                default: break;
             }
-            prefetch_l2_bulk(p.ws + p.L.W + (size_t)nx.ch * 16384, 16384);
-            prefetch_l2_bulk(p.ws + p.L.Ut + (size_t)nx.ch * 16384, 16384);
-            prefetch_l2_bulk(p.ws + p.L.Tm + (size_t)nx.ch * 8192, 8192);
-            prefetch_l2_bulk(p.ws + p.L.hc + (size_t)nx.ch * 32768, 32768);
-            prefetch_l2_bulk(p.ws + p.L.dhn + (size_t)nx.ch * 32768, 32768);
         }
     }
     if (threadIdx.x < kC) {
@@ -705,12 +718,12 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 1);
 
     // ---- phase 1
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + slot(0), op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
+        mma_commit(&bar_mma);   // the P readout needs only S; the two products below are covered by phase 2's commit
         mma_tile<128, 64, 128>(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
         mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
-        mma_commit(&bar_mma);
     }
     // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up)
     float hh = 0.f;
@@ -727,7 +740,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 3);
     const int mi = q4 * 16 + lane;     // row of an M = 64 accumulator held by this lane (lanes 0..15 only)
     const int j0 = grp * kTG;
-    if (ok) {   // P_ij = (q_i . k_j) D_ij for j <= i
+    if (ok && worker) {   // P_ij = (q_i . k_j) D_ij for j <= i
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             float v[8];
@@ -749,7 +762,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 4);
 
     // ---- phase 2
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<128, 64, 64>(tmem + slot(3), op_mn_major(sm + DO, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
@@ -759,7 +772,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     const int f = q4 * 32 + lane;      // feature (lane of the transposed accumulators)
     const int i0 = grp * kTG;          // first of this thread's 32 tokens
     float rs = 0.f;
-    if (ok) {
+    if (ok && worker) {
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             const int ib = i0 + part * 8;
@@ -803,16 +816,16 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     const int j0b = grp * kTG;              // first of its 16 columns in 64-column accumulators
 
     // ---- phase 3
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + 0 + LB, op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);           // dO U^T
         mma_tile<64, 128, 128>(tmem + 0, op_k_major(sm + DO, 64), op_k_major(sm + HH, 128), false);                 // dO h^T
         mma_tile<128, 64, 128>(tmem + 256, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
-        mma_commit(&bar_mma);
+        mma_commit(&bar_mma);   // (no early commit here: the readout overwrites the dO tile, which dO h^T reads)
     }
     GDN_TICK(2, 7);
     GDN_WAIT_MMA(23)
-    if (ok) {
+    if (ok && worker) {
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
@@ -836,14 +849,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 8);
 
     // ---- phase 4
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 128, 64>(tmem + 128, op_k_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 64), false);           // (dP.D) K
-        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
-        mma_tile<64, 128, 128>(tmem + 384, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);              // U dh'^T
         mma_tile<64, 128, 64>(tmem + 0 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);            // T^T dW
         mma_tile<64, 128, 64>(tmem + 128 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DUT, 128), false);          // T^T dU
-        mma_commit(&bar_mma);
+        mma_commit(&bar_mma);   // the two dk^col products are first read after phase 6
+        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
+        mma_tile<64, 128, 128>(tmem + 384, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);              // U dh'^T
     }
     GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
@@ -853,9 +866,9 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + gbase;
     __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + gbase;
     __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + gbase;
-    if (ok) {
+    if (ok && worker) {
         float acc = 0.f;   // group A: <q, dq> ; group B: <v, dXv> over this thread's columns
-#pragma unroll 1
+#pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
             float a[8], b[8], t8[8];
@@ -890,7 +903,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 10);
 
     // ---- phase 5
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
@@ -910,7 +923,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     }
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
-    if (ok) {
+    if (ok && worker) {
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
             float v[8], w[8];
@@ -936,7 +949,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     GDN_TICK(2, 12);
 
     // ---- phase 6
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 128, 64>(tmem + 256 + LB, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);       // G K
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), true);           // += (bG)^T K
@@ -946,9 +959,9 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     }
     GDN_TICK(2, 13);
     GDN_WAIT_MMA(26)
-    if (ok) {
+    if (ok && worker) {
         float acc = 0.f;   // group A: <k, dk^col> ; group B: db = <k, G K + Gam dXk>
-#pragma unroll 1
+#pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
             float a[8], b[8], c8[8], d8[8], kk[8];
@@ -999,7 +1012,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_intra_kernel(const __grid_
     __syncthreads();
     if (warp == 0 && ok) {
         float rsum = 0.f, hsum = 0.f;
-        for (int w = 0; w < kWideThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
+        for (int w = 0; w < kIntraThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
         write_dg_suffix(dgam, nullptr, rsum + Gam[kC - 1] * hsum, p.dg + (size_t)x.tok0 * H + x.hd, (size_t)H, x.len, lane);
     }
     tc_fence_before();
@@ -1189,7 +1202,7 @@ static int sm_count() {
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
-    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kWideThreads, P, st);
+    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kIntraThreads, P, st);
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static bool done = false;
