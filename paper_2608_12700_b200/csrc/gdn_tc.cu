@@ -43,7 +43,7 @@ constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column hal
 constexpr int kWideThreads = 512;
 constexpr int kGroups = kWideThreads / 128;   // column groups
 constexpr int kTG = kC / kGroups;             // token columns per group (16)
-constexpr int kIntraThreads = kWideThreads + 32;   // the gradient kernel adds one warp that only issues MMAs and copies
+constexpr int kIntraThreads = kWideThreads + 32;   // the chunk kernels add one warp whose first lane only issues MMAs
 struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
@@ -112,7 +112,7 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF = 384, C_E = 0;
 }  // namespace prep
 
-__global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
     using namespace prep;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ... and pulls the inputs of its
@@ -130,6 +130,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    const bool worker = warp < 16;                       // warps 0..15 read accumulators and do the fp32 work
+    const bool issuer = threadIdx.x == kWideThreads;     // first lane of warp 16 feeds the tensor pipe
 
     if (threadIdx.x == 0) {
         mbar_init(&bar_qk, 1); mbar_init(&bar_vo, 1); mbar_init(&bar_mma, 1);
@@ -148,25 +150,27 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     chunk_info(p, x, item);
     GDN_TICK(0, 0);
 
-    if (threadIdx.x == 0) {
+    if (issuer) {
         mbar_expect_tx(&bar_qk, 32768);
-        for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_qk);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_qk);
-        }
         mbar_expect_tx(&bar_vo, bwd ? 32768 : 16384);
-        for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + VO + cb * 16384, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_vo);
-            if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_vo);
-        }
+    }
+    if (lane == 0 && warp < 8) {   // one TMA load and one L2 prefetch per warp: their issue cost runs in parallel
+        const int cb = warp & 1, which = warp >> 1, xq = x.hd * D + cb * 64;
         ChunkInfo nx;
-        if (item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x)) {   // next trip's inputs -> L2
-            for (int cb = 0; cb < 2; ++cb) {
-                prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
-                prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
-                prefetch_l2_tma_2d(&P.tm_v, nx.hd * D + cb * 64, nx.tok0);
-                if (bwd) prefetch_l2_tma_2d(&P.tm_do, nx.hd * D + cb * 64, nx.tok0);
-            }
+        const bool pf = item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x);   // next trip's inputs -> L2
+        const int xn = pf ? nx.hd * D + cb * 64 : 0;
+        if (which == 0) {
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_qk);
+            if (pf) prefetch_l2_tma_2d(&P.tm_q, xn, nx.tok0);
+        } else if (which == 1) {
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_qk);
+            if (pf) prefetch_l2_tma_2d(&P.tm_k, xn, nx.tok0);
+        } else if (which == 2) {
+            tma_load_2d(sm + VO + cb * 16384, &P.tm_v, xq, x.tok0, &bar_vo);
+            if (pf) prefetch_l2_tma_2d(&P.tm_v, xn, nx.tok0);
+        } else if (bwd) {
+            tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, xq, x.tok0, &bar_vo);
+            if (pf) prefetch_l2_tma_2d(&P.tm_do, xn, nx.tok0);
         }
     }
     // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
@@ -216,7 +220,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     GDN_TICK(0, 1);
 
     // ---- phase 1: S1 = [Q; K] K^T  (rows 0..63: Q K^T, rows 64..127: K K^T)
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
         mma_commit(&bar_mma);
@@ -227,7 +231,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     for (int t = threadIdx.x; t < kC * kLdi; t += blockDim.x) Tf[t] = 0.f;
     GDN_WAIT_MMA(2)
     GDN_TICK(0, 2);
-    if (ok) {
+    if (ok && worker) {
         const int i = (q4 & 1) * 32 + lane, j0 = grp * kTG;
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
@@ -296,12 +300,14 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     GDN_TICK(0, 5);
 
     // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T ; (P^T dO)^T = dO^T P
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<128, 64, 64>(tmem + C_W, op_mn_major(sm + QK, 128, 64), op_k_major(sm + TP, 64), false);
         mma_tile<128, 64, 64>(tmem + C_U, op_mn_major(sm + VO, 128, 0), op_k_major(sm + TPP, 64), false);
         if (bwd) mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
+    }
+    if (ok && threadIdx.x == 0) {
         bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
         bulk_commit();
     }
@@ -317,7 +323,7 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
         }
     }
     GDN_WAIT_MMA(3)
-    if (ok) {
+    if (ok && worker) {
         const int f = q4 * 32 + lane, i0 = grp * kTG;
 #pragma unroll 1
         for (int part = 0; part < kTG / 8; ++part) {
@@ -350,20 +356,24 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     GDN_TICK(0, 6);
 
     // ---- phase 3: Nm = K^T (Diag(e) W) ; Bf = K^T (Diag(e) U~) ; E = Q^T R - W^T (P^T dO)
-    if (ok && threadIdx.x == 0) {
+    if (ok && issuer) {
         tc_fence_after();
         mma_tile<128, 128, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
         mma_tile<128, 128, 64>(tmem + C_BF, op_mn_major(sm + QK, 128, 64), op_k_major(sm + UET, 128), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
+    }
+    if (ok && threadIdx.x == 0) {
         bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
+        bulk_commit();
+    } else if (ok && threadIdx.x == 96) {
         bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
         bulk_commit();
     }
     GDN_WAIT_MMA(4)
     GDN_TICK(0, 7);
-    if (ok) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
+    if (ok && worker) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
         const int r = q4 * 32 + lane, c0 = grp * (D / kGroups);
         const float sc = p.d.scale;
 #pragma unroll 1
@@ -399,6 +409,8 @@ __global__ void __launch_bounds__(kWideThreads, 1) tc_prep_kernel(const __grid_c
     } else if (threadIdx.x == 64 && bwd) {
         if (ok) { bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768); bulk_commit(); }
         bulk_wait_read<0>();
+    } else if (threadIdx.x == 96) {
+        bulk_wait_read<0>();   // the U~^T store issued earlier by this thread
     }
     tc_fence_before();
     __syncthreads();          // the next trip overwrites the tiles
@@ -1180,7 +1192,7 @@ static int sm_count();
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
-    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kWideThreads, P, st);
+    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kIntraThreads, P, st);
 }
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static bool done = false;
