@@ -27,11 +27,15 @@ namespace gdn {
 __device__ long long g_ticks[4][32];
 __device__ int g_tick_trip = 0;   // which trip of a persistent CTA is stamped
 __device__ int g_trip_now = 0;
+__device__ long long g_trip_ns[2][24];   // wall-clock (ns) at kernel entry [0], at each trip start [1 + trip], at exit
+__device__ __forceinline__ long long tick_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define GDN_TRIP(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (idx) < 24) g_trip_ns[kern][idx] = tick_ns(); } while (0)
 #define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (kern != 2 || g_trip_now == g_tick_trip)) g_ticks[kern][idx] = clock64(); } while (0)
 #define GDN_TICKT(tid, kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == (tid)) g_ticks[kern][idx] = clock64(); } while (0)
 #else
 #define GDN_TICK(kern, idx) do { } while (0)
 #define GDN_TICKT(tid, kern, idx) do { } while (0)
+#define GDN_TRIP(kern, idx) do { } while (0)
 #endif
 
 namespace {
@@ -113,6 +117,7 @@ constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF 
 }  // namespace prep
 
 __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
+    GDN_TRIP(0, 0);
     using namespace prep;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ... and pulls the inputs of its
@@ -144,11 +149,28 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     const uint32_t tmem = tmem_slot;
     bool ok = true;
     uint32_t mma_phase = 0, in_phase = 0;
+    // The chunk table entry and the gate values of a trip are fetched one trip ahead into registers: they are tiny, but
+    // read at the top of a trip their DRAM latency would be fully exposed.
+    ChunkInfo xn;
+    chunk_info(p, xn, blockIdx.x);
+    float ng = 0.f, nb = 0.f;
+    auto fetch_gates = [&](const ChunkInfo& c) {   // g (0 when padded) and the erase gate b of this thread's token
+        ng = nb = 0.f;
+        if ((int)threadIdx.x < c.len) {
+            const size_t idx = (size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd;
+            ng = p.g[idx];
+            nb = p.beta[idx];
+        }
+    };
+    fetch_gates(xn);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-    ChunkInfo x;
-    chunk_info(p, x, item);
+    const ChunkInfo x = xn;
+    const float g_now = ng, b_now = nb;
+    const bool has_next = item + (int)gridDim.x < n_items;
+    if (has_next) chunk_info(p, xn, item + gridDim.x);
     GDN_TICK(0, 0);
+    GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
 
     if (issuer) {
         mbar_expect_tx(&bar_qk, 32768);
@@ -156,33 +178,15 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     }
     if (lane == 0 && warp < 8) {   // one TMA load and one L2 prefetch per warp: their issue cost runs in parallel
         const int cb = warp & 1, which = warp >> 1, xq = x.hd * D + cb * 64;
-        ChunkInfo nx;
-        const bool pf = item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x);   // next trip's inputs -> L2
-        const int xn = pf ? nx.hd * D + cb * 64 : 0;
-        if (which == 0) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_qk);
-            if (pf) prefetch_l2_tma_2d(&P.tm_q, xn, nx.tok0);
-        } else if (which == 1) {
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_qk);
-            if (pf) prefetch_l2_tma_2d(&P.tm_k, xn, nx.tok0);
-        } else if (which == 2) {
-            tma_load_2d(sm + VO + cb * 16384, &P.tm_v, xq, x.tok0, &bar_vo);
-            if (pf) prefetch_l2_tma_2d(&P.tm_v, xn, nx.tok0);
-        } else if (bwd) {
-            tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, xq, x.tok0, &bar_vo);
-            if (pf) prefetch_l2_tma_2d(&P.tm_do, xn, nx.tok0);
-        }
+        if (which == 0) tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_qk);
+        else if (which == 1) tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_qk);
+        else if (which == 2) tma_load_2d(sm + VO + cb * 16384, &P.tm_v, xq, x.tok0, &bar_vo);
+        else if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, xq, x.tok0, &bar_vo);
     }
     // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
-        float g = 0.f, b = 0.f;
-        if (i < x.len) {
-            const size_t idx = (size_t)(x.tok0 + i) * H + x.hd;
-            g = p.g[idx];
-            b = p.beta[idx];
-        }
-        gam[i] = g; bb[i] = b; ww[i] = b;
+        gam[i] = g_now; bb[i] = b_now; ww[i] = b_now;
     }
     __syncthreads();
     if (warp == 0) {   // inclusive prefix sum of the 64 log decays: lane l owns tokens l and l + 32
@@ -229,6 +233,16 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][kLdi]  T
     float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
     for (int t = threadIdx.x; t < kC * kLdi; t += blockDim.x) Tf[t] = 0.f;
+    if (has_next) {   // while the product runs: next trip's gates -> registers, its input tiles -> L2
+        if (threadIdx.x < kC) fetch_gates(xn);
+        if (lane == 0 && warp >= 8 && warp < 16) {
+            const int cb = warp & 1, which = (warp >> 1) & 3, xq = xn.hd * D + cb * 64;
+            if (which == 0) prefetch_l2_tma_2d(&P.tm_q, xq, xn.tok0);
+            else if (which == 1) prefetch_l2_tma_2d(&P.tm_k, xq, xn.tok0);
+            else if (which == 2) prefetch_l2_tma_2d(&P.tm_v, xq, xn.tok0);
+            else if (bwd) prefetch_l2_tma_2d(&P.tm_do, xq, xn.tok0);
+        }
+    }
     GDN_WAIT_MMA(2)
     GDN_TICK(0, 2);
     if (ok && worker) {
@@ -417,6 +431,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     GDN_TICK(0, 8);
     if (!ok) break;
     }
+    GDN_TRIP(0, 20);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -605,10 +620,10 @@ namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
 constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB   later staged dv
 constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
-constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
+constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB   later staged dk
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
-constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each, then staged dk
+constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each
 constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
 constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each
@@ -616,15 +631,16 @@ constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
 constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
 // token-major staging of dq (over dU^T, last read by the early products of phase 4), of dv (in place over V: a thread
-// overwrites exactly the chunk it has just read) and of dk (over dXk, dXv, last read by phase 5).  None of these is
-// read by the late products of phase 4 or rewritten within the trip, so the asynchronous stores need no wait before
-// the trip ends.
-constexpr uint32_t STG_A = DUT, STG_B = VT, STG_K = HH;
+// overwrites exactly the chunk it has just read) and of dk (over W^T, last read by phase 5).  None of these is read
+// by the late products of phase 4 or rewritten within the trip (the loads that run ahead go to other regions), so
+// the asynchronous stores need no wait before the trip ends.
+constexpr uint32_t STG_A = DUT, STG_B = VT, STG_K = UT;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
 }  // namespace intra
 
-__global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
+    GDN_TRIP(1, 0);
     using namespace intra;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
@@ -639,20 +655,27 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC];
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
-    __shared__ uint64_t bar_in0, bar_in1, bar_mma;
+    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    // Warps 0..15 read accumulators; warp 16 only issues: its first lane feeds the tensor pipe, and the warp spreads the
-    // bulk loads of a trip over its lanes (each such instruction costs its issuer hundreds of cycles).  Because the
-    // issuer has no readout duties, a phase can commit the products the next readout needs first and keep issuing the
-    // ones that are only needed later while the readout already runs.
+    // Warps 0..15 read accumulators; the first lane of warp 16 only feeds the tensor pipe.  Because the issuer has no
+    // readout duties, a phase can commit the products the next readout needs first and keep issuing the ones that
+    // are only needed later while the readout already runs.
     const bool worker = warp < 16;
     const bool issuer = threadIdx.x == kWideThreads;
+    // Warp 17 only moves data.  Its first lane issues every bulk / TMA instruction of the steady state (each costs its
+    // issuer hundreds of cycles): the stores of the staged gradients, and the loads of the NEXT trip's tiles, each as
+    // soon as the region it goes to has been read for the last time in this trip.  It shares no block-wide barrier
+    // with the other warps inside the loop (they use a named barrier); it follows them through mbarriers.
+    const bool loader = warp == 17;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar_in0, 1); mbar_init(&bar_in1, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_k, 1); mbar_init(&bar_g1, 1); mbar_init(&bar_g2, 1);
+        mbar_init(&bar_ld0, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_ld2, 1);
+        mbar_init(&bar_st1, 1); mbar_init(&bar_st2, 1); mbar_init(&bar_kfree, 16); mbar_init(&bar_free, 1);
+        mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
@@ -661,72 +684,145 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     bool ok = true;
+
+    // The tiles of a trip arrive in three groups, one mbarrier each, loaded during the previous trip:
+    //   g1  Q, U~^T, dh', h, W   once the products of phase 5 are done       needed by phase 1
+    //   g2  dO, T, V             once the products of phase 6 are done       needed from phase 2 on
+    //   k   K                    once the last readout holds its K values    needed by phase 1
+    constexpr uint32_t K_BYTES = 16384, G1_BYTES = 16384 + 16384 + 32768 + 32768 + 16384, G2_BYTES = 16384 + 8192 + 16384;
+    auto load_piece = [&](int piece, const ChunkInfo& c) {
+        const int cb = piece & 1, xq = c.hd * D + cb * 64;
+        switch (piece) {
+            case 0: case 1: tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, c.tok0, &bar_k); break;
+            case 2: case 3: tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, c.tok0, &bar_g1); break;
+            case 4: bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)c.ch * 16384, 16384, &bar_g1); break;
+            case 5: bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)c.ch * 32768, 32768, &bar_g1); break;
+            case 6: bulk_load(sm + HH, p.ws + p.L.hc + (size_t)c.ch * 32768, 32768, &bar_g1); break;
+            case 7: bulk_load(sm + WT, p.ws + p.L.W + (size_t)c.ch * 16384, 16384, &bar_g1); break;
+            case 8: case 9: tma_load_2d(sm + DO + cb * 8192, &P.tm_do, xq, c.tok0, &bar_g2); break;
+            case 10: case 11: tma_load_2d(sm + VT + cb * 8192, &P.tm_v, xq, c.tok0, &bar_g2); break;
+            case 12: bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)c.ch * 8192, 8192, &bar_g2); break;
+            default: break;
+        }
+    };
+
+    if (loader) {
+        if (lane == 0) {
+            uint32_t ph = 0;
+            bool lok = true, pend_k = false, pend1 = false, pend2 = false;
+#pragma unroll 1
+            for (int item = blockIdx.x; item < n_items && lok; item += gridDim.x, ph ^= 1) {
+                ChunkInfo x, nx;
+                chunk_info(p, x, item);
+                const bool has_next = item + (int)gridDim.x < n_items;
+                if (has_next) chunk_info(p, nx, item + gridDim.x);
+                const bool full = x.len == kC;
+                pend_k = pend1 = pend2 = false;
+                // the trip is under way (all its tiles have arrived): K of the next one, the only late load, -> L2
+                if (!(lok = mbar_wait(&bar_ld0, ph))) break;
+                if (has_next) {
+                    prefetch_l2_tma_2d(&P.tm_k, nx.hd * D, nx.tok0);
+                    prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + 64, nx.tok0);
+                }
+                // dq, dv are staged
+                if (!(lok = mbar_wait(&bar_st1, ph))) break;
+                if (full) {
+                    for (int cb = 0; cb < 2; ++cb) {
+                        tma_store_2d(&P.tm_dq, x.hd * D + cb * 64, x.tok0, sm + STG_A + cb * 8192);
+                        tma_store_2d(&P.tm_dv, x.hd * D + cb * 64, x.tok0, sm + STG_B + cb * 8192);
+                    }
+                    bulk_commit();
+                }
+                // phase 5 is done
+                if (!(lok = mbar_wait(&bar_ld1, ph))) break;
+                if (has_next) {
+                    mbar_expect_tx(&bar_g1, G1_BYTES);
+                    pend1 = true;
+#pragma unroll 1
+                    for (int piece = 2; piece <= 7; ++piece) load_piece(piece, nx);
+                }
+                // phase 6 is done; V goes where dv is staged, so that store must have read its source
+                if (!(lok = mbar_wait(&bar_ld2, ph))) break;
+                if (has_next) {
+                    bulk_wait_read<0>();
+                    mbar_expect_tx(&bar_g2, G2_BYTES);
+                    pend2 = true;
+#pragma unroll 1
+                    for (int piece = 8; piece <= 12; ++piece) load_piece(piece, nx);
+                }
+                // the last readout holds its K values in registers
+                if (!(lok = mbar_wait(&bar_kfree, ph))) break;
+                if (has_next) {
+                    mbar_expect_tx(&bar_k, K_BYTES);
+                    pend_k = true;
+                    load_piece(0, nx);
+                    load_piece(1, nx);
+                }
+                // dk is staged
+                if (!(lok = mbar_wait(&bar_st2, ph))) break;
+                if (full) {
+                    for (int cb = 0; cb < 2; ++cb) tma_store_2d(&P.tm_dk, x.hd * D + cb * 64, x.tok0, sm + STG_K + cb * 8192);
+                    bulk_commit();
+                }
+                bulk_wait_read<0>();
+                mbar_arrive(&bar_free);   // the staging regions may be rewritten
+            }
+            bulk_wait_read<0>();
+            if (!lok) {   // after a timeout a copy may still be in flight: wait for it before the CTA may retire
+                if (pend_k) (void)mbar_wait(&bar_k, ph ^ 1);
+                if (pend1) (void)mbar_wait(&bar_g1, ph ^ 1);
+                if (pend2) (void)mbar_wait(&bar_g2, ph ^ 1);
+            }
+        }
+        return;
+    }
+
+    auto cta_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory"); };   // all warps but the loader
     uint32_t mma_phase = 0, in_phase = 0;
+    // chunk table entry and gates of a trip are fetched one trip ahead into registers (their latency would be exposed)
+    ChunkInfo xn;
+    chunk_info(p, xn, blockIdx.x);
+    float ng = 0.f, ngend = 0.f, nb = 0.f;
+    auto fetch_gates = [&](const ChunkInfo& c) {   // cumulative log decay of this thread's token and of the chunk end, gate b
+        const float* gsrc = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)c.ch * kC;
+        ng = gsrc[threadIdx.x];
+        ngend = gsrc[kC - 1];
+        nb = ((int)threadIdx.x < c.len) ? p.beta[(size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd] : 0.f;
+    };
+    // first trip: every group is loaded at once, one instruction per warp
+    if (issuer) { mbar_expect_tx(&bar_k, K_BYTES); mbar_expect_tx(&bar_g1, G1_BYTES); mbar_expect_tx(&bar_g2, G2_BYTES); }
+    if (lane == 0 && warp < 13) load_piece(warp, xn);
+    if (threadIdx.x < kC) fetch_gates(xn);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-    ChunkInfo x;
-    chunk_info(p, x, item);
+    const ChunkInfo x = xn;
+    const float g_now = ng, gend_now = ngend, b_now = nb;
+    const bool has_next = item + (int)gridDim.x < n_items;
+    const bool first = item == (int)blockIdx.x;
+    if (has_next) chunk_info(p, xn, item + gridDim.x);
 #ifdef GDN_PHASE_TIMING
     if (blockIdx.x == 0 && threadIdx.x == 0) g_trip_now = (item - (int)blockIdx.x) / (int)gridDim.x;
 #endif
     GDN_TICK(2, 0);
+    GDN_TRIP(1, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
 
-    if (issuer) {
-        mbar_expect_tx(&bar_in0, 32768 + 16384 + 32768 + 32768);
-        mbar_expect_tx(&bar_in1, 16384 + 16384 + 16384 + 8192);
-    }
-    if (lane == 0 && worker) {   // one bulk / TMA load and one L2 prefetch per warp: their issue cost runs in parallel
-        const int cb = warp & 1, xq = x.hd * D + cb * 64;
-        switch (warp) {
-            case 0: case 1: tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_in0); break;
-            case 2: case 3: tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_in0); break;
-            case 4: bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in0); break;
-            case 5: bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in0); break;
-            case 6: bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)x.ch * 32768, 32768, &bar_in0); break;
-            case 8: case 9: tma_load_2d(sm + VT + cb * 8192, &P.tm_v, xq, x.tok0, &bar_in1); break;
-            case 10: case 11: tma_load_2d(sm + DO + cb * 8192, &P.tm_do, xq, x.tok0, &bar_in1); break;
-            case 12: bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in1); break;
-            case 13: bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)x.ch * 8192, 8192, &bar_in1); break;
-            default: break;
-        }
-        ChunkInfo nx;
-        if (item + (int)gridDim.x < n_items && chunk_info(p, nx, item + gridDim.x)) {   // next trip's tiles -> L2
-            const int xn = nx.hd * D + cb * 64;
-            switch (warp) {
-                case 0: case 1: prefetch_l2_tma_2d(&P.tm_q, xn, nx.tok0); break;
-                case 2: case 3: prefetch_l2_tma_2d(&P.tm_k, xn, nx.tok0); break;
-                case 4: prefetch_l2_bulk(p.ws + p.L.W + (size_t)nx.ch * 16384, 16384); break;
-                case 5: prefetch_l2_bulk(p.ws + p.L.hc + (size_t)nx.ch * 32768, 32768); break;
-                case 6: prefetch_l2_bulk(p.ws + p.L.dhn + (size_t)nx.ch * 32768, 32768); break;
-                case 8: case 9: prefetch_l2_tma_2d(&P.tm_v, xn, nx.tok0); break;
-                case 10: case 11: prefetch_l2_tma_2d(&P.tm_do, xn, nx.tok0); break;
-                case 12: prefetch_l2_bulk(p.ws + p.L.Ut + (size_t)nx.ch * 16384, 16384); break;
-                case 13: prefetch_l2_bulk(p.ws + p.L.Tm + (size_t)nx.ch * 8192, 8192); break;
-                default: break;
-            }
-        }
-    }
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
-        const float* gsrc = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC;
-        const float g = gsrc[i], gend = gsrc[kC - 1];
-        gl[i] = g * kLog2e;
-        Gam[i] = expf(g);
-        ee[i] = expf(gend - g);
-        bb[i] = (i < x.len) ? p.beta[(size_t)(x.tok0 + i) * H + x.hd] : 0.f;
+        gl[i] = g_now * kLog2e;
+        Gam[i] = expf(g_now);
+        ee[i] = expf(gend_now - g_now);
+        bb[i] = b_now;
     }
     if (ok) {
-        ok = mbar_wait(&bar_in0, in_phase) && mbar_wait(&bar_in1, in_phase);
+        ok = mbar_wait(&bar_g1, in_phase) && mbar_wait(&bar_k, in_phase);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
     }
     if (ok && x.len < kC) {
-        zero_tail_rows(sm + QK, 128, 0, x.len);
-        zero_tail_rows(sm + QK, 128, 64, x.len);
-        zero_tail_rows(sm + VT, 64, 0, x.len);
-        zero_tail_rows(sm + DO, 64, 0, x.len);
+        zero_tail_rows(sm + QK, 128, 0, x.len, kIntraThreads);
+        zero_tail_rows(sm + QK, 128, 64, x.len, kIntraThreads);
         fence_async_smem();
     }
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 1);
 
     // ---- phase 1
@@ -737,10 +833,12 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
         mma_tile<128, 64, 128>(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
         mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
     }
+    if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // every tile of this trip has arrived
     // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up)
+    if (has_next && threadIdx.x < kC) fetch_gates(xn);
     float hh = 0.f;
 #pragma unroll 1
-    for (int t = threadIdx.x; t < 2048; t += blockDim.x) {
+    for (int t = threadIdx.x; t < 2048; t += kIntraThreads) {
         float a[8], b[8];
         unpack8(*reinterpret_cast<const uint4*>(sm + HH + t * 16), a);
         unpack8(*reinterpret_cast<const uint4*>(sm + DH + t * 16), b);
@@ -768,9 +866,17 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
             }
         }
     }
+    if (ok) {
+        ok = mbar_wait(&bar_g2, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 27);
+    }
+    if (ok && x.len < kC) {
+        zero_tail_rows(sm + VT, 64, 0, x.len, kIntraThreads);
+        zero_tail_rows(sm + DO, 64, 0, x.len, kIntraThreads);
+    }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 4);
 
     // ---- phase 2
@@ -781,6 +887,10 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     }
     GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
+    if (ok && !first) {   // U^T and dU^T held the previous trip's staged dk and dq: their stores must have read them
+        ok = mbar_wait(&bar_free, in_phase ^ 1);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 28);
+    }
     const int f = q4 * 32 + lane;      // feature (lane of the transposed accumulators)
     const int i0 = grp * kTG;          // first of this thread's 32 tokens
     float rs = 0.f;
@@ -809,7 +919,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 6);
 
     // From here on the accumulators that become gradients are produced token-major (64 token rows x 128 features,
@@ -857,7 +967,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 8);
 
     // ---- phase 4
@@ -911,7 +1021,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 10);
 
     // ---- phase 5
@@ -920,18 +1030,15 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
-    } else if (ok && full && threadIdx.x == 32) {
-        // staged dq, dv leave through the async proxy (generic global stores would stall the next proxy fence); a
-        // thread of another warp issues them so that the MMA issue is not delayed
-        for (int cb = 0; cb < 2; ++cb) {
-            tma_store_2d(&P.tm_dq, x.hd * D + cb * 64, x.tok0, sm + STG_A + cb * 8192);
-            tma_store_2d(&P.tm_dv, x.hd * D + cb * 64, x.tok0, sm + STG_B + cb * 8192);
-        }
-        bulk_commit();
+        mma_commit(&bar_ld1);   // Q, U~^T, dh', h (by now dXk, dXv) have been read for the last time
+    } else if (threadIdx.x == 32) {
+        // staged dq, dv leave through the async proxy (generic global stores would stall the next proxy fence); the
+        // loader issues the stores
+        mbar_arrive(&bar_st1);
     }
     if (ok && !full) {   // ragged tail: rows beyond the sequence must not be written
-        flush_rows(sm + STG_A, gdq, rowp, x.len);
-        flush_rows(sm + STG_B, gdv, rowp, x.len);
+        flush_rows(sm + STG_A, gdq, rowp, x.len, kIntraThreads);
+        flush_rows(sm + STG_B, gdv, rowp, x.len, kIntraThreads);
     }
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
@@ -957,7 +1064,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 12);
 
     // ---- phase 6
@@ -968,11 +1075,21 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
         mma_tile<64, 128, 64>(tmem + 0, op_k_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), false);             // (bG) K
         mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);               // T^T dW again, group A
         mma_commit(&bar_mma);
+        mma_commit(&bar_ld2);   // dW^T (over dO) and T have been read for the last time
     }
     GDN_TICK(2, 13);
     GDN_WAIT_MMA(26)
-    if (ok && worker) {
+    GDN_TICK(2, 16);
+    if (worker) {   // this thread's K values leave shared memory now, so that the next trip's K can be loaded over them
+        uint4 kraw[4];
+#pragma unroll
+        for (int part = 0; part < 4; ++part)
+            kraw[part] = *reinterpret_cast<const uint4*>(sm + QK + tile_chunk_off(128, 64 + tr, (cb0 >> 3) + part));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_kfree);
+        GDN_TICK(2, 17);
         float acc = 0.f;   // group A: <k, dk^col> ; group B: db = <k, G K + Gam dXk>
+        if (ok) {
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
@@ -982,7 +1099,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
             tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: dk^col part   B: G K
             tmem_ld8(tmem + lane_base + 384 + cb, d8);    // A: U dh'^T
             tmem_wait_ld();
-            chunk_load(sm + QK, 128, 64 + tr, cb >> 3, kk);
+            unpack8(kraw[part], kk);
             if (ga) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -996,24 +1113,19 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
                 for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], a[j], c8[j]), acc);
             }
         }
+        }
         red[ga ? 3 : 2][grp][tr] = acc;
     }
+    GDN_TICK(2, 18);
     // block totals of sum_j r_j and <dh', h>
     rs = warp_sum(rs);
     hh = warp_sum(hh);
     if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(2, 14);
-    if (ok && full) {
-        if (threadIdx.x == 32) {
-            for (int cb = 0; cb < 2; ++cb) tma_store_2d(&P.tm_dk, x.hd * D + cb * 64, x.tok0, sm + STG_K + cb * 8192);
-            bulk_commit();
-            bulk_wait_read<0>();   // all staged gradients of this trip have left shared memory
-        }
-    } else if (ok) {
-        flush_rows(sm + STG_K, gdk, rowp, x.len);
-    }
+    if (threadIdx.x == 32) mbar_arrive(&bar_st2);   // dk is staged: the loader stores it
+    if (ok && !full) flush_rows(sm + STG_K, gdk, rowp, x.len, kIntraThreads);
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
         auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
@@ -1021,17 +1133,18 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_intra_kernel(const __grid
         if (i < x.len) p.dbeta[(size_t)(x.tok0 + i) * H + x.hd] = db + dw;
         dgam[i] = fmaf(bb[i], db, qdq - kcol);
     }
-    __syncthreads();
+    cta_sync();
     if (warp == 0 && ok) {
         float rsum = 0.f, hsum = 0.f;
         for (int w = 0; w < kIntraThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
         write_dg_suffix(dgam, nullptr, rsum + Gam[kC - 1] * hsum, p.dg + (size_t)x.tok0 * H + x.hd, (size_t)H, x.len, lane);
     }
     tc_fence_before();
-    __syncthreads();   // every reader of this trip's tiles and scratch is done
+    cta_sync();   // every reader of this trip's tiles and scratch is done
     GDN_TICK(2, 15);
     if (!ok) break;
     }
+    GDN_TRIP(1, 20);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -1214,7 +1327,7 @@ static int sm_count() {
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
-    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kIntraThreads, P, st);
+    return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kIntraThreads + 32, P, st);
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static bool done = false;
@@ -1259,6 +1372,9 @@ cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st
 #ifdef GDN_PHASE_TIMING
 extern "C" int gdn_debug_tick_trip(int trip) {
     return (int)cudaMemcpyToSymbol(gdn::g_tick_trip, &trip, sizeof(int));
+}
+extern "C" int gdn_debug_trips(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, gdn::g_trip_ns, sizeof(long long) * 2 * 24);
 }
 extern "C" int gdn_debug_ticks(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks, sizeof(long long) * 4 * 32);

@@ -49,12 +49,15 @@ __device__ __forceinline__ void tile_put(unsigned char* tile, int R, int r, int 
     *reinterpret_cast<__nv_bfloat16*>(tile + tile_off(R, r, c)) = __float2bfloat16_rn(x);
 }
 
-// Zero rows [row0 + len, row0 + 64) of a tile with R rows and 128 columns.
-__device__ __forceinline__ void zero_tail_rows(unsigned char* tile, int R, int row0, int len) {
-    for (int t = threadIdx.x; t < (kC - len) * 16; t += blockDim.x) {
+// Zero rows [row0 + len, row0 + 64) of a tile with R rows and 128 columns (threads 0 .. nthr-1 of the CTA take part).
+__device__ __forceinline__ void zero_tail_rows(unsigned char* tile, int R, int row0, int len, int nthr) {
+    for (int t = threadIdx.x; t < (kC - len) * 16; t += nthr) {
         const int r = row0 + len + t / 16, ch = t % 16;
         *reinterpret_cast<uint4*>(tile + tile_chunk_off(R, r, ch)) = make_uint4(0, 0, 0, 0);
     }
+}
+__device__ __forceinline__ void zero_tail_rows(unsigned char* tile, int R, int row0, int len) {
+    zero_tail_rows(tile, R, row0, len, (int)blockDim.x);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -90,11 +93,14 @@ __device__ __forceinline__ float reduce8(float (&v)[8], int lane) {
 }
 
 // Copy a staged [64 tokens][128 features] bf16 tile to a [T, H, 128] tensor with 16-byte stores (rows < len only).
-__device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloat16* gbase, size_t row_pitch, int len) {
-    for (int t = threadIdx.x; t < kC * 16; t += blockDim.x) {
+__device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloat16* gbase, size_t row_pitch, int len, int nthr) {
+    for (int t = threadIdx.x; t < kC * 16; t += nthr) {
         const int i = t >> 4, chk = t & 15;
         if (i < len) *reinterpret_cast<uint4*>(gbase + (size_t)i * row_pitch + chk * 8) = *reinterpret_cast<const uint4*>(tile + tile_chunk_off(64, i, chk));
     }
+}
+__device__ __forceinline__ void flush_rows(const unsigned char* tile, __nv_bfloat16* gbase, size_t row_pitch, int len) {
+    flush_rows(tile, gbase, row_pitch, len, (int)blockDim.x);
 }
 
 // dg_j = sum_{i >= j} dgam_i inside a chunk (gam_i = sum_{j <= i} g_j), by one warp: lane l owns tokens l and l + 32.

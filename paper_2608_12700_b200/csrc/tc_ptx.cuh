@@ -56,10 +56,13 @@ __device__ __forceinline__ uint64_t global_ns() {
 // Bounded wait: gives up after about two seconds and returns false; the caller records the failure and
 // leaves through its normal teardown (no trap, no endless spin).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    // (rolled loops: a kernel has dozens of waits, and unrolled polling would multiply its code size)
+#pragma unroll 1
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (;;) {
+#pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (global_ns() - t0 > 2000000000ull) return false;
