@@ -89,26 +89,28 @@ __device__ __forceinline__ void inv_level(const float* At, float* Tf) {
         }
         *reinterpret_cast<float4*>(Tf + (rb + ii) * kLdi + cb + j4) = make_float4(-s.x, -s.y, -s.z, -s.w);
     }
-    __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------------------
 // tc_prep
 // ------------------------------------------------------------------------------------------------
 namespace prep {
-constexpr uint32_t QK = 0;                    // [Q rows 0..63 ; K rows 64..127] x 128   32 KB (later: Nm image)
-constexpr uint32_t VO = 32768;                // [V ; dO] x 128                           32 KB (later: Bf image)
-constexpr uint32_t TT = 65536;                // T                      [64][64]           8 KB
-constexpr uint32_t TP = TT + 8192;            // T Diag(b Gam)
+// The input tiles are never reused within a trip, so the next trip's inputs are loaded into them as soon as the last
+// product that reads them is done; the three output images are staged over tiles that are dead by then.
+constexpr uint32_t QK = 0;                    // [Q rows 0..63 ; K rows 64..127] x 128   32 KB
+constexpr uint32_t VO = 32768;                // [V ; dO] x 128                           32 KB
+constexpr uint32_t TT = 65536;                // T                      [64][64]           8 KB  (these four: finally
+constexpr uint32_t TP = TT + 8192;            // T Diag(b Gam)                                    the Nm image)
 constexpr uint32_t TPP = TP + 8192;           // T Diag(w)
 constexpr uint32_t PT = TPP + 8192;           // P = tril(Q K^T . D)
 constexpr uint32_t WT = PT + 8192;            // W^T   [128 dk][64 tokens]                16 KB (before: fp32 scratch S)
-constexpr uint32_t WET = WT + 16384;          // (Diag(e) W)^T
-constexpr uint32_t UTT = WET + 16384;         // U~^T  [128 dv][64]
-constexpr uint32_t UET = UTT + 16384;         // (Diag(e) U~)^T
+constexpr uint32_t UTT = WT + 16384;          // U~^T  [128 dv][64]
+constexpr uint32_t WET = UTT + 16384;         // (Diag(e) W)^T                                    (these two: finally
+constexpr uint32_t UET = WET + 16384;         // (Diag(e) U~)^T                                   the Bf image)
 constexpr uint32_t X = UET + 16384;           // fp32 A and T during the inversion; then R = Diag(Gam) dO and
 constexpr uint32_t XA = X, XT = X + 17408;    // (P^T dO)^T; finally the E image
 constexpr uint32_t XR = X, XPDO = X + 16384;
+constexpr uint32_t NMS = TT, BFS = WET, ES = X;   // staging of the three output images
 constexpr uint32_t TILES_END = X + 34816;
 constexpr uint32_t SMEM_BYTES = TILES_END + 1024 /* alignment slack */;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -116,12 +118,12 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF = 384, C_E = 0;
 }  // namespace prep
 
-__global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
     GDN_TRIP(0, 0);
     using namespace prep;
     const Problem& p = P.p;
-    // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ... and pulls the inputs of its
-    // next one into L2 while it works on the current one.
+    // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...; the inputs of its next one
+    // are loaded while it works on the current one.
     const int H = p.d.H;
     const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
     if ((int)blockIdx.x >= n_items) return;
@@ -130,16 +132,22 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
     __shared__ __align__(16) float gam[kC], gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC], bgam[kC];
-    __shared__ uint64_t bar_qk, bar_vo, bar_mma;
+    __shared__ uint64_t bar_qk, bar_vo, bar_ld0, bar_t, bar_vofree, bar_ld1, bar_st, bar_tfree, bar_free1, bar_free, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     const bool worker = warp < 16;                       // warps 0..15 read accumulators and do the fp32 work
     const bool issuer = threadIdx.x == kWideThreads;     // first lane of warp 16 feeds the tensor pipe
+    // Warp 17 only moves data: its first lane issues the bulk stores of a trip's results and the loads of the next
+    // trip's inputs (each such instruction costs its issuer hundreds of cycles).  It follows the other warps through
+    // mbarriers and shares no block-wide barrier with them inside the loop (they use a named barrier).
+    const bool loader = warp == 17;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar_qk, 1); mbar_init(&bar_vo, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_qk, 1); mbar_init(&bar_vo, 1); mbar_init(&bar_ld0, 1); mbar_init(&bar_t, 1);
+        mbar_init(&bar_vofree, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_st, 1); mbar_init(&bar_tfree, 1);
+        mbar_init(&bar_free1, 1); mbar_init(&bar_free, 1); mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
@@ -148,6 +156,85 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
     bool ok = true;
+    const uint32_t VO_BYTES = bwd ? 32768 : 16384;
+    auto load_piece = [&](int piece, const ChunkInfo& c) {   // 0,1: Q  2,3: K  4,5: V  6,7: dO   (column halves)
+        const int cb = piece & 1, xq = c.hd * D + cb * 64;
+        switch (piece >> 1) {
+            case 0: tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, c.tok0, &bar_qk); break;
+            case 1: tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, c.tok0, &bar_qk); break;
+            case 2: tma_load_2d(sm + VO + cb * 16384, &P.tm_v, xq, c.tok0, &bar_vo); break;
+            case 3: if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, xq, c.tok0, &bar_vo); break;
+            default: break;
+        }
+    };
+
+    if (loader) {
+        if (lane == 0) {
+            uint32_t ph = 0;
+            bool lok = true, pend_qk = false, pend_vo = false;
+#pragma unroll 1
+            for (int item = blockIdx.x; item < n_items && lok; item += gridDim.x, ph ^= 1) {
+                ChunkInfo x, nx;
+                chunk_info(p, x, item);
+                const bool has_next = item + (int)gridDim.x < n_items;
+                if (has_next) chunk_info(p, nx, item + gridDim.x);
+                pend_qk = pend_vo = false;
+                // the trip is under way: Q, K of the next one (loaded late in this trip) -> L2
+                if (!(lok = mbar_wait(&bar_ld0, ph))) break;
+                if (has_next) {
+                    for (int cb = 0; cb < 2; ++cb) {
+                        prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
+                        prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
+                    }
+                }
+                // T is staged
+                if (!(lok = mbar_wait(&bar_t, ph))) break;
+                bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
+                bulk_commit();
+                // W^T, U~^T are staged and V, dO have been read for the last time
+                if (!(lok = mbar_wait(&bar_vofree, ph))) break;
+                bulk_wait_read<0>();
+                mbar_arrive(&bar_tfree);   // the T tile may be overwritten (by the staged Nm image)
+                bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
+                bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
+                bulk_commit();
+                if (has_next) {
+                    mbar_expect_tx(&bar_vo, VO_BYTES);
+                    pend_vo = true;
+#pragma unroll 1
+                    for (int piece = 4; piece < 8; ++piece) load_piece(piece, nx);
+                }
+                // phase 3 is done: Q, K have been read for the last time
+                if (!(lok = mbar_wait(&bar_ld1, ph))) break;
+                if (has_next) {
+                    mbar_expect_tx(&bar_qk, 32768);
+                    pend_qk = true;
+#pragma unroll 1
+                    for (int piece = 0; piece < 4; ++piece) load_piece(piece, nx);
+                }
+                // the three images are staged.  A store drains shared memory at some 32 bytes per cycle, so they leave in
+                // the order in which the next trip rewrites their tiles: E (fp32 scratch) and Nm (P) first, Bf last
+                if (!(lok = mbar_wait(&bar_st, ph))) break;
+                if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + ES, 32768);
+                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + NMS, 32768);
+                bulk_commit();
+                bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + BFS, 32768);
+                bulk_commit();
+                bulk_wait_read<1>();
+                mbar_arrive(&bar_free1);   // the E and Nm staging tiles may be rewritten
+                bulk_wait_read<0>();
+                mbar_arrive(&bar_free);    // every staging tile may be rewritten
+            }
+            bulk_wait_read<0>();
+            if (!lok) {   // after a timeout a copy may still be in flight: wait for it before the CTA may retire
+                if (pend_qk) (void)mbar_wait(&bar_qk, ph ^ 1);
+                if (pend_vo) (void)mbar_wait(&bar_vo, ph ^ 1);
+            }
+        }
+        return;
+    }
+
+    auto cta_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory"); };   // all warps but the loader
     uint32_t mma_phase = 0, in_phase = 0;
     // The chunk table entry and the gate values of a trip are fetched one trip ahead into registers: they are tiny, but
     // read at the top of a trip their DRAM latency would be fully exposed.
@@ -163,32 +250,25 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         }
     };
     fetch_gates(xn);
+    // first trip: the inputs are loaded at once, one instruction per warp
+    if (issuer) { mbar_expect_tx(&bar_qk, 32768); mbar_expect_tx(&bar_vo, VO_BYTES); }
+    if (lane == 0 && warp < 8) load_piece(warp, xn);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
     const ChunkInfo x = xn;
     const float g_now = ng, b_now = nb;
     const bool has_next = item + (int)gridDim.x < n_items;
+    const bool first = item == (int)blockIdx.x;
     if (has_next) chunk_info(p, xn, item + gridDim.x);
     GDN_TICK(0, 0);
     GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
 
-    if (issuer) {
-        mbar_expect_tx(&bar_qk, 32768);
-        mbar_expect_tx(&bar_vo, bwd ? 32768 : 16384);
-    }
-    if (lane == 0 && warp < 8) {   // one TMA load and one L2 prefetch per warp: their issue cost runs in parallel
-        const int cb = warp & 1, which = warp >> 1, xq = x.hd * D + cb * 64;
-        if (which == 0) tma_load_2d(sm + QK + cb * 16384, &P.tm_q, xq, x.tok0, &bar_qk);
-        else if (which == 1) tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, xq, x.tok0, &bar_qk);
-        else if (which == 2) tma_load_2d(sm + VO + cb * 16384, &P.tm_v, xq, x.tok0, &bar_vo);
-        else if (bwd) tma_load_2d(sm + VO + cb * 16384 + 8192, &P.tm_do, xq, x.tok0, &bar_vo);
-    }
     // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
         gam[i] = g_now; bb[i] = b_now; ww[i] = b_now;
     }
-    __syncthreads();
+    cta_sync();
     if (warp == 0) {   // inclusive prefix sum of the 64 log decays: lane l owns tokens l and l + 32
         float a = gam[lane], b = gam[lane + 32];
 #pragma unroll
@@ -200,7 +280,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         gam[lane] = a;
         gam[lane + 32] = b;
     }
-    __syncthreads();
+    cta_sync();
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
         gl[i] = gam[i] * kLog2e;
@@ -214,13 +294,13 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
     }
     if (ok && x.len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
-        zero_tail_rows(sm + QK, 128, 0, x.len);
-        zero_tail_rows(sm + QK, 128, 64, x.len);
-        zero_tail_rows(sm + VO, 128, 0, x.len);
-        if (bwd) zero_tail_rows(sm + VO, 128, 64, x.len);
+        zero_tail_rows(sm + QK, 128, 0, x.len, kIntraThreads);
+        zero_tail_rows(sm + QK, 128, 64, x.len, kIntraThreads);
+        zero_tail_rows(sm + VO, 128, 0, x.len, kIntraThreads);
+        if (bwd) zero_tail_rows(sm + VO, 128, 64, x.len, kIntraThreads);
         fence_async_smem();
     }
-    __syncthreads();
+    cta_sync();
     GDN_TICK(0, 1);
 
     // ---- phase 1: S1 = [Q; K] K^T  (rows 0..63: Q K^T, rows 64..127: K K^T)
@@ -229,21 +309,16 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
         mma_commit(&bar_mma);
     }
+    if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // this trip's inputs have arrived
     float* Af = reinterpret_cast<float*>(sm + XA);   // [64][kLdi]  strictly lower part of I + A
     float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][kLdi]  T
     float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
-    for (int t = threadIdx.x; t < kC * kLdi; t += blockDim.x) Tf[t] = 0.f;
-    if (has_next) {   // while the product runs: next trip's gates -> registers, its input tiles -> L2
-        if (threadIdx.x < kC) fetch_gates(xn);
-        if (lane == 0 && warp >= 8 && warp < 16) {
-            const int cb = warp & 1, which = (warp >> 1) & 3, xq = xn.hd * D + cb * 64;
-            if (which == 0) prefetch_l2_tma_2d(&P.tm_q, xq, xn.tok0);
-            else if (which == 1) prefetch_l2_tma_2d(&P.tm_k, xq, xn.tok0);
-            else if (which == 2) prefetch_l2_tma_2d(&P.tm_v, xq, xn.tok0);
-            else if (bwd) prefetch_l2_tma_2d(&P.tm_do, xq, xn.tok0);
-        }
-    }
+    if (has_next && threadIdx.x < kC) fetch_gates(xn);   // next trip's gates -> registers while the product runs
     GDN_WAIT_MMA(2)
+    if (ok && !first) {   // the previous trip's E and Nm stores have read their tiles (the fp32 scratch and P are next)
+        ok = mbar_wait(&bar_free1, in_phase ^ 1);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 6);
+    }
     GDN_TICK(0, 2);
     if (ok && worker) {
         const int i = (q4 & 1) * 32 + lane, j0 = grp * kTG;
@@ -268,7 +343,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         }
     }
     tc_fence_before();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(0, 3);
     // ---- T = (I + A)^-1 by blocks of 16: diagonal blocks by forward substitution, then block row r of block
     // column c from  T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc),  one block diagonal at a time.  All fp32.
@@ -284,21 +359,33 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
             Tf[(b0 + i) * kLdi + b0 + j] = s;
         }
     }
-    __syncthreads();
+    cta_sync();
     GDN_TICK(0, 16);
+    if (ok && !first) {   // every store of the previous trip has read its tile (the scratch S lies over W^T)
+        ok = mbar_wait(&bar_free, in_phase ^ 1);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 5);
+    }
     inv_premul(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
-    __syncthreads();
+    cta_sync();
     inv_level<1>(Sf, Tf);
+    cta_sync();
     GDN_TICK(0, 17);
     inv_level<2>(Sf, Tf);
+    cta_sync();
     GDN_TICK(0, 18);
     inv_level<3>(Sf, Tf);
+    cta_sync();
     GDN_TICK(0, 4);
-    for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
+    for (int t = threadIdx.x; t < kC * 8; t += kIntraThreads) {
         const int i = t >> 3, cch = t & 7;
         float a[8], b[8], w8[8];
-        *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8);
-        *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8 + 4);
+        if ((cch >> 1) <= (i >> 4)) {   // the blocks above the block diagonal are zero and were never written
+            *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8);
+            *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8 + 4);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) a[k] = 0.f;
+        }
         *reinterpret_cast<float4*>(b) = *reinterpret_cast<const float4*>(bgam + cch * 8);
         *reinterpret_cast<float4*>(b + 4) = *reinterpret_cast<const float4*>(bgam + cch * 8 + 4);
         *reinterpret_cast<float4*>(w8) = *reinterpret_cast<const float4*>(ww + cch * 8);
@@ -310,7 +397,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         chunk_store(sm + TPP, 64, i, cch, w8);
     }
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(0, 5);
 
     // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T ; (P^T dO)^T = dO^T P
@@ -321,13 +408,10 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         if (bwd) mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
     }
-    if (ok && threadIdx.x == 0) {
-        bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
-        bulk_commit();
-    }
+    if (threadIdx.x == 32) mbar_arrive(&bar_t);   // the loader stores the T tile
     // R = Diag(Gam) dO (token-major tile), while the MMAs run.  The fp32 A / T scratch is dead by now.
     if (bwd) {
-        for (int t = threadIdx.x; t < kC * 16; t += blockDim.x) {
+        for (int t = threadIdx.x; t < kC * 16; t += kIntraThreads) {
             const int i = t >> 4, cch = t & 15;
             float v[8];
             chunk_load(sm + VO, 128, 64 + i, cch, v);
@@ -366,7 +450,7 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
+    cta_sync();
     GDN_TICK(0, 6);
 
     // ---- phase 3: Nm = K^T (Diag(e) W) ; Bf = K^T (Diag(e) U~) ; E = Q^T R - W^T (P^T dO)
@@ -377,15 +461,15 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
-    }
-    if (ok && threadIdx.x == 0) {
-        bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
-        bulk_commit();
-    } else if (ok && threadIdx.x == 96) {
-        bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
-        bulk_commit();
+        mma_commit(&bar_ld1);   // Q, K have been read for the last time
+    } else if (threadIdx.x == 32) {
+        mbar_arrive(&bar_vofree);   // W^T, U~^T are staged; V, dO were last read by phase 2 and the pass that formed R
     }
     GDN_WAIT_MMA(4)
+    if (ok) {   // the T tile, part of the Nm staging area, has left through its store
+        ok = mbar_wait(&bar_tfree, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 7);
+    }
     GDN_TICK(0, 7);
     if (ok && worker) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
         const int r = q4 * 32 + lane, c0 = grp * (D / kGroups);
@@ -396,38 +480,23 @@ __global__ void __launch_bounds__(kIntraThreads, 1) tc_prep_kernel(const __grid_
             float v[8];
             tmem_ld8(tmem + lane_base + C_NM + cb, v);
             tmem_wait_ld();
-            chunk_store(sm + QK, 128, r, cb >> 3, v);
+            chunk_store(sm + NMS, 128, r, cb >> 3, v);
             tmem_ld8(tmem + lane_base + C_BF + cb, v);
             tmem_wait_ld();
-            chunk_store(sm + VO, 128, r, cb >> 3, v);
+            chunk_store(sm + BFS, 128, r, cb >> 3, v);
             if (bwd) {
                 tmem_ld8(tmem + lane_base + C_E + cb, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 8; ++k) v[k] *= sc;
-                chunk_store(sm + X, 128, r, cb >> 3, v);
+                chunk_store(sm + ES, 128, r, cb >> 3, v);
             }
         }
     }
     tc_fence_before();
     fence_async_smem();
-    __syncthreads();
-    // one bulk store per image, issued by threads of three different warps (bulk copies are slow to issue); each waits
-    // until its store has read shared memory, which the next trip overwrites
-    if (threadIdx.x == 0) {
-        if (ok) { bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + QK, 32768); bulk_commit(); }
-        bulk_wait_read<0>();   // also covers the T, W^T and U~^T stores issued earlier by this thread
-    } else if (threadIdx.x == 32) {
-        if (ok) { bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + VO, 32768); bulk_commit(); }
-        bulk_wait_read<0>();
-    } else if (threadIdx.x == 64 && bwd) {
-        if (ok) { bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + X, 32768); bulk_commit(); }
-        bulk_wait_read<0>();
-    } else if (threadIdx.x == 96) {
-        bulk_wait_read<0>();   // the U~^T store issued earlier by this thread
-    }
-    tc_fence_before();
-    __syncthreads();          // the next trip overwrites the tiles
+    cta_sync();
+    if (threadIdx.x == 32) mbar_arrive(&bar_st);   // the three images are staged: the loader stores them
     GDN_TICK(0, 8);
     if (!ok) break;
     }
@@ -1305,7 +1374,7 @@ static int sm_count();
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
-    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kIntraThreads, P, st);
+    return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kIntraThreads + 32, P, st);
 }
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static bool done = false;
