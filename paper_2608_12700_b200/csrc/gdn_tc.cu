@@ -953,6 +953,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         tc_fence_after();
         mma_tile<128, 64, 64>(tmem + slot(3), op_mn_major(sm + DO, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
+        // dO h^T (token-major, group A of columns 384..511) is first read after phase 4: it runs under the readout
+        mma_tile<64, 128, 128>(tmem + 384, op_k_major(sm + DO, 64), op_k_major(sm + HH, 128), false);
     }
     GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
@@ -996,10 +998,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // accumulator occupies lanes 0..15 of each quadrant ("group A"); a second one sits in lanes 16..31 of the same
     // columns ("group B", address + 16 lanes), and one tcgen05.ld serves both groups.
     //   columns   group A                               group B
-    //   0..127    dO h^T (ph 3) -> (bG) K (ph 6)        dP (ph 3, 64 cols) -> dXk (ph 4)
+    //   0..127    U dh'^T (ph 4)                        dP (ph 3, 64 cols) -> dXk (ph 4)
     //   128..255  (dP.D) K (ph 4) -> dXk again (ph 6)   dXv (ph 4)
     //   256..383  dW^T (ph 3, all lanes) -> dk^col      G K (ph 6)
-    //   384..511  U dh'^T (ph 4)                        dA (ph 5, 64 cols)
+    //   384..511  dO h^T (ph 2) -> (bG) K (ph 6)        dA (ph 5, 64 cols)
     constexpr uint32_t LB = 16u << 16;
     const bool ga = lane < 16;
     const int tr = q4 * 16 + (lane & 15);   // token row of this lane in token-major accumulators
@@ -1010,9 +1012,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + 0 + LB, op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);           // dO U^T
-        mma_tile<64, 128, 128>(tmem + 0, op_k_major(sm + DO, 64), op_k_major(sm + HH, 128), false);                 // dO h^T
         mma_tile<128, 64, 128>(tmem + 256, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
-        mma_commit(&bar_mma);   // (no early commit here: the readout overwrites the dO tile, which dO h^T reads)
+        mma_commit(&bar_mma);   // (also covers dO h^T of phase 2: the readout overwrites the dO tile, which it reads)
     }
     GDN_TICK(2, 7);
     GDN_WAIT_MMA(23)
@@ -1047,7 +1048,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_tile<64, 128, 64>(tmem + 128 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DUT, 128), false);          // T^T dU
         mma_commit(&bar_mma);   // the two dk^col products are first read after phase 6
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
-        mma_tile<64, 128, 128>(tmem + 384, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);              // U dh'^T
+        mma_tile<64, 128, 128>(tmem + 0, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);                // U dh'^T
     }
     GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
@@ -1062,8 +1063,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
-            float a[8], b[8], t8[8];
-            tmem_ld8(tmem + lane_base + 0 + cb, a);       // A: dO h^T      B: dXk
+            float a[8], b[8], t8[8], xk[8];
+            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: dO h^T
+            tmem_ld8(tmem + lane_base + 0 + cb, xk);      //                B: dXk
             tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: (dP.D) K    B: dXv
             tmem_wait_ld();
             if (ga) {
@@ -1075,7 +1077,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 }
                 chunk_store(sm + STG_A, 64, tr, cb >> 3, a);
             } else {
-                chunk_store(sm + DXK, 64, tr, cb >> 3, a);
+                chunk_store(sm + DXK, 64, tr, cb >> 3, xk);
                 chunk_store(sm + DXV, 64, tr, cb >> 3, b);
                 chunk_load(sm + VT, 64, tr, cb >> 3, t8);
 #pragma unroll
@@ -1141,7 +1143,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         tc_fence_after();
         mma_tile<64, 128, 64>(tmem + 256 + LB, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);       // G K
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), true);           // += (bG)^T K
-        mma_tile<64, 128, 64>(tmem + 0, op_k_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), false);             // (bG) K
+        mma_tile<64, 128, 64>(tmem + 384, op_k_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), false);           // (bG) K
         mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);               // T^T dW again, group A
         mma_commit(&bar_mma);
         mma_commit(&bar_ld2);   // dW^T (over dO) and T have been read for the last time
@@ -1163,10 +1165,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
             float a[8], b[8], c8[8], d8[8], kk[8];
-            tmem_ld8(tmem + lane_base + 0 + cb, a);       // A: (bG) K        B: dXk
+            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: (bG) K
             tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: dXk
             tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: dk^col part   B: G K
-            tmem_ld8(tmem + lane_base + 384 + cb, d8);    // A: U dh'^T
+            tmem_ld8(tmem + lane_base + 0 + cb, d8);      // A: U dh'^T       B: dXk
             tmem_wait_ld();
             unpack8(kraw[part], kk);
             if (ga) {
@@ -1179,7 +1181,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 chunk_store(sm + STG_K, 64, tr, cb >> 3, a);
             } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], a[j], c8[j]), acc);
+                for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], d8[j], c8[j]), acc);
             }
         }
         }
