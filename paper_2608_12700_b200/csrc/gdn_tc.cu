@@ -513,25 +513,34 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 // ring of bulk copies; the chunk decays exp(gamma_e) are fetched once per chain.
 // ------------------------------------------------------------------------------------------------
 namespace scan {
-constexpr int STAGES = 2;
-constexpr int PREFETCH_AHEAD = 3;                // steps by which L2 prefetches run ahead of the ring loads
 constexpr int GE_CAP = 2048;                     // chunk decays cached per chain (longer chains read them from global)
-constexpr uint32_t NM = 0;                       // ring: Nm tile image (32 KB) + additive-term image (32 KB) per stage
-constexpr uint32_t ADD = 32768;
-constexpr uint32_t STAGE_BYTES = 65536;
-constexpr uint32_t HT = STAGES * STAGE_BYTES;    // two state tiles [128][128], 32 KB each (one feeds the MMA and the
-                                                 // bulk store of this step while the next step's is being written)
-constexpr uint32_t SMEM_BYTES = HT + 2 * 32768 + 1024;
-static_assert(SMEM_BYTES + GE_CAP * 4 <= 227 * 1024, "shared memory budget");
+constexpr uint32_t NM = 0, ADD = 32768;          // ring stage: Nm tile image (32 KB) + the CTA's columns of the additive image
+// S = number of CTAs that share a chain, each carrying 128 / S state columns (the columns of the state evolve
+// independently).  S = 2 is used when there are too few chains to fill the machine.
+template <int S> struct Cfg {
+    static constexpr int NS = D / S;                         // state columns of this CTA
+    static constexpr int STAGES = S == 1 ? 2 : 3;
+    static constexpr int PREFETCH_AHEAD = STAGES + 1;        // steps by which L2 prefetches run ahead of the ring loads
+    static constexpr uint32_t ADD_BYTES = 32768 / S, STAGE_BYTES = 32768 + ADD_BYTES;
+    static constexpr uint32_t HT = STAGES * STAGE_BYTES;     // two state tiles [128][NS] (one feeds the MMA and the bulk
+    static constexpr uint32_t HT_BYTES = 32768 / S;          // store of this step while the next step's is being written)
+    static constexpr uint32_t SMEM_BYTES = HT + 2 * HT_BYTES + 1024;
+    static_assert(SMEM_BYTES + GE_CAP * 4 <= 227 * 1024, "shared memory budget");
+};
 }  // namespace scan
 
+template <int S>
 __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_constant__ TcParams P) {
     using namespace scan;
+    using C = Cfg<S>;
+    constexpr int NS = C::NS, NSH = NS / 2, STAGES = C::STAGES, PREFETCH_AHEAD = C::PREFETCH_AHEAD;
+    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES, ADD_BYTES = C::ADD_BYTES, HT = C::HT, HT_BYTES = C::HT_BYTES;
+    const int part = (int)blockIdx.x % S, bid = (int)blockIdx.x / S;   // column block of the state, (chain, direction)
     const Problem& p = P.p;
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
     if (hdr->status != GDN_OK) return;
-    const int reverse = P.scan_dirs == 2 ? (blockIdx.x & 1) : P.scan_dirs;
-    const int chain = P.scan_dirs == 2 ? (blockIdx.x >> 1) : blockIdx.x;
+    const int reverse = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
+    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
     const int n = chain / p.d.H, hd = chain % p.d.H;
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
     const int c0 = seq_first[n], c1 = seq_first[n + 1], nsteps = c1 - c0;
@@ -544,7 +553,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, hf = warp >> 2;
     const int r = q4 * 32 + lane;              // state row owned by this thread
-    const int gc0 = hf * 64;                   // first of its 64 columns
+    const int lc0 = hf * NSH;                  // first of its NSH columns inside the CTA's block
+    const int gc0 = part * NS + lc0;           // ... and inside the state
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
@@ -552,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
         mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 128); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, NS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -560,39 +570,39 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 
     auto chunk_of = [&](int s) { return reverse ? (c1 - 1 - s) : (c0 + s); };
     const char* nm_base = p.ws + p.L.Nm;
-    const char* add_base = p.ws + (reverse ? p.L.E : p.L.Bf);
-    char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
+    const char* add_base = p.ws + (reverse ? p.L.E : p.L.Bf) + part * ADD_BYTES;
+    char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc) + part * HT_BYTES;
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
     auto fill = [&](int s) {   // thread 0: bring chunk step s into ring slot s % STAGES
         const int stage = s % STAGES;
         const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
-        mbar_expect_tx(&bar_full[stage], 65536);
+        mbar_expect_tx(&bar_full[stage], STAGE_BYTES);
         bulk_load(sm + stage * STAGE_BYTES + NM, nm_base + ch * 32768, 32768, &bar_full[stage]);
-        bulk_load(sm + stage * STAGE_BYTES + ADD, add_base + ch * 32768, 32768, &bar_full[stage]);
+        bulk_load(sm + stage * STAGE_BYTES + ADD, add_base + ch * 32768, ADD_BYTES, &bar_full[stage]);
         // The ring gives a load one step of lead, less than an HBM round trip; pull the step after next into L2 now.
         if (s + PREFETCH_AHEAD < nsteps) {
             const size_t chn = (size_t)chunk_of(s + PREFETCH_AHEAD) * p.d.H + hd;
             prefetch_l2_bulk(nm_base + chn * 32768, 32768);
-            prefetch_l2_bulk(add_base + chn * 32768, 32768);
+            prefetch_l2_bulk(add_base + chn * 32768, ADD_BYTES);
         }
     };
     if (threadIdx.x == 32) {
         for (int s = STAGES; s < STAGES + PREFETCH_AHEAD && s < nsteps; ++s) {
             const size_t chn = (size_t)chunk_of(s) * p.d.H + hd;
             prefetch_l2_bulk(nm_base + chn * 32768, 32768);
-            prefetch_l2_bulk(add_base + chn * 32768, 32768);
+            prefetch_l2_bulk(add_base + chn * 32768, ADD_BYTES);
         }
         for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
     }
     for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
         ge[s] = expf(gamma[((size_t)chunk_of(s) * p.d.H + hd) * kC + kC - 1]);
     // initial state
-    float st[64];
+    float st[NSH];
     {
         const float* init = reverse ? p.dhT : p.h0;
         const size_t soff = ((size_t)n * p.d.H + hd) * D * D + (size_t)r * D + gc0;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
+        for (int k = 0; k < NSH / 4; ++k) {
             float4 v = init ? *reinterpret_cast<const float4*>(init + soff + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
             st[4 * k] = v.x; st[4 * k + 1] = v.y; st[4 * k + 2] = v.z; st[4 * k + 3] = v.w;
         }
@@ -602,7 +612,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     uint32_t mma_phase = 0;
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
-        unsigned char* Ht = sm + HT + (s & 1) * 32768;
+        unsigned char* Ht = sm + HT + (s & 1) * HT_BYTES;
         const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
         const int stage = s % STAGES;
         const unsigned char* ring = sm + stage * STAGE_BYTES;
@@ -610,7 +620,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
         const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
         // state -> bf16: operand tile of the MMA; the same bytes are the per-chunk state the gradient stage reads
 #pragma unroll
-        for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, hf * 8 + k)) = pack8(st + 8 * k);
+        for (int k = 0; k < NSH / 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
         fence_async_smem();
         __syncthreads();
         if (s < 4) GDN_TICK(1, s * 5 + 1);
@@ -619,14 +629,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
             if (ok) {
                 tc_fence_after();
                 const Operand a = reverse ? op_mn_major(ring + NM, 128) : op_k_major(ring + NM, 128);
-                mma_tile<128, 128, 128>(tmem, a, op_mn_major(Ht, 128), false);
+                mma_tile<128, NS, 128>(tmem, a, op_mn_major(Ht, 128), false);
             } else {
                 report_timeout(p.ws, 10);
             }
             // The tile leaves through the async proxy: generic global stores here would stall the next step's proxy
             // fence until they drain.  Waiting for the previous step's store to have read its tile before committing the
             // MMA orders that read before the overwrite of the tile two steps later.
-            bulk_store(keep_base + ch * 32768, Ht, 32768);
+            bulk_store(keep_base + ch * 32768, Ht, HT_BYTES);
             bulk_commit();
             bulk_wait_read<1>();
             mma_commit(&bar_mma);
@@ -643,10 +653,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
         tc_fence_after();
         if (s < 4) GDN_TICK(1, s * 5 + 3);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < NSH / 8; ++k) {
             float dl[8], ad[8];
-            tmem_ld8(tmem + lane_base + gc0 + 8 * k, dl);
-            chunk_load(ring + ADD, 128, r, hf * 8 + k, ad);
+            tmem_ld8(tmem + lane_base + lc0 + 8 * k, dl);
+            chunk_load(ring + ADD, 128, r, (lc0 >> 3) + k, ad);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 8; ++j) st[8 * k + j] = fmaf(Ge, st[8 * k + j], ad[j] - dl[j]);
@@ -658,12 +668,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     if (fin && ok) {
         const size_t soff = ((size_t)n * p.d.H + hd) * D * D + (size_t)r * D + gc0;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
+        for (int k = 0; k < NSH / 4; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
     }
     if (threadIdx.x == 0) bulk_wait_read<0>();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 128);
+    if (warp == 0) tmem_dealloc(tmem, NS);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1378,11 +1388,6 @@ static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
     return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kIntraThreads + 32, P, st);
 }
-static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
-    static bool done = false;
-    const int chains = P.p.d.N * P.p.d.H;
-    return launch_chunk_kernel(tc_scan_kernel, done, scan::SMEM_BYTES, ST_SCANS, chains * (P.scan_dirs == 2 ? 2 : 1), kThreads, P, st);
-}
 // Number of SMs of the current device (persistent kernels launch one CTA per SM).
 static int sm_count() {
     static int cached[64] = {};
@@ -1395,6 +1400,15 @@ static int sm_count() {
     return cached[dev];
 }
 
+static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
+    static bool done = false;
+    static bool done2 = false;
+    const int ctas = P.p.d.N * P.p.d.H * (P.scan_dirs == 2 ? 2 : 1);
+    // few chains: two CTAs per (chain, direction), each carrying half of the state columns
+    if (2 * ctas <= sm_count())
+        return launch_chunk_kernel(tc_scan_kernel<2>, done2, scan::Cfg<2>::SMEM_BYTES, ST_SCANS, 2 * ctas, kThreads, P, st);
+    return launch_chunk_kernel(tc_scan_kernel<1>, done, scan::Cfg<1>::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
+}
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
     static bool done = false;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
