@@ -175,9 +175,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 #pragma unroll 1
             for (int item = blockIdx.x; item < n_items && lok; item += gridDim.x, ph ^= 1) {
                 ChunkInfo x, nx;
-                chunk_info(p, x, item);
+                chunk_entry(p, x, item);
                 const bool has_next = item + (int)gridDim.x < n_items;
-                if (has_next) chunk_info(p, nx, item + gridDim.x);
+                if (has_next) chunk_entry(p, nx, item + gridDim.x);
                 pend_qk = pend_vo = false;
                 // the trip is under way: Q, K of the next one (loaded late in this trip) -> L2
                 if (!(lok = mbar_wait(&bar_ld0, ph))) break;
@@ -207,10 +207,18 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 // phase 3 is done: Q, K have been read for the last time
                 if (!(lok = mbar_wait(&bar_ld1, ph))) break;
                 if (has_next) {
+#ifdef GDN_PHASE_TIMING
+                    if (blockIdx.x == 0) g_ticks[3][10] = clock64();
+#endif
                     mbar_expect_tx(&bar_qk, 32768);
                     pend_qk = true;
 #pragma unroll 1
-                    for (int piece = 0; piece < 4; ++piece) load_piece(piece, nx);
+                    for (int piece = 0; piece < 4; ++piece) {
+                        load_piece(piece, nx);
+#ifdef GDN_PHASE_TIMING
+                        if (blockIdx.x == 0) g_ticks[3][11 + piece] = clock64();
+#endif
+                    }
                 }
                 // the three images are staged.  A store drains shared memory at some 32 bytes per cycle, so they leave in
                 // the order in which the next trip rewrites their tiles: E (fp32 scratch) and Nm (P) first, Bf last
@@ -239,58 +247,66 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     // The chunk table entry and the gate values of a trip are fetched one trip ahead into registers: they are tiny, but
     // read at the top of a trip their DRAM latency would be fully exposed.
     ChunkInfo xn;
-    chunk_info(p, xn, blockIdx.x);
-    float ng = 0.f, nb = 0.f;
-    auto fetch_gates = [&](const ChunkInfo& c) {   // g (0 when padded) and the erase gate b of this thread's token
-        ng = nb = 0.f;
-        if ((int)threadIdx.x < c.len) {
-            const size_t idx = (size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd;
-            ng = p.g[idx];
-            nb = p.beta[idx];
+    chunk_entry(p, xn, blockIdx.x);
+    // Warp 0 owns the gates: lane l holds g (0 when padded) and the erase gate b of tokens l and l + 32.
+    float ng[2] = {0.f, 0.f}, nb[2] = {0.f, 0.f};
+    auto fetch_gates = [&](const ChunkInfo& c) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int i = lane + 32 * h;
+            ng[h] = nb[h] = 0.f;
+            if (i < c.len) {
+                const size_t idx = (size_t)(c.tok0 + i) * H + c.hd;
+                ng[h] = p.g[idx];
+                nb[h] = p.beta[idx];
+            }
         }
     };
-    fetch_gates(xn);
+    if (warp == 0) fetch_gates(xn);
     // first trip: the inputs are loaded at once, one instruction per warp
     if (issuer) { mbar_expect_tx(&bar_qk, 32768); mbar_expect_tx(&bar_vo, VO_BYTES); }
     if (lane == 0 && warp < 8) load_piece(warp, xn);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
     const ChunkInfo x = xn;
-    const float g_now = ng, b_now = nb;
+    const float g_now[2] = {ng[0], ng[1]}, b_now[2] = {nb[0], nb[1]};
     const bool has_next = item + (int)gridDim.x < n_items;
     const bool first = item == (int)blockIdx.x;
-    if (has_next) chunk_info(p, xn, item + gridDim.x);
+    if (has_next) chunk_entry(p, xn, item + gridDim.x);
     GDN_TICK(0, 0);
     GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
 
-    // gates: g (0 when padded), erase gate b, write gate w; chunk-local cumulative decay
-    if (threadIdx.x < kC) {
-        const int i = threadIdx.x;
-        gam[i] = g_now; bb[i] = b_now; ww[i] = b_now;
-    }
-    cta_sync();
-    if (warp == 0) {   // inclusive prefix sum of the 64 log decays: lane l owns tokens l and l + 32
-        float a = gam[lane], b = gam[lane + 32];
+    // gates: erase gate b, write gate w, chunk-local cumulative decay gam (inclusive prefix sum of the 64 log decays),
+    // all by warp 0 in registers; the barrier before phase 1 publishes the arrays
+    if (warp == 0) {
+        float a = g_now[0], b = g_now[1];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
             if (lane >= o) { a += ua; b += ub; }
         }
         b += __shfl_sync(0xffffffffu, a, 31);
-        gam[lane] = a;
-        gam[lane + 32] = b;
+        const float gend = __shfl_sync(0xffffffffu, b, 31);
+        const float gc[2] = {a, b};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int i = lane + 32 * h;
+            const float G = expf(gc[h]);
+            gam[i] = gc[h];
+            gl[i] = gc[h] * kLog2e;
+            Gam[i] = G;
+            bb[i] = b_now[h]; ww[i] = b_now[h];
+            bgam[i] = b_now[h] * G;
+            ee[i] = expf(gend - gc[h]);
+            reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gc[h];
+        }
     }
-    cta_sync();
-    if (threadIdx.x < kC) {
-        const int i = threadIdx.x;
-        gl[i] = gam[i] * kLog2e;
-        Gam[i] = expf(gam[i]);
-        bgam[i] = bb[i] * Gam[i];
-        ee[i] = expf(gam[kC - 1] - gam[i]);
-        reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gam[i];
-    }
+    GDN_TICK(0, 20);
     if (ok) {
-        ok = mbar_wait(&bar_qk, in_phase) && mbar_wait(&bar_vo, in_phase);
+        ok = mbar_wait(&bar_vo, in_phase);
+        GDN_TICK(0, 21);
+        ok = ok && mbar_wait(&bar_qk, in_phase);
+        GDN_TICK(0, 22);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
     }
     if (ok && x.len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
@@ -313,7 +329,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     float* Af = reinterpret_cast<float*>(sm + XA);   // [64][kLdi]  strictly lower part of I + A
     float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][kLdi]  T
     float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
-    if (has_next && threadIdx.x < kC) fetch_gates(xn);   // next trip's gates -> registers while the product runs
+    if (has_next && warp == 0) fetch_gates(xn);   // next trip's gates -> registers while the product runs
     GDN_WAIT_MMA(2)
     if (ok && !first) {   // the previous trip's E and Nm stores have read their tiles (the fp32 scratch and P are next)
         ok = mbar_wait(&bar_free1, in_phase ^ 1);
@@ -792,9 +808,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 #pragma unroll 1
             for (int item = blockIdx.x; item < n_items && lok; item += gridDim.x, ph ^= 1) {
                 ChunkInfo x, nx;
-                chunk_info(p, x, item);
+                chunk_entry(p, x, item);
                 const bool has_next = item + (int)gridDim.x < n_items;
-                if (has_next) chunk_info(p, nx, item + gridDim.x);
+                if (has_next) chunk_entry(p, nx, item + gridDim.x);
                 const bool full = x.len == kC;
                 pend_k = pend1 = pend2 = false;
                 // the trip is under way (all its tiles have arrived): K of the next one, the only late load, -> L2
@@ -820,22 +836,21 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 #pragma unroll 1
                     for (int piece = 2; piece <= 7; ++piece) load_piece(piece, nx);
                 }
-                // phase 6 is done; V goes where dv is staged, so that store must have read its source
+                // phase 6 is done and the last readout holds its K values in registers: K first, the next trip starts with
+                // it; dO, T, V are not needed before its second phase (V goes where dv is staged, so that store must have
+                // read its source)
                 if (!(lok = mbar_wait(&bar_ld2, ph))) break;
-                if (has_next) {
-                    bulk_wait_read<0>();
-                    mbar_expect_tx(&bar_g2, G2_BYTES);
-                    pend2 = true;
-#pragma unroll 1
-                    for (int piece = 8; piece <= 12; ++piece) load_piece(piece, nx);
-                }
-                // the last readout holds its K values in registers
                 if (!(lok = mbar_wait(&bar_kfree, ph))) break;
                 if (has_next) {
                     mbar_expect_tx(&bar_k, K_BYTES);
                     pend_k = true;
                     load_piece(0, nx);
                     load_piece(1, nx);
+                    bulk_wait_read<0>();
+                    mbar_expect_tx(&bar_g2, G2_BYTES);
+                    pend2 = true;
+#pragma unroll 1
+                    for (int piece = 8; piece <= 12; ++piece) load_piece(piece, nx);
                 }
                 // dk is staged
                 if (!(lok = mbar_wait(&bar_st2, ph))) break;
@@ -860,7 +875,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     uint32_t mma_phase = 0, in_phase = 0;
     // chunk table entry and gates of a trip are fetched one trip ahead into registers (their latency would be exposed)
     ChunkInfo xn;
-    chunk_info(p, xn, blockIdx.x);
+    chunk_entry(p, xn, blockIdx.x);
     float ng = 0.f, ngend = 0.f, nb = 0.f;
     auto fetch_gates = [&](const ChunkInfo& c) {   // cumulative log decay of this thread's token and of the chunk end, gate b
         const float* gsrc = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)c.ch * kC;
@@ -878,7 +893,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const float g_now = ng, gend_now = ngend, b_now = nb;
     const bool has_next = item + (int)gridDim.x < n_items;
     const bool first = item == (int)blockIdx.x;
-    if (has_next) chunk_info(p, xn, item + gridDim.x);
+    if (has_next) chunk_entry(p, xn, item + gridDim.x);
 #ifdef GDN_PHASE_TIMING
     if (blockIdx.x == 0 && threadIdx.x == 0) g_trip_now = (item - (int)blockIdx.x) / (int)gridDim.x;
 #endif

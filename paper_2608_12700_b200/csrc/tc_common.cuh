@@ -131,6 +131,15 @@ __device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int i
     return true;
 }
 __device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) { return chunk_info(p, x, (int)blockIdx.x); }
+// Same for an item already known to exist: no header read and no branch, so the two table loads can stay in flight
+// until their values are used (the persistent kernels fetch the entry one trip ahead).
+__device__ __forceinline__ void chunk_entry(const Problem& p, ChunkInfo& x, int item) {
+    x.c = item / p.d.H;
+    x.hd = item % p.d.H;
+    x.ch = item;
+    x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
+    x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
+}
 
 // Wait for the MMAs committed to `bar`; on a timeout record it once.
 #define GDN_WAIT_MMA(where)                                                    \
