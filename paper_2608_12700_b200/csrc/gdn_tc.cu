@@ -1084,7 +1084,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + gbase;
     __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + gbase;
     if (ok && worker) {
-        float acc = 0.f;   // group A: <q, dq> ; group B: <v, dXv> over this thread's columns
+        // The two lane groups hold different quantities but share one instruction stream where they can (a warp runs
+        // both sides of a branch one after the other):
+        //   group A: dq = scale Gam (dO h^T) + (dP.D) K, staged ; acc = <q, dq>
+        //   group B: dXk, dXv -> operand tiles ; acc = <v, dXv> (dw partial) ; dv = w dXv, staged
+        float acc = 0.f;
+        const float coef = sc * Gam[tr], outscale = ga ? 1.f : bb[tr];
+        const unsigned char* dot_tile = sm + (ga ? QK : VT);   // q rows (128-row tile) or v rows (64-row tile)
+        unsigned char* stage = sm + (ga ? STG_A : STG_B);
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
@@ -1093,25 +1100,18 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             tmem_ld8(tmem + lane_base + 0 + cb, xk);      //                B: dXk
             tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: (dP.D) K    B: dXv
             tmem_wait_ld();
-            if (ga) {
-                chunk_load(sm + QK, 128, tr, cb >> 3, t8);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    a[j] = fmaf(sc * Gam[tr], a[j], b[j]);              // dq = scale Gam (dO h^T) + (dP.D) K
-                    acc = fmaf(t8[j], a[j], acc);
-                }
-                chunk_store(sm + STG_A, 64, tr, cb >> 3, a);
-            } else {
+            unpack8(*reinterpret_cast<const uint4*>(dot_tile + tile_chunk_off(ga ? 128 : 64, tr, cb >> 3)), t8);
+            if (!ga) {
                 chunk_store(sm + DXK, 64, tr, cb >> 3, xk);
                 chunk_store(sm + DXV, 64, tr, cb >> 3, b);
-                chunk_load(sm + VT, 64, tr, cb >> 3, t8);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    acc = fmaf(t8[j], b[j], acc);                       // dw partial
-                    b[j] *= bb[tr];                                     // dv = w dXv
-                }
-                chunk_store(sm + STG_B, 64, tr, cb >> 3, b);
             }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float val = ga ? fmaf(coef, a[j], b[j]) : b[j];   // (a select, not a zero coefficient: group B's
+                acc = fmaf(t8[j], val, acc);                            // lanes of `a` hold an unrelated accumulator)
+                b[j] = val * outscale;
+            }
+            chunk_store(stage, 64, tr, cb >> 3, b);
         }
         red[ga ? 0 : 1][grp][tr] = acc;
     }
@@ -1185,6 +1185,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         if (lane == 0) mbar_arrive(&bar_kfree);
         GDN_TICK(2, 17);
         float acc = 0.f;   // group A: <k, dk^col> ; group B: db = <k, G K + Gam dXk>
+        const float s6 = ga ? ee[tr] : Gam[tr], bg6 = bb[tr] * Gam[tr];
         if (ok) {
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
@@ -1196,17 +1197,17 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             tmem_ld8(tmem + lane_base + 0 + cb, d8);      // A: U dh'^T       B: dXk
             tmem_wait_ld();
             unpack8(kraw[part], kk);
+            // shared by both groups: A: dk^col = e (U dh'^T) + (dP.D)^T Q + (bG)^T K ; B: G K + Gam dXk; dotted with k
+            float t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                t[j] = fmaf(s6, d8[j], c8[j]);
+                acc = fmaf(kk[j], t[j], acc);
+            }
             if (ga) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float kcol = fmaf(ee[tr], d8[j], c8[j]);                     // dk^col
-                    acc = fmaf(kk[j], kcol, acc);
-                    a[j] = a[j] + bb[tr] * Gam[tr] * b[j] + kcol;                      // dk = Diag(b)(G K + Gam dXk) + dk^col
-                }
+                for (int j = 0; j < 8; ++j) a[j] = fmaf(bg6, b[j], a[j]) + t[j];       // dk = Diag(b)(G K + Gam dXk) + dk^col
                 chunk_store(sm + STG_K, 64, tr, cb >> 3, a);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) acc = fmaf(kk[j], fmaf(Gam[tr], d8[j], c8[j]), acc);
             }
         }
         }
