@@ -883,6 +883,23 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         ngend = gsrc[kC - 1];
         nb = ((int)threadIdx.x < c.len) ? p.beta[(size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd] : 0.f;
     };
+    // dbeta and dg of the previous trip's chunk, from its token-wise partial sums (warps 0 and 1; see the trip's end)
+    ChunkInfo xp = xn;
+    bool have_prev = false;
+    float bb_prev = 0.f, Gam_last_prev = 0.f;
+    auto finish_gates = [&]() {
+        const int i = threadIdx.x;
+        auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
+        const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
+        if (i < xp.len) p.dbeta[(size_t)(xp.tok0 + i) * H + xp.hd] = db + dw;
+        dgam[i] = fmaf(bb_prev, db, qdq - kcol);
+        asm volatile("bar.sync 2, 64;" ::: "memory");
+        if (warp == 0) {
+            constexpr int nw = kIntraThreads / 32;   // per-warp partial sums, one per lane
+            const float rsum = warp_sum(lane < nw ? scal[0][lane] : 0.f), hsum = warp_sum(lane < nw ? scal[1][lane] : 0.f);
+            write_dg_suffix(dgam, nullptr, rsum + Gam_last_prev * hsum, p.dg + (size_t)xp.tok0 * H + xp.hd, (size_t)H, xp.len, lane);
+        }
+    };
     // first trip: every group is loaded at once, one instruction per warp
     if (issuer) { mbar_expect_tx(&bar_k, K_BYTES); mbar_expect_tx(&bar_g1, G1_BYTES); mbar_expect_tx(&bar_g2, G2_BYTES); }
     if (lane == 0 && warp < 13) load_piece(warp, xn);
@@ -907,8 +924,12 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         ee[i] = expf(gend_now - g_now);
         bb[i] = b_now;
     }
+    GDN_TICK(2, 19);
     if (ok) {
-        ok = mbar_wait(&bar_g1, in_phase) && mbar_wait(&bar_k, in_phase);
+        ok = mbar_wait(&bar_g1, in_phase);
+        GDN_TICK(2, 20);
+        ok = ok && mbar_wait(&bar_k, in_phase);
+        GDN_TICK(2, 21);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
     }
     if (ok && x.len < kC) {
@@ -928,11 +949,13 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
     }
     if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // every tile of this trip has arrived
-    // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up)
     if (has_next && threadIdx.x < kC) fetch_gates(xn);
+    // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up); warps 0 and 1
+    // finish the previous chunk's gate gradients instead
     float hh = 0.f;
+    if (ok && have_prev && warp < 2) finish_gates();
 #pragma unroll 1
-    for (int t = threadIdx.x; t < 2048; t += kIntraThreads) {
+    for (int t = (int)threadIdx.x - 64; t >= 0 && t < 2048; t += kIntraThreads - 64) {
         float a[8], b[8];
         unpack8(*reinterpret_cast<const uint4*>(sm + HH + t * 16), a);
         unpack8(*reinterpret_cast<const uint4*>(sm + DH + t * 16), b);
@@ -1223,24 +1246,17 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     GDN_TICK(2, 14);
     if (threadIdx.x == 32) mbar_arrive(&bar_st2);   // dk is staged: the loader stores it
     if (ok && !full) flush_rows(sm + STG_K, gdk, rowp, x.len, kIntraThreads);
-    if (threadIdx.x < kC) {
-        const int i = threadIdx.x;
-        auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
-        const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
-        if (i < x.len) p.dbeta[(size_t)(x.tok0 + i) * H + x.hd] = db + dw;
-        dgam[i] = fmaf(bb[i], db, qdq - kcol);
-    }
-    cta_sync();
-    if (warp == 0 && ok) {
-        float rsum = 0.f, hsum = 0.f;
-        for (int w = 0; w < kIntraThreads / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
-        write_dg_suffix(dgam, nullptr, rsum + Gam[kC - 1] * hsum, p.dg + (size_t)x.tok0 * H + x.hd, (size_t)H, x.len, lane);
-    }
+    // The token-wise sums are complete; turning them into dbeta and dg is left to warps 0 and 1 during the next trip's
+    // first products (finish_gates).  They keep what the next trip overwrites: this chunk's gates and place.
+    if (threadIdx.x < kC) { bb_prev = bb[threadIdx.x]; Gam_last_prev = Gam[kC - 1]; }
+    xp = x;
+    have_prev = true;
     tc_fence_before();
     cta_sync();   // every reader of this trip's tiles and scratch is done
     GDN_TICK(2, 15);
     if (!ok) break;
     }
+    if (ok && have_prev && warp < 2) finish_gates();
     GDN_TRIP(1, 20);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
