@@ -15,6 +15,14 @@
 #include "tc_common.cuh"
 
 namespace gdn {
+
+// Optional phase timing (compile with -DGDN_PHASE_TIMING): thread 0 of CTA 0 stamps clock64() at phase borders of one step.
+#ifdef GDN_PHASE_TIMING
+__device__ long long g_ticks64[32];
+#define T64(idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && s == 5) g_ticks64[idx] = clock64(); } while (0)
+#else
+#define T64(idx) do { } while (0)
+#endif
 namespace {
 
 constexpr int D6 = 64;
@@ -48,8 +56,8 @@ __global__ void tc64_gamma_kernel(Problem p) {
     out[lane + 32] = b;
 }
 
-__device__ __forceinline__ void zero_tail_rows64(unsigned char* tile, int len) {   // [64][64] tile
-    for (int t = threadIdx.x; t < (kC - len) * 8; t += blockDim.x)
+__device__ __forceinline__ void zero_tail_rows64(unsigned char* tile, int len) {   // [64][64] tile; threads 0 .. kThreads64-1
+    for (int t = threadIdx.x; t < (kC - len) * 8; t += kThreads64)
         *reinterpret_cast<uint4*>(tile + tile_chunk_off(64, len + t / 8, t % 8)) = make_uint4(0, 0, 0, 0);
 }
 
@@ -252,7 +260,7 @@ static_assert(2 * (SMEM_BYTES + 4096) <= 227 * 1024, "two CTAs per SM");
 constexpr uint32_t C0 = 0, C1 = 64, C2 = 128, C3 = 192, LB = 16u << 16;
 }  // namespace b64
 
-__global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_constant__ Tc64Params P) {
+__global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __grid_constant__ Tc64Params P) {
     using namespace b64;
     const Problem& p = P.p;
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
@@ -267,8 +275,8 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], dgp[2][kC], scal[2][kThreads64 / 32];
-    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ __align__(16) float gl2[2][kC], Gam2[2][kC], ee2[2][kC], dgp[2][kC], scal[2][kThreads64 / 32];
+    __shared__ uint64_t bar_full[STAGES], bar_st, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, half = warp >> 2;
@@ -277,8 +285,13 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
     const int cb0 = half * 32;                // first of this thread's 32 columns
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
+    // Warp 8 only moves data: its first lane stores a step's staged gradients and then loads the tiles of the step
+    // after next into the ring slot they came from.  It follows the other warps through an mbarrier and shares no
+    // block-wide barrier with them inside the loop (they use a named barrier).
+    const bool loader = warp == kThreads64 / 32;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) mbar_init(&bar_full[s], 1);
+        mbar_init(&bar_st, 1);
         mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
@@ -298,8 +311,29 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         tma_load_2d(st + OT, &P.tm_do, hd * D6, tok0, &bar_full[stage]);
         bulk_load(st + HT, p.ws + p.L.hc + ((size_t)c * H + hd) * 8192, 8192, &bar_full[stage]);
     };
-    if (threadIdx.x == 0)
-        for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
+    if (loader) {
+        if (lane == 0) {
+            for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
+#pragma unroll 1
+            for (int s = 0; s < nsteps; ++s) {
+                if (!mbar_wait(&bar_st, s & 1)) break;          // step s has staged its gradient rows (or flushed them)
+                const int c = c1 - 1 - s;
+                if (chunk_len[c] == kC) {
+                    const int tok0 = chunk_tok0[c];
+                    unsigned char* st = sm + (s % STAGES) * STAGE_BYTES;
+                    tma_store_2d(&P.tm_dv, hd * D6, tok0, st + VT);
+                    tma_store_2d(&P.tm_dk, hd * D6, tok0, st + KT);
+                    tma_store_2d(&P.tm_dq, hd * D6, tok0, st + QT);
+                    bulk_commit();
+                    bulk_wait_read<0>();   // the ring slot is loaded over next
+                }
+                if (s + STAGES < nsteps) fill(s + STAGES);
+            }
+            bulk_wait_read<0>();
+        }
+        return;
+    }
+    auto cta_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kThreads64) : "memory"); };   // all warps but the loader
 
     float st[32];   // group A: dh' row r, columns cb0 .. cb0 + 31 (gradient w.r.t. the state leaving the current chunk)
     const size_t soff = ((size_t)n * H + hd) * D6 * D6 + (size_t)r * D6 + cb0;
@@ -308,24 +342,35 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         float4 v = (p.dhT && ga) ? *reinterpret_cast<const float4*>(p.dhT + soff + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
         st[4 * k] = v.x; st[4 * k + 1] = v.y; st[4 * k + 2] = v.z; st[4 * k + 3] = v.w;
     }
+    // Gate arrays of a step (log2-scaled cumulative decay, Gam = exp(gam), e = exp(gam_end - gam)) are prepared one
+    // step ahead, into the other of two sets, while the tensor pipe works; their inputs are fetched a step before that.
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
-    float gnext = (threadIdx.x < kC && nsteps > 0) ? gamma[((size_t)(c1 - 1) * H + hd) * kC + threadIdx.x] : 0.f;
+    auto gate_row = [&](int step) { return gamma + ((size_t)(c1 - 1 - step) * H + hd) * kC; };
+    auto make_gates = [&](int set, float g, float gend) {
+        gl2[set][threadIdx.x] = g * kLog2e;
+        Gam2[set][threadIdx.x] = expf(g);
+        ee2[set][threadIdx.x] = ex2((gend - g) * kLog2e);
+    };
+    float gnext = 0.f, gend_next = 0.f;
+    if (threadIdx.x < kC && nsteps > 0) {
+        make_gates(0, gate_row(0)[threadIdx.x], gate_row(0)[kC - 1]);
+        if (nsteps > 1) { gnext = gate_row(1)[threadIdx.x]; gend_next = gate_row(1)[kC - 1]; }
+    }
     bool ok = true;
     uint32_t mma_phase = 0;
+    int len_n = nsteps > 0 ? chunk_len[c1 - 1] : 0, tok0_n = nsteps > 0 ? chunk_tok0[c1 - 1] : 0;   // fetched a step ahead
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
-        const int c = c1 - 1 - s, stage = s % STAGES, len = chunk_len[c], tok0 = chunk_tok0[c];
+        const int c = c1 - 1 - s, stage = s % STAGES, len = len_n, tok0 = tok0_n;
+        if (s + 1 < nsteps) { len_n = chunk_len[c - 1]; tok0_n = chunk_tok0[c - 1]; }
         const size_t ch = (size_t)c * H + hd;
         unsigned char* tiles = sm + stage * STAGE_BYTES;
-        if (threadIdx.x < kC) {
-            gl[threadIdx.x] = gnext * kLog2e;
-            Gam[threadIdx.x] = expf(gnext);
-            if (s + 1 < nsteps) gnext = gamma[(ch - H) * kC + threadIdx.x];
-        }
-        __syncthreads();
-        if (threadIdx.x < kC) ee[threadIdx.x] = ex2(gl[kC - 1] - gl[threadIdx.x]);
+        const float *gl = gl2[s & 1], *Gam = Gam2[s & 1], *ee = ee2[s & 1];
+        T64(0);
+        T64(1);
         ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 50); break; }
+        T64(2);
         if (len < kC) {
             zero_tail_rows64(tiles + QT, len);
             zero_tail_rows64(tiles + KT, len);
@@ -344,8 +389,9 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             }
         }
         fence_async_smem();
-        __syncthreads();
+        cta_sync();
         const float Ge = Gam[kC - 1];
+        T64(3);
         // ---- phase 1: S = Q K^T ; dO V^T ; K dh' (group A) | dO h^T ; V dh'^T (group B)
         if (threadIdx.x == 0) {
             tc_fence_after();
@@ -356,9 +402,15 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             mma_tile<64, 64, 64>(tmem + C2 + LB, op_k_major(tiles + VT, 64), op_k_major(sm + DH, 64), false);
             mma_commit(&bar_mma);
         }
+        T64(4);
+        if (threadIdx.x < kC && s + 1 < nsteps) {
+            make_gates((s + 1) & 1, gnext, gend_next);
+            if (s + 2 < nsteps) { gnext = gate_row(s + 2)[threadIdx.x]; gend_next = gate_row(s + 2)[kC - 1]; }
+        }
         GDN_WAIT_MMA(51)
         if (!ok) break;
-        for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {   // Diag(Gam) dO over the dh' tile, which no MMA reads any more
+        T64(5);
+        for (int t = threadIdx.x; t < kC * 8; t += kThreads64) {   // Diag(Gam) dO over the dh' tile, which no MMA reads any more
             const int i = t >> 3, cch = t & 7;
             float v[8];
             chunk_load(tiles + OT, 64, i, cch, v);
@@ -366,6 +418,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
             chunk_store(sm + DH, 64, i, cch, v);
         }
+        T64(6);
         float rs = 0.f;   // sum_j r_j, r_j = e_j <(K dh')_j, V_j>
 #pragma unroll 1
         for (int part = 0; part < 4; ++part) {
@@ -393,7 +446,8 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         rs *= ee[r];
         tc_fence_before();
         fence_async_smem();
-        __syncthreads();
+        cta_sync();
+        T64(7);
         // ---- phase 2: P^T dO ; (Diag(Gam) Q)^T dO (group A) | (dP.D) K ; (dP.D)^T Q (group B)
         if (threadIdx.x == 0) {
             tc_fence_after();
@@ -403,11 +457,14 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             mma_tile<64, 64, 64>(tmem + C3 + LB, op_mn_major(sm + DPD, 64), op_mn_major(tiles + QT, 64), false);
             mma_commit(&bar_mma);
         }
+        T64(8);
         GDN_WAIT_MMA(52)
         if (!ok) break;
+        T64(9);
         float dot = 0.f;   // group B: <q_r, dq_r> - <k_r, dk_r> over this thread's columns
-        // Gradient rows are staged token-major over tiles that phase 2 has finished with (dv over P, dk over dP.D, dq
-        // over Diag(Gam) dO) and leave by TMA stores; generic global stores here would be one 16-byte piece per row.
+        // Gradient rows are staged token-major in place over this step's input tiles (dv over V, which was last read in
+        // phase 1; dk over K and dq over Q, where a thread overwrites exactly the piece it has just read) and leave by TMA
+        // stores; generic global stores here would be one 16-byte piece per row.
 #pragma unroll 1
         for (int part = 0; part < 4; ++part) {
             float a[8], b[8], x[8];
@@ -418,7 +475,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
             if (ga) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) a[j] = fmaf(sc, a[j], ee[r] * b[j]);      // dv = scale P^T dO + Diag(e) K dh'
-                chunk_store(sm + PX, 64, r, jb >> 3, a);
+                chunk_store(tiles + VT, 64, r, jb >> 3, a);
             } else {
                 chunk_load(tiles + KT, 64, r, jb >> 3, x);
 #pragma unroll
@@ -426,7 +483,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
                     a[j] = fmaf(ee[r], b[j], a[j]);                                    // dk = (dP.D)^T Q + Diag(e) V dh'^T
                     dot = fmaf(-x[j], a[j], dot);
                 }
-                chunk_store(sm + DPD, 64, r, jb >> 3, a);
+                chunk_store(tiles + KT, 64, r, jb >> 3, a);
             }
             tmem_ld8(tmem + lane_base + C0 + jb, a);     //                  B: dO h^T
             tmem_ld8(tmem + lane_base + C1 + jb, b);     //                  B: (dP.D) K
@@ -438,9 +495,10 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
                     a[j] = fmaf(sc * Gam[r], a[j], b[j]);                              // dq = scale Gam dO h^T + (dP.D) K
                     dot = fmaf(x[j], a[j], dot);
                 }
-                chunk_store(sm + DH, 64, r, jb >> 3, a);
+                chunk_store(tiles + QT, 64, r, jb >> 3, a);
             }
         }
+        T64(10);
         if (!ga) dgp[half][r] = dot;
         // group A: dh = Gam_e dh' + scale (Diag(Gam) Q)^T dO
 #pragma unroll
@@ -456,41 +514,35 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_bwd_kernel(const __grid_co
         if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
         tc_fence_before();
         fence_async_smem();
-        __syncthreads();   // every reader of this stage's tiles is done; partial sums and staged rows are visible
-        if (len == kC) {
-            if (threadIdx.x == 32) {
-                tma_store_2d(&P.tm_dv, hd * D6, tok0, sm + PX);
-                tma_store_2d(&P.tm_dk, hd * D6, tok0, sm + DPD);
-                tma_store_2d(&P.tm_dq, hd * D6, tok0, sm + DH);
-                bulk_commit();
-                if (s + STAGES < nsteps) fill(s + STAGES);
-                bulk_wait_read<0>();   // the staging tiles are rewritten right after the next barrier
-            }
-        } else {   // ragged tail: rows beyond the sequence must not be written
+        cta_sync();   // every reader of this stage's tiles is done; partial sums and staged rows are visible
+        if (len < kC) {   // ragged tail: rows beyond the sequence must not be written
             const size_t gbase = ((size_t)tok0 * H + hd) * D6;
-            for (int t = threadIdx.x; t < kC * 8; t += blockDim.x) {
+            for (int t = threadIdx.x; t < kC * 8; t += kThreads64) {
                 const int i = t >> 3, chk = t & 7;
                 if (i < len) {
                     const size_t o = gbase + (size_t)i * H * D6 + chk * 8;
-                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dv) + o) = *reinterpret_cast<const uint4*>(sm + PX + tile_chunk_off(64, i, chk));
-                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dk) + o) = *reinterpret_cast<const uint4*>(sm + DPD + tile_chunk_off(64, i, chk));
-                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dq) + o) = *reinterpret_cast<const uint4*>(sm + DH + tile_chunk_off(64, i, chk));
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dv) + o) = *reinterpret_cast<const uint4*>(tiles + VT + tile_chunk_off(64, i, chk));
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dk) + o) = *reinterpret_cast<const uint4*>(tiles + KT + tile_chunk_off(64, i, chk));
+                    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.dq) + o) = *reinterpret_cast<const uint4*>(tiles + QT + tile_chunk_off(64, i, chk));
                 }
             }
-            if (threadIdx.x == 32 && s + STAGES < nsteps) fill(s + STAGES);
+            cta_sync();   // the ring slot is handed to the loader only after every row has been read
         }
+        T64(11);
+        if (threadIdx.x == 32) mbar_arrive(&bar_st);
         if (warp == 0) {
             float rsum = 0.f, hsum = 0.f;
             for (int w = 0; w < kThreads64 / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
             write_dg_suffix(dgp[0], dgp[1], rsum + Ge * hsum, p.dg + (size_t)tok0 * H + hd, (size_t)H, len, lane);
         }
+        T64(12);
     }
     if (p.dh0 && ok && ga) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) *reinterpret_cast<float4*>(p.dh0 + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
     }
     tc_fence_before();
-    __syncthreads();
+    cta_sync();
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
@@ -582,9 +634,15 @@ cudaError_t tc64_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t 
     const int chains = p.d.N * p.d.H;
     if (chains > 0) {
         StageScope t(ST_RSCAN, st);
-        tc64_bwd_kernel<<<chains, kThreads64, b64::SMEM_BYTES, st>>>(P);
+        tc64_bwd_kernel<<<chains, kThreads64 + 32, b64::SMEM_BYTES, st>>>(P);
     }
     return cudaGetLastError();
 }
 
 }  // namespace gdn
+
+#ifdef GDN_PHASE_TIMING
+extern "C" int gdn_debug_ticks64(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks64, sizeof(long long) * 32);
+}
+#endif
