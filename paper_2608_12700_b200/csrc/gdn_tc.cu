@@ -42,12 +42,14 @@ namespace {
 
 constexpr int D = 128;          // d_k = d_v
 constexpr int kThreads = 256;   // 8 warps: lane quadrant = warp % 4, column half = warp / 4 (scan, out)
-// The chunk kernels run 16 warps: four warps share a TMEM lane quadrant and split the 64 token columns four ways,
-// which shortens every thread's serial readout chain and gives the scheduler more warps to hide latencies with.
+// The chunk kernels run 16 readout warps: four warps share a TMEM lane quadrant and split the 64 token columns four
+// ways, which shortens every thread's serial readout chain and gives the scheduler more warps to hide latencies with.
 constexpr int kWideThreads = 512;
 constexpr int kGroups = kWideThreads / 128;   // column groups
 constexpr int kTG = kC / kGroups;             // token columns per group (16)
-constexpr int kIntraThreads = kWideThreads + 32;   // the chunk kernels add one warp whose first lane only issues MMAs
+constexpr int kIntraThreads = kWideThreads + 32;   // ... plus one warp whose first lane only issues MMAs; the kernels are
+                                                   // launched with one more warp on top (kIntraThreads + 32) that only
+                                                   // issues bulk copies and takes no part in the named barrier
 struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
@@ -698,8 +700,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 // Products (all on tcgen05, outputs transposed: features on TMEM lanes, tokens on columns, except the 64 x 64
 // token-token matrices which use M = 64):
 //   phase 1  S = Q K^T ; (W h)^T ; (K dh')^T                      -> P = tril(S . D)
-//   phase 2  (P^T dO)^T                                            -> U = U~ - W h ; dU = scale P^T dO + Diag(e) K dh'
-//   phase 3  dO U^T ; (dO h^T)^T ; -(dU h^T)^T                     -> dPD = scale tril(dO U^T) . D ; dW
+//   phase 2  (P^T dO)^T ; then, under the readout, dO h^T          -> U = U~ - W h ; dU = scale P^T dO + Diag(e) K dh'
+//   phase 3  dO U^T ; -(dU h^T)^T                                  -> dPD = scale tril(dO U^T) . D ; dW
 //   phase 4  (dPD K)^T ; (T^T dW)^T ; (T^T dU)^T ; (dPD^T Q)^T ; (U dh'^T)^T
 //                                                                  -> dq ; dXk ; dXv ; dv ; dw
 //   phase 5  dXk W^T + dXv U~^T                                    -> G = -stril(.) . D ; Diag(b) G
@@ -715,20 +717,20 @@ namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
 constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB   later staged dv
 constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
-constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB   later staged dk
+constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
 constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each
 constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
-constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each
+constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each, then staged dk
 constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dq
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
 constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
 // token-major staging of dq (over dU^T, last read by the early products of phase 4), of dv (in place over V: a thread
-// overwrites exactly the chunk it has just read) and of dk (over W^T, last read by phase 5).  None of these is read
-// by the late products of phase 4 or rewritten within the trip (the loads that run ahead go to other regions), so
-// the asynchronous stores need no wait before the trip ends.
+// overwrites exactly the chunk it has just read) and of dk (over G, last read by phase 6).  None of these is read by
+// the late products of phase 4 or rewritten within the trip, and of the loads that run ahead only V targets one of
+// them (after its store has read it), so the asynchronous stores need no wait on the critical path.
 constexpr uint32_t STG_A = DUT, STG_B = VT, STG_K = UT;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
@@ -739,7 +741,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     using namespace intra;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
-    // tiles of its next one are pulled into L2, so that the loads at the top of the next trip do not wait for HBM.
+    // tiles of its next one are loaded into the regions the current one has finished with.
     const int H = p.d.H;
     const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
     if ((int)blockIdx.x >= n_items) return;
