@@ -58,14 +58,46 @@ struct TcParams {
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
 };
 
-// Blocked inverse of I + A (unit lower triangular, 16 x 16 blocks), fp32 in shared memory, rows of kLdi floats:
-//   T_rr = (I + A_rr)^-1 ;  At_rk = T_rr A_rk (r > k) ;  T_rc = -sum_{k=c}^{r-1} At_rk T_kc, one block diagonal at a time.
-// These steps are bound by shared-memory load issue, so a thread produces four adjacent outputs of a row: one scalar
-// (broadcast) and one 16-byte load feed four FMAs.  inv_premul forms every At_rk; inv_level fills block diagonal DIST.
+// Blocked inverse of I + A (unit lower triangular), fp32 in shared memory, rows of kLdi floats:
+//   diagonal 8 x 8 blocks by forward substitution; the 8 x 8 block below the diagonal of every 16 x 16 diagonal block
+//   from T10 = -T11 (A10 T00); then with 16 x 16 blocks  At_rk = T_rr A_rk (r > k)  and
+//   T_rc = -sum_{k=c}^{r-1} At_rk T_kc, one block diagonal at a time.
+// These steps are chains of dependent FMAs fed by shared-memory loads, so a thread produces four adjacent outputs of a
+// row (one broadcast scalar and one 16-byte load feed four FMAs) and the longer sums are split over SPLIT adjacent
+// lanes and combined by shuffles.
 constexpr int kLdi = 68;   // row pitch: 16-byte aligned rows, conflict-free for the access patterns below
+__device__ __forceinline__ void inv_diag8(const float* Af, float* Tf) {   // threads 0..63: column j of block b0
+    if (threadIdx.x < kC) {   // t_i = [i == j] - sum_{m<i} A_im t_m
+        const int b0 = (threadIdx.x >> 3) * 8, j = threadIdx.x & 7;
+        float t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float s = (i == j) ? 1.f : 0.f;
+#pragma unroll
+            for (int m = 0; m < i; ++m) s = fmaf(-Af[(b0 + i) * kLdi + b0 + m], t[m], s);
+            t[i] = s;
+            Tf[(b0 + i) * kLdi + b0 + j] = s;
+        }
+    }
+}
+__device__ __forceinline__ void inv_diag16(const float* Af, float* Tf, float* Xf) {   // threads 0..255: one entry each
+    if (threadIdx.x < 256) {
+        const int r0 = (threadIdx.x >> 6) * 16, i = (threadIdx.x >> 3) & 7, j = threadIdx.x & 7;
+        float x = 0.f;   // X = A10 T00
+#pragma unroll
+        for (int m = 0; m < 8; ++m) x = fmaf(Af[(r0 + 8 + i) * kLdi + r0 + m], Tf[(r0 + m) * kLdi + r0 + j], x);
+        Xf[(r0 + 8 + i) * kLdi + r0 + j] = x;
+        asm volatile("bar.sync 4, 256;" ::: "memory");
+        float s = 0.f;   // T10 = -T11 X
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s = fmaf(Tf[(r0 + 8 + i) * kLdi + r0 + 8 + k], Xf[(r0 + 8 + k) * kLdi + r0 + j], s);
+        Tf[(r0 + 8 + i) * kLdi + r0 + j] = -s;     // (disjoint from T00 and T11, which other threads still read)
+        Tf[(r0 + i) * kLdi + r0 + 8 + j] = 0.f;    // the block above the diagonal
+    }
+}
 __device__ __forceinline__ void inv_premul(const float* Af, const float* Tf, float* Sf) {
     // six blocks below the diagonal: (1,0) (2,0) (2,1) (3,0) (3,1) (3,2)
-    for (int o = threadIdx.x; o < 6 * 64; o += blockDim.x) {
+    for (int o = threadIdx.x; o < 6 * 64; o += kIntraThreads) {
         const int blk = o >> 6, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
         const int rb = (blk == 0 ? 1 : blk < 3 ? 2 : 3) * 16, cb = (blk == 0 ? 0 : blk < 3 ? blk - 1 : blk - 3) * 16;
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -78,18 +110,30 @@ __device__ __forceinline__ void inv_premul(const float* Af, const float* Tf, flo
         *reinterpret_cast<float4*>(Sf + (rb + ii) * kLdi + cb + j4) = s;
     }
 }
-template <int DIST>
+template <int DIST, int SPLIT>
 __device__ __forceinline__ void inv_level(const float* At, float* Tf) {
-    for (int o = threadIdx.x; o < (4 - DIST) * 64; o += blockDim.x) {
+    constexpr int items = (4 - DIST) * 64, len = 16 * DIST / SPLIT;
+    static_assert(items * SPLIT <= kWideThreads && (items * SPLIT) % 32 == 0, "one pass, whole warps");
+    if (threadIdx.x < items * SPLIT) {
+        // a warp serves 32 / SPLIT items; the lanes of a quarter-warp share `part`, so their 16-byte loads fall into one
+        // row of T (no bank conflicts), and the partial sums of an item sit 32 / SPLIT lanes apart
+        constexpr int G = 32 / SPLIT;
+        const int wl = threadIdx.x & 31, o = (threadIdx.x >> 5) * G + (wl % G), part = wl / G;
         const int cb = (o >> 6) * 16, rb = cb + DIST * 16, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int m = 0; m < 16 * DIST; ++m) {
+        for (int mm = 0; mm < len; ++mm) {
+            const int m = part * len + mm;
             const float a = At[(rb + ii) * kLdi + cb + m];
             const float4 v = *reinterpret_cast<const float4*>(Tf + (cb + m) * kLdi + cb + j4);
             s.x = fmaf(a, v.x, s.x); s.y = fmaf(a, v.y, s.y); s.z = fmaf(a, v.z, s.z); s.w = fmaf(a, v.w, s.w);
         }
-        *reinterpret_cast<float4*>(Tf + (rb + ii) * kLdi + cb + j4) = make_float4(-s.x, -s.y, -s.z, -s.w);
+#pragma unroll
+        for (int d = G; d < 32; d <<= 1) {
+            s.x += __shfl_xor_sync(0xffffffffu, s.x, d); s.y += __shfl_xor_sync(0xffffffffu, s.y, d);
+            s.z += __shfl_xor_sync(0xffffffffu, s.z, d); s.w += __shfl_xor_sync(0xffffffffu, s.w, d);
+        }
+        if (part == 0) *reinterpret_cast<float4*>(Tf + (rb + ii) * kLdi + cb + j4) = make_float4(-s.x, -s.y, -s.z, -s.w);
     }
 }
 
@@ -363,35 +407,25 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     tc_fence_before();
     cta_sync();
     GDN_TICK(0, 3);
-    // ---- T = (I + A)^-1 by blocks of 16: diagonal blocks by forward substitution, then block row r of block
-    // column c from  T_rc = -T_rr (sum_{k=c}^{r-1} A_rk T_kc),  one block diagonal at a time.  All fp32.
-    if (threadIdx.x < kC) {   // column j of the inverse of diagonal block b0: t_i = [i == j] - sum_{m<i} A_im t_m
-        const int b0 = (threadIdx.x >> 4) * 16, j = threadIdx.x & 15;
-        float t[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            float s = (i == j) ? 1.f : 0.f;
-#pragma unroll
-            for (int m = 0; m < i; ++m) s = fmaf(-Af[(b0 + i) * kLdi + b0 + m], t[m], s);
-            t[i] = s;
-            Tf[(b0 + i) * kLdi + b0 + j] = s;
-        }
-    }
-    cta_sync();
-    GDN_TICK(0, 16);
+    // ---- T = (I + A)^-1, blocked (see inv_diag8 ... inv_level).  All fp32.
+    inv_diag8(Af, Tf);
     if (ok && !first) {   // every store of the previous trip has read its tile (the scratch S lies over W^T)
         ok = mbar_wait(&bar_free, in_phase ^ 1);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 5);
     }
+    cta_sync();
+    inv_diag16(Af, Tf, Sf);
+    cta_sync();
+    GDN_TICK(0, 16);
     inv_premul(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
     cta_sync();
-    inv_level<1>(Sf, Tf);
+    inv_level<1, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 17);
-    inv_level<2>(Sf, Tf);
+    inv_level<2, 4>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 18);
-    inv_level<3>(Sf, Tf);
+    inv_level<3, 4>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 4);
     for (int t = threadIdx.x; t < kC * 8; t += kIntraThreads) {
