@@ -738,8 +738,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 //   phase 3  dO U^T ; -(dU h^T)^T                                  -> dPD = scale tril(dO U^T) . D ; dW
 //   phase 4  (dPD K)^T ; (T^T dW)^T ; (T^T dU)^T ; (dPD^T Q)^T ; (U dh'^T)^T
 //                                                                  -> dq ; dXk ; dXv ; dv ; dw
-//   phase 5  dXk W^T + dXv U~^T                                    -> G = -stril(.) . D ; Diag(b) G
-//   phase 6  (G K)^T ; += ((Diag(b) G)^T K)^T                      -> dk ; db ; dgamma -> dg
+//   phase 5  dXk W^T + dXv U~^T ; then, under the readout, T^T dW   -> G = -stril(.) . D ; Diag(b) G
+//   phase 6  G K ; += (Diag(b) G)^T K                               -> dk ; db ; dgamma -> dg
 // The decay gradient uses the identities  rowsum(dP.P) + scale Gam <q, dO h^T> = <q, dq>  and its analogues for
 // k:  dgamma_i = <q_i, dq_i> + <k_i, dk_i^row> - <k_i, dk_i^col>, where dk^row = Diag(b)(G K + Diag(Gam) dXk)
 // collects the terms in which k_i enters with exp(+gamma_i) and dk^col those with exp(-gamma_i); the last row
@@ -1083,9 +1083,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // columns ("group B", address + 16 lanes), and one tcgen05.ld serves both groups.
     //   columns   group A                               group B
     //   0..127    U dh'^T (ph 4)                        dP (ph 3, 64 cols) -> dXk (ph 4)
-    //   128..255  (dP.D) K (ph 4) -> dXk again (ph 6)   dXv (ph 4)
-    //   256..383  dW^T (ph 3, all lanes) -> dk^col      G K (ph 6)
-    //   384..511  dO h^T (ph 2) -> (bG) K (ph 6)        dA (ph 5, 64 cols)
+    //   128..255  (dP.D) K (ph 4) -> dXk again (ph 5)   dXv (ph 4)
+    //   256..383  dW^T (ph 3, all lanes) -> dk^col      -
+    //   384..511  dO h^T (ph 2) -> G K (ph 6)           dA (ph 5, 64 cols)
     constexpr uint32_t LB = 16u << 16;
     const bool ga = lane < 16;
     const int tr = q4 * 16 + (lane & 15);   // token row of this lane in token-major accumulators
@@ -1186,6 +1186,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
         mma_commit(&bar_mma);
         mma_commit(&bar_ld1);   // Q, U~^T, dh', h (by now dXk, dXv) have been read for the last time
+        // dXk once more, on the lanes of group A where dk is assembled; first read after phase 6
+        mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);
     } else if (threadIdx.x == 32) {
         // staged dq, dv leave through the async proxy (generic global stores would stall the next proxy fence); the
         // loader issues the stores
@@ -1225,10 +1227,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // ---- phase 6
     if (ok && issuer) {
         tc_fence_after();
-        mma_tile<64, 128, 64>(tmem + 256 + LB, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);       // G K
+        mma_tile<64, 128, 64>(tmem + 384, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);            // G K
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), true);           // += (bG)^T K
-        mma_tile<64, 128, 64>(tmem + 384, op_k_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), false);           // (bG) K
-        mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);               // T^T dW again, group A
         mma_commit(&bar_mma);
         mma_commit(&bar_ld2);   // dW^T (over dO) and T have been read for the last time
     }
@@ -1243,34 +1243,35 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar_kfree);
         GDN_TICK(2, 17);
-        float acc = 0.f;   // group A: <k, dk^col> ; group B: db = <k, G K + Gam dXk>
-        const float s6 = ga ? ee[tr] : Gam[tr], bg6 = bb[tr] * Gam[tr];
+        // Group A assembles dk = Diag(b)(G K + Gam dXk) + dk^col and both row dots with k; the lanes of group B hold
+        // nothing of this phase (Diag(b) G K is a row scaling of G K, so one product serves dk and db).
+        float acc_col = 0.f, acc_db = 0.f;   // <k, dk^col> ; db = <k, G K + Gam dXk>
+        const float e6 = ee[tr], G6 = Gam[tr], b6 = bb[tr];
         if (ok) {
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
             float a[8], b[8], c8[8], d8[8], kk[8];
-            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: (bG) K
+            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: G K
             tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: dXk
-            tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: dk^col part   B: G K
-            tmem_ld8(tmem + lane_base + 0 + cb, d8);      // A: U dh'^T       B: dXk
+            tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: (dP.D)^T Q + (bG)^T K
+            tmem_ld8(tmem + lane_base + 0 + cb, d8);      // A: U dh'^T
             tmem_wait_ld();
-            unpack8(kraw[part], kk);
-            // shared by both groups: A: dk^col = e (U dh'^T) + (dP.D)^T Q + (bG)^T K ; B: G K + Gam dXk; dotted with k
-            float t[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                t[j] = fmaf(s6, d8[j], c8[j]);
-                acc = fmaf(kk[j], t[j], acc);
-            }
             if (ga) {
+                unpack8(kraw[part], kk);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) a[j] = fmaf(bg6, b[j], a[j]) + t[j];       // dk = Diag(b)(G K + Gam dXk) + dk^col
+                for (int j = 0; j < 8; ++j) {
+                    const float kcol = fmaf(e6, d8[j], c8[j]);       // dk^col
+                    const float t = fmaf(G6, b[j], a[j]);            // G K + Gam dXk
+                    acc_col = fmaf(kk[j], kcol, acc_col);
+                    acc_db = fmaf(kk[j], t, acc_db);
+                    a[j] = fmaf(b6, t, kcol);
+                }
                 chunk_store(sm + STG_K, 64, tr, cb >> 3, a);
             }
         }
         }
-        red[ga ? 3 : 2][grp][tr] = acc;
+        if (ga) { red[2][grp][tr] = acc_db; red[3][grp][tr] = acc_col; }
     }
     GDN_TICK(2, 18);
     // block totals of sum_j r_j and <dh', h>
