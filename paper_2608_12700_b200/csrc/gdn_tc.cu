@@ -27,6 +27,7 @@ namespace gdn {
 __device__ long long g_ticks[4][32];
 __device__ int g_tick_trip = 0;   // which trip of a persistent CTA is stamped
 __device__ int g_trip_now = 0;
+__device__ long long g_sync[16][18];   // intra: arrival time of every warp at each named barrier of one trip, [17] = release
 __device__ long long g_trip_ns[2][24];   // wall-clock (ns) at kernel entry [0], at each trip start [1 + trip], at exit
 __device__ __forceinline__ long long tick_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define GDN_TRIP(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (idx) < 24) g_trip_ns[kern][idx] = tick_ns(); } while (0)
@@ -907,7 +908,17 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         return;
     }
 
+#ifdef GDN_PHASE_TIMING
+    int sync_no = 0;
+    auto cta_sync = [&] {
+        if (blockIdx.x == 0 && lane == 0 && g_trip_now == g_tick_trip && sync_no < 16) g_sync[sync_no][warp] = clock64();
+        asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory");
+        if (blockIdx.x == 0 && threadIdx.x == 0 && g_trip_now == g_tick_trip && sync_no < 16) g_sync[sync_no][17] = clock64();
+        ++sync_no;
+    };
+#else
     auto cta_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory"); };   // all warps but the loader
+#endif
     uint32_t mma_phase = 0, in_phase = 0;
     // chunk table entry and gates of a trip are fetched one trip ahead into registers (their latency would be exposed)
     ChunkInfo xn;
@@ -952,6 +963,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 #endif
     GDN_TICK(2, 0);
     GDN_TRIP(1, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
+#ifdef GDN_PHASE_TIMING
+    sync_no = 0;
+#endif
 
     if (threadIdx.x < kC) {
         const int i = threadIdx.x;
@@ -1529,6 +1543,9 @@ extern "C" int gdn_debug_tick_trip(int trip) {
 }
 extern "C" int gdn_debug_trips(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, gdn::g_trip_ns, sizeof(long long) * 2 * 24);
+}
+extern "C" int gdn_debug_syncs(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, gdn::g_sync, sizeof(long long) * 16 * 18);
 }
 extern "C" int gdn_debug_ticks(long long* out) {
     return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks, sizeof(long long) * 4 * 32);
