@@ -867,7 +867,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 }
                 // phase 5 is done
                 if (!(lok = mbar_wait(&bar_ld1, ph))) break;
-                if (has_next) {
+                // (Not in a CTA's first trip: there every CTA of the grid reaches this point at the same moment, the
+                // loads come as one burst of 25 MB, and the instruction fetches of the last phases, which run for the
+                // first time, queue behind it for microseconds.  The first trip loads at its end instead.)
+                const bool early = item != (int)blockIdx.x;
+                if (has_next && early) {
                     mbar_expect_tx(&bar_g1, G1_BYTES);
                     pend1 = true;
 #pragma unroll 1
@@ -878,7 +882,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 // read its source)
                 if (!(lok = mbar_wait(&bar_ld2, ph))) break;
                 if (!(lok = mbar_wait(&bar_kfree, ph))) break;
-                if (has_next) {
+                if (has_next && early) {
                     mbar_expect_tx(&bar_k, K_BYTES);
                     pend_k = true;
                     load_piece(0, nx);
@@ -897,6 +901,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 }
                 bulk_wait_read<0>();
                 mbar_arrive(&bar_free);   // the staging regions may be rewritten
+                if (has_next && !early) {
+                    mbar_expect_tx(&bar_k, K_BYTES);
+                    mbar_expect_tx(&bar_g1, G1_BYTES);
+                    mbar_expect_tx(&bar_g2, G2_BYTES);
+                    pend_k = pend1 = pend2 = true;
+#pragma unroll 1
+                    for (int piece = 0; piece <= 12; ++piece) load_piece(piece, nx);
+                }
             }
             bulk_wait_read<0>();
             if (!lok) {   // after a timeout a copy may still be in flight: wait for it before the CTA may retire

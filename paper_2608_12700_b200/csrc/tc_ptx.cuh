@@ -54,9 +54,10 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 // Bounded wait: gives up after about two seconds and returns false; the caller records the failure and
-// leaves through its normal teardown (no trap, no endless spin).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    // (rolled loops: a kernel has dozens of waits, and unrolled polling would multiply its code size)
+// leaves through its normal teardown (no trap, no endless spin).  Only the first probe is inlined at a wait site: a
+// kernel has dozens of them and the polling loop with its time-out would multiply the code size (the instruction
+// cache is cold at every launch and each CTA's first trip pays for every byte of code).
+static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
         if (mbar_try_wait(bar, parity)) return true;
@@ -67,6 +68,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
             if (mbar_try_wait(bar, parity)) return true;
         if (global_ns() - t0 > 2000000000ull) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    return mbar_try_wait(bar, parity) || mbar_wait_slow(bar, parity);
 }
 
 // ---------------------------------------------------------------- proxies and copies
