@@ -172,7 +172,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...; the inputs of its next one
     // are loaded while it works on the current one.
     const int H = p.d.H;
-    const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
+    init_header_if_untabled(p);
+    const int n_items = n_chunks_of(p) * H;
     if ((int)blockIdx.x >= n_items) return;
     const bool bwd = P.with_bwd != 0;
 
@@ -595,8 +596,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     const int reverse = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
     const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
     const int n = chain / p.d.H, hd = chain % p.d.H;
-    const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
-    const int c0 = seq_first[n], c1 = seq_first[n + 1], nsteps = c1 - c0;
+    const int c0 = seq_first_chunk(p, n), c1 = seq_first_chunk(p, n + 1), nsteps = c1 - c0;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
@@ -778,7 +778,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
     // tiles of its next one are loaded into the regions the current one has finished with.
     const int H = p.d.H;
-    const int n_items = reinterpret_cast<const WsHeader*>(p.ws)->n_chunks * H;
+    const int n_items = n_chunks_of(p) * H;
     if ((int)blockIdx.x >= n_items) return;
     const float sc = p.d.scale;
 
@@ -1523,9 +1523,14 @@ static cudaError_t empty_call(const Problem& p, bool bwd, cudaStream_t st) {
     return src ? cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) : cudaMemsetAsync(dst, 0, bytes, st);
 }
 
+// The chunk table is needed for packed sequences only (and for an empty call, whose only kernel it is).
+static cudaError_t launch_table_if_needed(const Problem& p, cudaStream_t st) {
+    return (p.cu || p.Ttot == 0) ? launch_table(p, st) : cudaSuccess;
+}
+
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st) {
     TcParams P;
-    cudaError_t e = launch_table(p, st);
+    cudaError_t e = launch_table_if_needed(p, st);
     if (e != cudaSuccess) return e;
     if (p.Ttot == 0) return empty_call(p, false, st);
     if (!fill_params(P, p, false, 0)) return cudaErrorUnknown;
@@ -1538,7 +1543,7 @@ cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st) {
 // rebuilt together with E, which needs dO.
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st) {
     TcParams P;
-    cudaError_t e = launch_table(p, st);
+    cudaError_t e = launch_table_if_needed(p, st);
     if (e != cudaSuccess) return e;
     if (p.Ttot == 0) return empty_call(p, true, st);
     if (!fill_params(P, p, true, skip_recompute ? 1 : 2)) return cudaErrorUnknown;

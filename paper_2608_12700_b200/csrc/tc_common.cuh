@@ -119,26 +119,46 @@ __device__ __forceinline__ void write_dg_suffix(const float* v0, const float* v1
     if (lane + 32 < len) dg[(size_t)(lane + 32) * stride] = b;
 }
 
+// Chunk geometry.  With packed sequences (cu_seqlens given) it is read from the table the table kernel wrote into the
+// workspace; with equal-length sequences it is plain arithmetic and that kernel is not launched at all (the first
+// kernel of the call initialises the header instead, see init_header_if_untabled).
 struct ChunkInfo { int c, hd, ch, tok0, len; };
-__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int item) {
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    x.c = item / p.d.H;
-    x.hd = item % p.d.H;
-    if (x.c >= hdr->n_chunks) return false;
-    x.ch = item;
-    x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
-    x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
-    return true;
+__device__ __forceinline__ int chunks_per_sequence(const Problem& p) { return (p.d.T + kC - 1) / kC; }
+__device__ __forceinline__ int n_chunks_of(const Problem& p) {
+    return p.cu ? reinterpret_cast<const WsHeader*>(p.ws)->n_chunks : p.d.N * chunks_per_sequence(p);
 }
-__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) { return chunk_info(p, x, (int)blockIdx.x); }
-// Same for an item already known to exist: no header read and no branch, so the two table loads can stay in flight
-// until their values are used (the persistent kernels fetch the entry one trip ahead).
+__device__ __forceinline__ int seq_first_chunk(const Problem& p, int n) {
+    return p.cu ? reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first)[n] : n * chunks_per_sequence(p);
+}
+// Entry of an item known to exist: no header read and no branch on loaded data, so the two table loads can stay in
+// flight until their values are used (the persistent kernels fetch the entry one trip ahead).
 __device__ __forceinline__ void chunk_entry(const Problem& p, ChunkInfo& x, int item) {
     x.c = item / p.d.H;
     x.hd = item % p.d.H;
     x.ch = item;
-    x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
-    x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
+    if (p.cu) {
+        x.tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[x.c];
+        x.len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[x.c];
+    } else {
+        const int cps = chunks_per_sequence(p), n = x.c / cps, pos = x.c - n * cps;
+        x.tok0 = n * p.d.T + pos * kC;
+        x.len = min(kC, p.d.T - pos * kC);
+    }
+}
+__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int item) {
+    if (item / p.d.H >= n_chunks_of(p)) return false;
+    chunk_entry(p, x, item);
+    return true;
+}
+__device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x) { return chunk_info(p, x, (int)blockIdx.x); }
+// Called at the top of the first kernel of a call: without the table kernel somebody has to reset the status word.
+__device__ __forceinline__ void init_header_if_untabled(const Problem& p) {
+    if (!p.cu && blockIdx.x == 0 && threadIdx.x == 0) {
+        WsHeader* hdr = reinterpret_cast<WsHeader*>(p.ws);
+        hdr->status = GDN_OK;
+        hdr->n_chunks = n_chunks_of(p);
+        hdr->detail = 0;
+    }
 }
 
 // Wait for the MMAs committed to `bar`; on a timeout record it once.
