@@ -31,8 +31,13 @@ __device__ long long g_sync[16][18];   // intra: arrival time of every warp at e
 __device__ long long g_trip_ns[2][24];   // wall-clock (ns) at kernel entry [0], at each trip start [1 + trip], at exit
 __device__ __forceinline__ long long tick_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define GDN_TRIP(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (idx) < 24) g_trip_ns[kern][idx] = tick_ns(); } while (0)
+#ifdef GDN_NO_TICKS   // barrier arrival times only: the phase stamps would delay thread 0
+#define GDN_TICK(kern, idx) do { } while (0)
+#define GDN_TICKT(tid, kern, idx) do { } while (0)
+#else
 #define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (kern != 2 || g_trip_now == g_tick_trip)) g_ticks[kern][idx] = clock64(); } while (0)
 #define GDN_TICKT(tid, kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == (tid)) g_ticks[kern][idx] = clock64(); } while (0)
+#endif
 #else
 #define GDN_TICK(kern, idx) do { } while (0)
 #define GDN_TICKT(tid, kern, idx) do { } while (0)
@@ -179,7 +184,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ __align__(16) float gam[kC], gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC], bgam[kC];
+    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC], bgam[kC];
     __shared__ uint64_t bar_qk, bar_vo, bar_ld0, bar_t, bar_vofree, bar_ld1, bar_st, bar_tfree, bar_free1, bar_free, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -340,7 +345,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         for (int h = 0; h < 2; ++h) {
             const int i = lane + 32 * h;
             const float G = expf(gc[h]);
-            gam[i] = gc[h];
             gl[i] = gc[h] * kLog2e;
             Gam[i] = G;
             bb[i] = b_now[h]; ww[i] = b_now[h];

@@ -363,7 +363,6 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
     for (int s = 0; s < nsteps; ++s) {
         const int c = c1 - 1 - s, stage = s % STAGES, len = len_n, tok0 = tok0_n;
         if (s + 1 < nsteps) { len_n = chunk_len[c - 1]; tok0_n = chunk_tok0[c - 1]; }
-        const size_t ch = (size_t)c * H + hd;
         unsigned char* tiles = sm + stage * STAGE_BYTES;
         const float *gl = gl2[s & 1], *Gam = Gam2[s & 1], *ee = ee2[s & 1];
         T64(0);
