@@ -1,4 +1,7 @@
 """GPU parity: the CUDA path (through the C ABI) against the CPU fp64 oracle on the same seeded inputs."""
+import json
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -213,3 +216,7 @@ def test_full_size_configs_sampled_chains(idx, heads):
     print(wl.name, errs)
     for n, v in got.items():
         assert np.isfinite(v).all(), n
+    # the acceptance bound the paper sets for its own assembled bf16 backward against its fp64 oracle (Section 4.5)
+    with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "paper_figures.json")) as f:
+        bound = json.load(f)["assembled_backward_acceptance_bound"]["value"]
+    assert max(errs.values()) <= bound, errs
