@@ -1034,12 +1034,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const int mi = q4 * 16 + lane;     // row of an M = 64 accumulator held by this lane (lanes 0..15 only)
     const int j0 = grp * kTG;
     if (ok && worker) {   // P_ij = (q_i . k_j) D_ij for j <= i
-#pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
-            float v[8];
+        float v2[2][8];
+        tmem_ld8(tmem + lane_base + slot(0) + j0, v2[0]);
+        tmem_ld8(tmem + lane_base + slot(0) + j0 + 8, v2[1]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            float (&v)[8] = v2[part];
             const int jb = j0 + part * 8;
-            tmem_ld8(tmem + lane_base + slot(0) + jb, v);
-            tmem_wait_ld();
             if (lane < 16) {
                 float g8[8];
                 ld8s(gl + jb, g8);
@@ -1080,17 +1082,21 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const int i0 = grp * kTG;          // first of this thread's 32 tokens
     float rs = 0.f;
     if (ok && worker) {
-#pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
+        float t2[2][8], kb2[2][8], pd2[2][8];
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            tmem_ld8(tmem + lane_base + slot(1) + i0 + part * 8, t2[part]);
+            tmem_ld8(tmem + lane_base + slot(2) + i0 + part * 8, kb2[part]);
+            tmem_ld8(tmem + lane_base + slot(3) + i0 + part * 8, pd2[part]);
+        }
+        tmem_wait_ld();
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
             const int ib = i0 + part * 8;
-            float u[8], t[8], kb[8], pd[8];
+            float u[8], e8[8];
+            float (&t)[8] = t2[part], (&kb)[8] = kb2[part], (&pd)[8] = pd2[part];
             chunk_load(sm + UTT, 128, f, ib >> 3, u);
-            tmem_ld8(tmem + lane_base + slot(1) + ib, t);
-            tmem_ld8(tmem + lane_base + slot(2) + ib, kb);
-            tmem_ld8(tmem + lane_base + slot(3) + ib, pd);
-            float e8[8];
             ld8s(ee + ib, e8);
-            tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 u[i] -= t[i];                                       // U = U~ - W h
@@ -1131,14 +1137,18 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     }
     GDN_TICK(2, 7);
     GDN_WAIT_MMA(23)
-    if (ok && worker) {
-#pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
-            float v[8], w[8];
+    if (ok && worker) {   // (all accumulator loads of the readout are issued before the one wait)
+        float v2[2][8], w2[2][8];
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            tmem_ld8(tmem + lane_base + 0 + j0b + part * 8, v2[part]);       // group B: dO U^T
+            tmem_ld8(tmem + lane_base + 256 + i0 + part * 8, w2[part]);      // all lanes: dW^T
+        }
+        tmem_wait_ld();
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
             const int jb = j0b + part * 8, ib = i0 + part * 8;
-            tmem_ld8(tmem + lane_base + 0 + jb, v);       // group B: dO U^T
-            tmem_ld8(tmem + lane_base + 256 + ib, w);     // all lanes: dW^T
-            tmem_wait_ld();
+            float (&v)[8] = v2[part];
             if (!ga) {   // dPD = scale tril(dO U^T) . D
                 float g8[8];
                 ld8s(gl + jb, g8);
@@ -1146,7 +1156,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? sc * v[j] * ex2(gl[tr] - g8[j]) : 0.f;
                 chunk_store(sm + DPD, 64, tr, jb >> 3, v);
             }
-            chunk_store(sm + DWT, 128, f, ib >> 3, w);              // dW^T = -(dU h^T)^T
+            chunk_store(sm + DWT, 128, f, ib >> 3, w2[part]);       // dW^T = -(dU h^T)^T
         }
     }
     tc_fence_before();
@@ -1230,12 +1240,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
     if (ok && worker) {
-#pragma unroll 1
-        for (int part = 0; part < kTG / 8; ++part) {
-            float v[8], w[8];
+        float v2[2][8];
+        tmem_ld8(tmem + lane_base + 384 + j0b, v2[0]);
+        tmem_ld8(tmem + lane_base + 384 + j0b + 8, v2[1]);
+        tmem_wait_ld();
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            float (&v)[8] = v2[part];
+            float w[8];
             const int jb = j0b + part * 8;
-            tmem_ld8(tmem + lane_base + 384 + jb, v);
-            tmem_wait_ld();
             if (!ga) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
                 float g8[8];
                 ld8s(gl + jb, g8);
