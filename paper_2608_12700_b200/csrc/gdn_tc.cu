@@ -425,10 +425,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     GDN_TICK(0, 16);
     inv_premul(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
     cta_sync();
-    inv_level<1, 2>(Sf, Tf);
+    inv_level<1, 1>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 17);
-    inv_level<2, 4>(Sf, Tf);
+    inv_level<2, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 18);
     inv_level<3, 4>(Sf, Tf);
