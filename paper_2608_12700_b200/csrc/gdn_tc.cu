@@ -791,7 +791,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC];
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
-    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma;
+    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
@@ -811,7 +811,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mbar_init(&bar_k, 1); mbar_init(&bar_g1, 1); mbar_init(&bar_g2, 1);
         mbar_init(&bar_ld0, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_ld2, 1);
         mbar_init(&bar_st1, 1); mbar_init(&bar_st2, 1); mbar_init(&bar_kfree, 16); mbar_init(&bar_free, 1);
-        mbar_init(&bar_mma, 1);
+        mbar_init(&bar_mma, 1); mbar_init(&bar_mma2, 1);
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
@@ -1132,32 +1132,44 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + 0 + LB, op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);           // dO U^T
+        mma_commit(&bar_mma);   // dPD is formed while dW^T is still being multiplied
         mma_tile<128, 64, 128>(tmem + 256, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
-        mma_commit(&bar_mma);   // (also covers dO h^T of phase 2: the readout overwrites the dO tile, which it reads)
+        // (a barrier of its own: two commits in a row on one mbarrier could complete two of its phases before a waiter
+        // has looked, and a parity wait cannot tell a phase from the one two later)
+        mma_commit(&bar_mma2);
     }
     GDN_TICK(2, 7);
     GDN_WAIT_MMA(23)
-    if (ok && worker) {   // (all accumulator loads of the readout are issued before the one wait)
-        float v2[2][8], w2[2][8];
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            tmem_ld8(tmem + lane_base + 0 + j0b + part * 8, v2[part]);       // group B: dO U^T
-            tmem_ld8(tmem + lane_base + 256 + i0 + part * 8, w2[part]);      // all lanes: dW^T
-        }
+    if (ok && worker) {   // dPD = scale tril(dO U^T) . D  (group B; the accumulator loads are warp-wide instructions)
+        float v2[2][8];
+        tmem_ld8(tmem + lane_base + 0 + j0b, v2[0]);
+        tmem_ld8(tmem + lane_base + 0 + j0b + 8, v2[1]);
         tmem_wait_ld();
+        if (!ga) {
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            const int jb = j0b + part * 8, ib = i0 + part * 8;
-            float (&v)[8] = v2[part];
-            if (!ga) {   // dPD = scale tril(dO U^T) . D
+            for (int part = 0; part < 2; ++part) {
+                const int jb = j0b + part * 8;
+                float (&v)[8] = v2[part];
                 float g8[8];
                 ld8s(gl + jb, g8);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? sc * v[j] * ex2(gl[tr] - g8[j]) : 0.f;
                 chunk_store(sm + DPD, 64, tr, jb >> 3, v);
             }
-            chunk_store(sm + DWT, 128, f, ib >> 3, w2[part]);       // dW^T = -(dU h^T)^T
         }
+    }
+    if (ok) {   // dW^T is complete (and with it dO h^T of phase 2, which reads the dO tile that dW^T now overwrites)
+        ok = mbar_wait(&bar_mma2, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 29);
+    }
+    tc_fence_after();
+    if (ok && worker) {
+        float w2[2][8];
+        tmem_ld8(tmem + lane_base + 256 + i0, w2[0]);
+        tmem_ld8(tmem + lane_base + 256 + i0 + 8, w2[1]);
+        tmem_wait_ld();
+        chunk_store(sm + DWT, 128, f, i0 >> 3, w2[0]);              // dW^T = -(dU h^T)^T
+        chunk_store(sm + DWT, 128, f, (i0 >> 3) + 1, w2[1]);
     }
     tc_fence_before();
     fence_async_smem();
