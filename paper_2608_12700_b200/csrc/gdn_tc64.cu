@@ -68,7 +68,7 @@ namespace f64 {
 constexpr int STAGES = 2;
 constexpr uint32_t KT = 0, VT = 8192, QT = 16384, STAGE_BYTES = 24576;   // per stage: K, V (and Q when o is wanted)
 constexpr uint32_t VE = STAGES * STAGE_BYTES;   // Diag(e) V
-constexpr uint32_t HT = VE + 8192;              // bf16 state tile (only when o is wanted)
+constexpr uint32_t HT = VE + 8192;              // bf16 state tile: leaves for the workspace by a bulk store; operand of Q h
 constexpr uint32_t PT = HT + 8192;              // P (only when o is wanted)
 constexpr uint32_t SMEM_BYTES = PT + 8192 + 1024;
 }  // namespace f64
@@ -131,11 +131,14 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
     float gnext = (threadIdx.x < kC && nsteps > 0) ? gamma[((size_t)c0 * H + hd) * kC + threadIdx.x] : 0.f;
     bool ok = true;
     uint32_t mma_phase = 0;
+    int len_n = nsteps > 0 ? chunk_len[c0] : 0;   // fetched a step ahead
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
-        const int c = c0 + s, stage = s % STAGES, len = chunk_len[c];
+        const int c = c0 + s, stage = s % STAGES, len = len_n;
+        if (s + 1 < nsteps) len_n = chunk_len[c + 1];
         const size_t ch = (size_t)c * H + hd;
         unsigned char* tiles = sm + stage * STAGE_BYTES;
+        if (threadIdx.x == 32) bulk_wait_read<0>();   // the previous step's state tile has left shared memory
         if (threadIdx.x < kC) {
             gl[threadIdx.x] = gnext * kLog2e;
             Gam[threadIdx.x] = expf(gnext);
@@ -160,18 +163,17 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
             for (int k = 0; k < 8; ++k) v[k] *= ee[i];
             chunk_store(sm + VE, 64, i, cch, v);
         }
-        if (act) {   // state entering the chunk -> workspace (and, for o, the MMA operand tile)
-            char* keep = p.ws + p.L.hc + ch * 8192;
+        if (act) {   // state entering the chunk -> bf16 tile: the workspace copy (and, for o, the MMA operand)
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const uint4 u = pack8(st + 8 * k);
-                const uint32_t off = tile_chunk_off(64, r, (cb0 >> 3) + k);
-                *reinterpret_cast<uint4*>(keep + off) = u;
-                if (want_o) *reinterpret_cast<uint4*>(sm + HT + off) = u;
-            }
+            for (int k = 0; k < 4; ++k)
+                *reinterpret_cast<uint4*>(sm + HT + tile_chunk_off(64, r, (cb0 >> 3) + k)) = pack8(st + 8 * k);
         }
         fence_async_smem();
         __syncthreads();
+        if (threadIdx.x == 32) {   // the tile leaves through the async proxy (generic global stores would stall the next proxy fence)
+            bulk_store(p.ws + p.L.hc + ch * 8192, sm + HT, 8192);
+            bulk_commit();
+        }
         if (threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 64, 64>(tmem + 0, op_mn_major(tiles + KT, 64), op_mn_major(sm + VE, 64), false);              // Kb^T V
@@ -183,6 +185,8 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
         }
         GDN_WAIT_MMA(41)
         if (!ok) break;
+        // without o the stage's K and V have now been read for the last time: refill it while the state is updated
+        if (!want_o && threadIdx.x == 32 && s + STAGES < nsteps) fill(s + STAGES);
         if (want_o) {   // o = scale (Gam_i (Q h)_i + (P V)_i)
 #pragma unroll 1
             for (int part = 0; part < 4; ++part) {
@@ -230,9 +234,12 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
             for (int j = 0; j < 8; ++j) st[8 * k + j] = fmaf(Ge, st[8 * k + j], bf[j]);
         }
         tc_fence_before();
-        __syncthreads();   // every reader of this stage's tiles is done
-        if (threadIdx.x == 0 && s + STAGES < nsteps) fill(s + STAGES);
+        if (want_o) {
+            __syncthreads();   // every reader of this stage's tiles is done
+            if (threadIdx.x == 0 && s + STAGES < nsteps) fill(s + STAGES);
+        }
     }
+    if (threadIdx.x == 32) bulk_wait_read<0>();
     if (p.hT && ok && act) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) *reinterpret_cast<float4*>(p.hT + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
