@@ -97,6 +97,22 @@ struct StageScope {
     ~StageScope() { stage_end(s, st); }
 };
 
+// Raising a kernel's dynamic shared-memory limit is a per-device function attribute: remember, per kernel, on which
+// devices it has been done (a process may drive several GPUs).
+struct SmemLimitOnce {
+    bool done[64] = {};
+    template <class Kernel>
+    cudaError_t ensure(Kernel kernel, uint32_t bytes) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64 && done[dev]) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e == cudaSuccess && dev >= 0 && dev < 64) done[dev] = true;
+        return e;
+    }
+};
+
 // Kernel families (each defined in its own translation unit).  They enqueue on `st` and return the
 // first CUDA error seen.
 cudaError_t launch_table(const Problem& p, cudaStream_t st);

@@ -1492,13 +1492,10 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
 }
 
 template <class Kernel>
-static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t smem, Stage stage, int grid, int threads,
+static cudaError_t launch_chunk_kernel(Kernel kernel, SmemLimitOnce& once, uint32_t smem, Stage stage, int grid, int threads,
                                        const TcParams& P, cudaStream_t st) {
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    const cudaError_t e = once.ensure(kernel, smem);
+    if (e != cudaSuccess) return e;
     if (grid > 0) {
         StageScope t(stage, st);
         kernel<<<grid, threads, smem, st>>>(P);
@@ -1508,7 +1505,7 @@ static cudaError_t launch_chunk_kernel(Kernel kernel, bool& attr_done, uint32_t 
 
 static int sm_count();
 static cudaError_t launch_prep(const TcParams& P, cudaStream_t st) {
-    static bool done = false;
+    static SmemLimitOnce done;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
     return launch_chunk_kernel(tc_prep_kernel, done, prep::SMEM_BYTES, ST_PREP, items < sms ? items : sms, kIntraThreads + 32, P, st);
 }
@@ -1525,8 +1522,8 @@ static int sm_count() {
 }
 
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
-    static bool done = false;
-    static bool done2 = false;
+    static SmemLimitOnce done;
+    static SmemLimitOnce done2;
     const int ctas = P.p.d.N * P.p.d.H * (P.scan_dirs == 2 ? 2 : 1);
     // few chains: two CTAs per (chain, direction), each carrying half of the state columns
     if (2 * ctas <= sm_count())
@@ -1534,12 +1531,12 @@ static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     return launch_chunk_kernel(tc_scan_kernel<1>, done, scan::Cfg<1>::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
 }
 static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
-    static bool done = false;
+    static SmemLimitOnce done;
     const int items = P.p.L.max_chunks * P.p.d.H, sms = sm_count();
     return launch_chunk_kernel(tc_intra_kernel, done, intra::SMEM_BYTES, ST_INTRA, items < sms ? items : sms, kIntraThreads + 32, P, st);
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
-    static bool done = false;
+    static SmemLimitOnce done;
     return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, kThreads, P, st);
 }
 

@@ -588,12 +588,9 @@ static cudaError_t tc64_prologue(const Problem& p, cudaStream_t st) {
 }
 
 static cudaError_t tc64_fwd_pass(const Tc64Params& P, cudaStream_t st) {
-    static bool done = false;
-    if (!done) {
-        cudaError_t e = cudaFuncSetAttribute(tc64_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f64::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        done = true;
-    }
+    static SmemLimitOnce once;
+    const cudaError_t e0 = once.ensure(tc64_fwd_kernel, f64::SMEM_BYTES);
+    if (e0 != cudaSuccess) return e0;
     const int chains = P.p.d.N * P.p.d.H;
     if (chains > 0) {
         StageScope t(ST_FSCAN, st);
@@ -631,12 +628,8 @@ cudaError_t tc64_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t 
         F.p.hT = nullptr;
         if ((e = tc64_fwd_pass(F, st)) != cudaSuccess) return e;
     }
-    static bool done = false;
-    if (!done) {
-        e = cudaFuncSetAttribute(tc64_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)b64::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        done = true;
-    }
+    static SmemLimitOnce once;
+    if ((e = once.ensure(tc64_bwd_kernel, b64::SMEM_BYTES)) != cudaSuccess) return e;
     const int chains = p.d.N * p.d.H;
     if (chains > 0) {
         StageScope t(ST_RSCAN, st);
