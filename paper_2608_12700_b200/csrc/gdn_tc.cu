@@ -101,45 +101,64 @@ __device__ __forceinline__ void inv_diag16(const float* Af, float* Tf, float* Xf
         Tf[(r0 + i) * kLdi + r0 + 8 + j] = 0.f;    // the block above the diagonal
     }
 }
+// R rows of a block per thread: the 16-byte load of a row of A feeds R x 4 FMAs (these steps are bound by the number of
+// shared-memory wavefronts, and a 16-byte load costs a warp four of them however many lanes share an address).
+template <int R>
 __device__ __forceinline__ void inv_premul(const float* Af, const float* Tf, float* Sf) {
-    // six blocks below the diagonal: (1,0) (2,0) (2,1) (3,0) (3,1) (3,2)
-    for (int o = threadIdx.x; o < 6 * 64; o += kIntraThreads) {
-        const int blk = o >> 6, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
+    // six blocks below the diagonal: (1,0) (2,0) (2,1) (3,0) (3,1) (3,2); per block 16 / R row groups x 4 column groups
+    constexpr int per_blk = (16 / R) * 4;
+    if (threadIdx.x < 6 * per_blk) {
+        const int o = threadIdx.x, blk = o / per_blk, ig = (o % per_blk) >> 2, j4 = (o & 3) * 4;
         const int rb = (blk == 0 ? 1 : blk < 3 ? 2 : 3) * 16, cb = (blk == 0 ? 0 : blk < 3 ? blk - 1 : blk - 3) * 16;
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 s[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) s[q] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int m = 0; m < 16; ++m) {   // T_rr is lower triangular: zeros above the diagonal
-            const float a = Tf[(rb + ii) * kLdi + rb + m];
             const float4 v = *reinterpret_cast<const float4*>(Af + (rb + m) * kLdi + cb + j4);
-            s.x = fmaf(a, v.x, s.x); s.y = fmaf(a, v.y, s.y); s.z = fmaf(a, v.z, s.z); s.w = fmaf(a, v.w, s.w);
+#pragma unroll
+            for (int q = 0; q < R; ++q) {   // rows ig, ig + 16 / R, ...: a warp's scalar loads fall into distinct banks
+                const float a = Tf[(rb + ig + q * (16 / R)) * kLdi + rb + m];
+                s[q].x = fmaf(a, v.x, s[q].x); s[q].y = fmaf(a, v.y, s[q].y); s[q].z = fmaf(a, v.z, s[q].z); s[q].w = fmaf(a, v.w, s[q].w);
+            }
         }
-        *reinterpret_cast<float4*>(Sf + (rb + ii) * kLdi + cb + j4) = s;
+#pragma unroll
+        for (int q = 0; q < R; ++q) *reinterpret_cast<float4*>(Sf + (rb + ig + q * (16 / R)) * kLdi + cb + j4) = s[q];
     }
 }
-template <int DIST, int SPLIT>
+template <int DIST, int SPLIT, int R>
 __device__ __forceinline__ void inv_level(const float* At, float* Tf) {
-    constexpr int items = (4 - DIST) * 64, len = 16 * DIST / SPLIT;
+    constexpr int items = (4 - DIST) * (16 / R) * 4, len = 16 * DIST / SPLIT;
     static_assert(items * SPLIT <= kWideThreads && (items * SPLIT) % 32 == 0, "one pass, whole warps");
     if (threadIdx.x < items * SPLIT) {
         // a warp serves 32 / SPLIT items; the lanes of a quarter-warp share `part`, so their 16-byte loads fall into one
         // row of T (no bank conflicts), and the partial sums of an item sit 32 / SPLIT lanes apart
-        constexpr int G = 32 / SPLIT;
+        constexpr int G = 32 / SPLIT, per_blk = (16 / R) * 4;
         const int wl = threadIdx.x & 31, o = (threadIdx.x >> 5) * G + (wl % G), part = wl / G;
-        const int cb = (o >> 6) * 16, rb = cb + DIST * 16, ii = (o >> 2) & 15, j4 = (o & 3) * 4;
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int cb = (o / per_blk) * 16, rb = cb + DIST * 16, ig = (o % per_blk) >> 2, j4 = (o & 3) * 4;
+        float4 s[R];
+#pragma unroll
+        for (int q = 0; q < R; ++q) s[q] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int mm = 0; mm < len; ++mm) {
             const int m = part * len + mm;
-            const float a = At[(rb + ii) * kLdi + cb + m];
             const float4 v = *reinterpret_cast<const float4*>(Tf + (cb + m) * kLdi + cb + j4);
-            s.x = fmaf(a, v.x, s.x); s.y = fmaf(a, v.y, s.y); s.z = fmaf(a, v.z, s.z); s.w = fmaf(a, v.w, s.w);
+#pragma unroll
+            for (int q = 0; q < R; ++q) {
+                const float a = At[(rb + ig + q * (16 / R)) * kLdi + cb + m];
+                s[q].x = fmaf(a, v.x, s[q].x); s[q].y = fmaf(a, v.y, s[q].y); s[q].z = fmaf(a, v.z, s[q].z); s[q].w = fmaf(a, v.w, s[q].w);
+            }
         }
 #pragma unroll
-        for (int d = G; d < 32; d <<= 1) {
-            s.x += __shfl_xor_sync(0xffffffffu, s.x, d); s.y += __shfl_xor_sync(0xffffffffu, s.y, d);
-            s.z += __shfl_xor_sync(0xffffffffu, s.z, d); s.w += __shfl_xor_sync(0xffffffffu, s.w, d);
+        for (int q = 0; q < R; ++q) {
+#pragma unroll
+            for (int d = G; d < 32; d <<= 1) {
+                s[q].x += __shfl_xor_sync(0xffffffffu, s[q].x, d); s[q].y += __shfl_xor_sync(0xffffffffu, s[q].y, d);
+                s[q].z += __shfl_xor_sync(0xffffffffu, s[q].z, d); s[q].w += __shfl_xor_sync(0xffffffffu, s[q].w, d);
+            }
+            if (part == 0)
+                *reinterpret_cast<float4*>(Tf + (rb + ig + q * (16 / R)) * kLdi + cb + j4) = make_float4(-s[q].x, -s[q].y, -s[q].z, -s[q].w);
         }
-        if (part == 0) *reinterpret_cast<float4*>(Tf + (rb + ii) * kLdi + cb + j4) = make_float4(-s.x, -s.y, -s.z, -s.w);
     }
 }
 
@@ -423,15 +442,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     inv_diag16(Af, Tf, Sf);
     cta_sync();
     GDN_TICK(0, 16);
-    inv_premul(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
+    inv_premul<2>(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
     cta_sync();
-    inv_level<1, 1>(Sf, Tf);
+    inv_level<1, 1, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 17);
-    inv_level<2, 2>(Sf, Tf);
+    inv_level<2, 2, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 18);
-    inv_level<3, 4>(Sf, Tf);
+    inv_level<3, 4, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 4);
     for (int t = threadIdx.x; t < kC * 8; t += kIntraThreads) {
