@@ -425,7 +425,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 float g8[8];
                 ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) Af[i * kLdi + jb + j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - g8[j]) : 0.f;
+                for (int j = 0; j < 8; ++j) v[j] = (jb + j < i) ? bb[i] * v[j] * ex2(gl[i] - g8[j]) : 0.f;
+                *reinterpret_cast<float4*>(Af + i * kLdi + jb) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4*>(Af + i * kLdi + jb + 4) = make_float4(v[4], v[5], v[6], v[7]);
             }
         }
     }
