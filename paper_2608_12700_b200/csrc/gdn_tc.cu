@@ -455,25 +455,30 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     inv_level<3, 4, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 4);
-    for (int t = threadIdx.x; t < kC * 8; t += kIntraThreads) {
-        const int i = t >> 3, cch = t & 7;
-        float a[8], b[8], w8[8];
-        if ((cch >> 1) <= (i >> 4)) {   // the blocks above the block diagonal are zero and were never written
-            *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8);
-            *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8 + 4);
-        } else {
+    if (threadIdx.x < kC * 4) {   // T -> bf16 tiles T, T Diag(b Gam), T Diag(w): a thread scales two rows of one 8-column piece
+        const int cch = threadIdx.x & 7;
+        float gb[8], gw[8];
+        *reinterpret_cast<float4*>(gb) = *reinterpret_cast<const float4*>(bgam + cch * 8);
+        *reinterpret_cast<float4*>(gb + 4) = *reinterpret_cast<const float4*>(bgam + cch * 8 + 4);
+        *reinterpret_cast<float4*>(gw) = *reinterpret_cast<const float4*>(ww + cch * 8);
+        *reinterpret_cast<float4*>(gw + 4) = *reinterpret_cast<const float4*>(ww + cch * 8 + 4);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) a[k] = 0.f;
+        for (int h = 0; h < 2; ++h) {
+            const int i = (threadIdx.x >> 3) + 32 * h;
+            float a[8], b[8], w8[8];
+            if ((cch >> 1) <= (i >> 4)) {   // the blocks above the block diagonal are zero and were never written
+                *reinterpret_cast<float4*>(a) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8);
+                *reinterpret_cast<float4*>(a + 4) = *reinterpret_cast<const float4*>(Tf + i * kLdi + cch * 8 + 4);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) a[k] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { b[k] = gb[k] * a[k]; w8[k] = gw[k] * a[k]; }
+            chunk_store(sm + TT, 64, i, cch, a);
+            chunk_store(sm + TP, 64, i, cch, b);
+            chunk_store(sm + TPP, 64, i, cch, w8);
         }
-        *reinterpret_cast<float4*>(b) = *reinterpret_cast<const float4*>(bgam + cch * 8);
-        *reinterpret_cast<float4*>(b + 4) = *reinterpret_cast<const float4*>(bgam + cch * 8 + 4);
-        *reinterpret_cast<float4*>(w8) = *reinterpret_cast<const float4*>(ww + cch * 8);
-        *reinterpret_cast<float4*>(w8 + 4) = *reinterpret_cast<const float4*>(ww + cch * 8 + 4);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { b[k] *= a[k]; w8[k] *= a[k]; }
-        chunk_store(sm + TT, 64, i, cch, a);
-        chunk_store(sm + TP, 64, i, cch, b);
-        chunk_store(sm + TPP, 64, i, cch, w8);
     }
     fence_async_smem();
     cta_sync();
