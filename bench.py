@@ -128,7 +128,11 @@ def run_ours(args):
     if st != binding.GDN_OK:
         raise binding.GdnError(st, "warm-up")
     sampler = benchutil.ClockSampler(local)
-    binding.gdn_stage_timing_enable(True)
+    # per-kernel durations are sampled inside the timed region: the kernels of every `period`-th step are bracketed
+    # by events (an event between two kernels costs the stream a few microseconds; bracketing every launch slows a
+    # 0.35 ms step by 5 %)
+    period = max(1, args.steps // 12)
+    binding.gdn_stage_timing_enable(period)
     binding.gdn_stage_timing_read()
     launches0 = binding.gdn_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -219,6 +223,7 @@ def run_ours(args):
                           "t_tensor_us": t_tc * 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
                           "frac": path_roof_s / (ms_per_step * 1e-3), "peak_source": peaks["source"]},
         "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()},
+        "stage_timed_steps": max(v[1] for v in stages.values()),
     }
     if not args.no_cpu_baseline and world == 1:
         v, cores, sample, used = time_oracle_sample(wl, args.cpu_seconds)

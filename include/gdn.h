@@ -144,8 +144,10 @@ gdn_status gdn_bwd_noalloc(const gdn_desc* desc,
 
 /* ---- measurement hooks (not part of the method; the paper has no counterpart) -------------------
  * gdn_launch_count: number of kernels this library has launched in this process.
- * gdn_stage_timing_enable(1): from now on every kernel launch is bracketed by a pair of CUDA events
- * recorded on the launching stream (events are created lazily and reused; no device memory).
+ * gdn_stage_timing_enable(n), n >= 1: from now on every kernel launch of every n-th call of gdn_fwd_recompute /
+ * gdn_bwd (the first one included) is bracketed by a pair of CUDA events recorded on the launching stream (events
+ * are created lazily and reused; no device memory).  An event between two kernels costs the stream a few
+ * microseconds, which is why a timed loop samples (n > 1) instead of bracketing every launch.  0 switches it off.
  * gdn_stage_timing_read: synchronises the recorded events, adds up per-stage durations since the last
  * read, writes up to max_stages entries (total_ms, launches, names: static strings) and resets the
  * record.  Returns the number of stages through *n_stages.  Not thread-safe; diagnostic use only. */

@@ -149,8 +149,9 @@ def gdn_launch_count() -> int:
     return int(lib().gdn_launch_count())
 
 
-def gdn_stage_timing_enable(on: bool) -> None:
-    lib().gdn_stage_timing_enable(1 if on else 0)
+def gdn_stage_timing_enable(on) -> None:
+    """False/0: off.  True/1: every call's kernels are bracketed by events.  n > 1: every n-th call's."""
+    lib().gdn_stage_timing_enable(int(on))
 
 
 def gdn_stage_timing_read():

@@ -12,7 +12,9 @@ namespace gdn {
 // ---- launch counting and optional per-stage event timing ----
 namespace {
 std::atomic<uint64_t> g_launches{0};
-bool g_timing = false;
+int g_period = 0;         // 0: no stage timing; n: the stages of every n-th call are bracketed by events
+uint64_t g_calls = 0;     // calls since timing was switched on
+bool g_timing = false;    // the stages of the call under way are timed
 struct Rec { Stage s; cudaEvent_t a, b; };
 std::vector<Rec> g_recs;          // recorded since the last read
 std::vector<cudaEvent_t> g_pool;  // reusable events
@@ -24,6 +26,7 @@ cudaEvent_t take_event() {
     cudaEventCreate(&e);
     return e;
 }
+void call_begin() { g_timing = g_period > 0 && (g_calls++ % (uint64_t)g_period) == 0; }
 }  // namespace
 
 void stage_begin(Stage, cudaStream_t st) {
@@ -103,6 +106,7 @@ gdn_status gdn_workspace_bytes(const gdn_desc* desc, size_t* fwd_bytes, size_t* 
 gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g,
                              const float* beta, const float* h0, const int32_t* cu, void* o, float* hT,
                              void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    call_begin();
     gdn_status s = check_desc(desc);
     if (s != GDN_OK) return s;
     if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
@@ -129,6 +133,7 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
                    const float* h0, const void* dO, const float* dhT, const int32_t* cu, void* dq, void* dk, void* dv,
                    float* dg, float* dbeta, float* dh0, void* workspace, size_t workspace_bytes,
                    int32_t workspace_is_fresh_from_fwd, void* cuda_stream) {
+    call_begin();
     gdn_status s = check_desc(desc);
     if (s != GDN_OK) return s;
     if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
@@ -228,7 +233,9 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
 uint64_t gdn_launch_count(void) { return g_launches.load(); }
 
 gdn_status gdn_stage_timing_enable(int32_t on) {
-    g_timing = on != 0;
+    g_period = on > 0 ? on : 0;
+    g_calls = 0;
+    g_timing = false;
     return GDN_OK;
 }
 
