@@ -34,26 +34,32 @@ struct Tc64Params {
     CUtensorMap tm_dq, tm_dk, tm_dv;       // same geometry, for the gradient stores of full chunks
 };
 
-// chunk-local cumulative log decay, one warp per chunk-head (lane l owns tokens l and l + 32)
-__global__ void tc64_gamma_kernel(Problem p) {
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    const int lane = threadIdx.x & 31;
-    const int ch = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int c = ch / p.d.H, hd = ch % p.d.H;
-    if (c >= hdr->n_chunks) return;
-    const int tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0)[c];
-    const int len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len)[c];
-    float a = lane < len ? p.g[(size_t)(tok0 + lane) * p.d.H + hd] : 0.f;
-    float b = lane + 32 < len ? p.g[(size_t)(tok0 + lane + 32) * p.d.H + hd] : 0.f;
+// Chunk-local cumulative log decay.  A block takes one chunk and 32 heads: the [64 tokens][32 heads] patch of g is
+// read token by token (128 contiguous bytes each), then each warp scans the tokens of four heads (lane l owns
+// tokens l and l + 32).  First kernel of a call.
+__global__ void __launch_bounds__(256) tc64_gamma_kernel(Problem p) {
+    init_header_if_untabled(p);
+    __shared__ float gs[kC][33];
+    const int c = blockIdx.x, h0 = blockIdx.y * 32, H = p.d.H;
+    if (c >= n_chunks_of(p)) return;
+    const ChunkGeom cg = chunk_geom(p);
+    const int tok0 = cg.chunk_tok0(c), len = cg.chunk_len(c);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = warp; i < kC; i += 8)
+        gs[i][lane] = (i < len && h0 + lane < H) ? p.g[(size_t)(tok0 + i) * H + h0 + lane] : 0.f;
+    __syncthreads();
+    for (int hh = warp; hh < 32 && h0 + hh < H; hh += 8) {
+        float a = gs[lane][hh], b = gs[lane + 32][hh];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
-        if (lane >= o) { a += ua; b += ub; }
+        for (int o = 1; o < 32; o <<= 1) {
+            const float ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
+            if (lane >= o) { a += ua; b += ub; }
+        }
+        b += __shfl_sync(0xffffffffu, a, 31);
+        float* out = reinterpret_cast<float*>(p.ws + p.L.gamma) + ((size_t)c * H + h0 + hh) * kC;
+        out[lane] = a;
+        out[lane + 32] = b;
     }
-    b += __shfl_sync(0xffffffffu, a, 31);
-    float* out = reinterpret_cast<float*>(p.ws + p.L.gamma) + (size_t)ch * kC;
-    out[lane] = a;
-    out[lane + 32] = b;
 }
 
 __device__ __forceinline__ void zero_tail_rows64(unsigned char* tile, int len) {   // [64][64] tile; threads 0 .. kThreads64-1
@@ -80,10 +86,8 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
     if (hdr->status != GDN_OK) return;
     const int H = p.d.H;
     const int n = blockIdx.x / H, hd = blockIdx.x % H;
-    const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
-    const int32_t* chunk_tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0);
-    const int32_t* chunk_len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len);
-    const int c0 = seq_first[n], nsteps = seq_first[n + 1] - c0;
+    const SeqGeom cg = seq_geom(p, n);
+    const int c0 = cg.c0, nsteps = cg.n_chunks;
     const bool want_o = p.o != nullptr;
 
     extern __shared__ unsigned char smem_raw[];
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
     const uint32_t tmem = tmem_slot;
 
     auto fill = [&](int s) {
-        const int stage = s % STAGES, tok0 = chunk_tok0[c0 + s];
+        const int stage = s % STAGES, tok0 = cg.chunk_tok0(c0 + s);
         unsigned char* st = sm + stage * STAGE_BYTES;
         mbar_expect_tx(&bar_full[stage], want_o ? 24576 : 16384);
         tma_load_2d(st + KT, &P.tm_k, hd * D6, tok0, &bar_full[stage]);
@@ -131,11 +135,11 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
     float gnext = (threadIdx.x < kC && nsteps > 0) ? gamma[((size_t)c0 * H + hd) * kC + threadIdx.x] : 0.f;
     bool ok = true;
     uint32_t mma_phase = 0;
-    int len_n = nsteps > 0 ? chunk_len[c0] : 0;   // fetched a step ahead
+    int len_n = nsteps > 0 ? cg.chunk_len(c0) : 0;   // fetched a step ahead
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
         const int c = c0 + s, stage = s % STAGES, len = len_n;
-        if (s + 1 < nsteps) len_n = chunk_len[c + 1];
+        if (s + 1 < nsteps) len_n = cg.chunk_len(c + 1);
         const size_t ch = (size_t)c * H + hd;
         unsigned char* tiles = sm + stage * STAGE_BYTES;
         if (threadIdx.x == 32) bulk_wait_read<0>();   // the previous step's state tile has left shared memory
@@ -212,7 +216,7 @@ __global__ void __launch_bounds__(kThreads64, 2) tc64_fwd_kernel(const __grid_co
             }
             GDN_WAIT_MMA(42)
             if (!ok) break;
-            __nv_bfloat16* go = reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)(chunk_tok0[c] + r) * H + hd) * D6;
+            __nv_bfloat16* go = reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)(cg.chunk_tok0(c) + r) * H + hd) * D6;
 #pragma unroll 1
             for (int part = 0; part < 4; ++part) {
                 float a[8], b[8];
@@ -274,10 +278,8 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
     if (hdr->status != GDN_OK) return;
     const int H = p.d.H;
     const int n = blockIdx.x / H, hd = blockIdx.x % H;
-    const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
-    const int32_t* chunk_tok0 = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0);
-    const int32_t* chunk_len = reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len);
-    const int c0 = seq_first[n], c1 = seq_first[n + 1], nsteps = c1 - c0;
+    const SeqGeom cg = seq_geom(p, n);
+    const int c0 = cg.c0, nsteps = cg.n_chunks, c1 = c0 + nsteps;
     const float sc = p.d.scale;
 
     extern __shared__ unsigned char smem_raw[];
@@ -309,7 +311,7 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
     const uint32_t tmem = tmem_slot;
 
     auto fill = [&](int s) {   // step s handles chunk c1 - 1 - s
-        const int stage = s % STAGES, c = c1 - 1 - s, tok0 = chunk_tok0[c];
+        const int stage = s % STAGES, c = c1 - 1 - s, tok0 = cg.chunk_tok0(c);
         unsigned char* st = sm + stage * STAGE_BYTES;
         mbar_expect_tx(&bar_full[stage], 40960);
         tma_load_2d(st + QT, &P.tm_q, hd * D6, tok0, &bar_full[stage]);
@@ -325,8 +327,8 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
             for (int s = 0; s < nsteps; ++s) {
                 if (!mbar_wait(&bar_st, s & 1)) break;          // step s has staged its gradient rows (or flushed them)
                 const int c = c1 - 1 - s;
-                if (chunk_len[c] == kC) {
-                    const int tok0 = chunk_tok0[c];
+                if (cg.chunk_len(c) == kC) {
+                    const int tok0 = cg.chunk_tok0(c);
                     unsigned char* st = sm + (s % STAGES) * STAGE_BYTES;
                     tma_store_2d(&P.tm_dv, hd * D6, tok0, st + VT);
                     tma_store_2d(&P.tm_dk, hd * D6, tok0, st + KT);
@@ -365,11 +367,11 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
     }
     bool ok = true;
     uint32_t mma_phase = 0;
-    int len_n = nsteps > 0 ? chunk_len[c1 - 1] : 0, tok0_n = nsteps > 0 ? chunk_tok0[c1 - 1] : 0;   // fetched a step ahead
+    int len_n = nsteps > 0 ? cg.chunk_len(c1 - 1) : 0, tok0_n = nsteps > 0 ? cg.chunk_tok0(c1 - 1) : 0;   // fetched a step ahead
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
         const int c = c1 - 1 - s, stage = s % STAGES, len = len_n, tok0 = tok0_n;
-        if (s + 1 < nsteps) { len_n = chunk_len[c - 1]; tok0_n = chunk_tok0[c - 1]; }
+        if (s + 1 < nsteps) { len_n = cg.chunk_len(c - 1); tok0_n = cg.chunk_tok0(c - 1); }
         unsigned char* tiles = sm + stage * STAGE_BYTES;
         const float *gl = gl2[s & 1], *Gam = Gam2[s & 1], *ee = ee2[s & 1];
         T64(0);
@@ -577,12 +579,14 @@ static bool fill_params64(Tc64Params& P, const Problem& p, bool with_bwd) {
 }
 
 static cudaError_t tc64_prologue(const Problem& p, cudaStream_t st) {
-    cudaError_t e = launch_table(p, st);
-    if (e != cudaSuccess) return e;
-    const int CH = p.L.max_chunks * p.d.H;
-    if (CH > 0 && p.Ttot > 0) {
+    // the chunk table is needed for packed sequences only (and for an empty call, whose only kernel it is)
+    if (p.cu || p.Ttot == 0) {
+        const cudaError_t e = launch_table(p, st);
+        if (e != cudaSuccess) return e;
+    }
+    if (p.L.max_chunks > 0 && p.Ttot > 0) {
         StageScope t(ST_PREP, st);
-        tc64_gamma_kernel<<<(CH + 7) / 8, 256, 0, st>>>(p);
+        tc64_gamma_kernel<<<dim3(p.L.max_chunks, (p.d.H + 31) / 32), 256, 0, st>>>(p);
     }
     return cudaGetLastError();
 }

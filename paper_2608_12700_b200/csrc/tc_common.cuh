@@ -145,6 +145,48 @@ __device__ __forceinline__ void chunk_entry(const Problem& p, ChunkInfo& x, int 
         x.len = min(kC, p.d.T - pos * kC);
     }
 }
+// The same geometry for kernels that walk along whole sequences.
+struct ChunkGeom {
+    const int32_t *first, *tok0, *len;   // tables (packed sequences), else null
+    int cps, T;                          // equal lengths: chunks per sequence, tokens per sequence
+    __device__ __forceinline__ int seq_first(int n) const { return first ? first[n] : n * cps; }
+    __device__ __forceinline__ int chunk_tok0(int c) const {
+        if (tok0) return tok0[c];
+        const int n = c / cps;
+        return n * T + (c - n * cps) * kC;
+    }
+    __device__ __forceinline__ int chunk_len(int c) const { return len ? len[c] : min(kC, T - (c % cps) * kC); }
+};
+__device__ __forceinline__ ChunkGeom chunk_geom(const Problem& p) {
+    ChunkGeom g;
+    g.first = p.cu ? reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first) : nullptr;
+    g.tok0 = p.cu ? reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_tok0) : nullptr;
+    g.len = p.cu ? reinterpret_cast<const int32_t*>(p.ws + p.L.chunk_len) : nullptr;
+    g.cps = max(1, chunks_per_sequence(p));
+    g.T = p.d.T;
+    return g;
+}
+// One sequence, for the kernels that walk along it: its chunks are consecutive, each starts 64 tokens after the one
+// before, only the last can be short.  (cu_seqlens has been validated by the table kernel by the time it is read here.)
+struct SeqGeom {
+    int c0, n_chunks, tok0, len;   // first chunk, number of chunks, first token, tokens
+    __device__ __forceinline__ int chunk_tok0(int c) const { return tok0 + (c - c0) * kC; }
+    __device__ __forceinline__ int chunk_len(int c) const { return min(kC, len - (c - c0) * kC); }
+};
+__device__ __forceinline__ SeqGeom seq_geom(const Problem& p, int n) {
+    SeqGeom g;
+    if (p.cu) {
+        g.tok0 = p.cu[n];
+        g.len = p.cu[n + 1] - g.tok0;
+        g.c0 = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first)[n];
+    } else {
+        g.tok0 = n * p.d.T;
+        g.len = p.d.T;
+        g.c0 = n * chunks_per_sequence(p);
+    }
+    g.n_chunks = (g.len + kC - 1) / kC;
+    return g;
+}
 __device__ __forceinline__ bool chunk_info(const Problem& p, ChunkInfo& x, int item) {
     if (item / p.d.H >= n_chunks_of(p)) return false;
     chunk_entry(p, x, item);
