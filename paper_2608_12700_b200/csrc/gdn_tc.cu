@@ -203,8 +203,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC], ww[kC], bgam[kC];
-    __shared__ uint64_t bar_qk, bar_vo, bar_ld0, bar_t, bar_vofree, bar_ld1, bar_st, bar_tfree, bar_free1, bar_free, bar_mma;
+    // gate arrays, two sets: a trip's set is written during the trip before it
+    __shared__ __align__(16) float gate_sets[2][6][kC];
+    __shared__ uint64_t bar_qk, bar_vo, bar_ld0, bar_t, bar_vofree, bar_ld1, bar_st, bar_tfree, bar_free1, bar_free2, bar_free, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
@@ -219,7 +220,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     if (threadIdx.x == 0) {
         mbar_init(&bar_qk, 1); mbar_init(&bar_vo, 1); mbar_init(&bar_ld0, 1); mbar_init(&bar_t, 1);
         mbar_init(&bar_vofree, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_st, 1); mbar_init(&bar_tfree, 1);
-        mbar_init(&bar_free1, 1); mbar_init(&bar_free, 1); mbar_init(&bar_mma, 1);
+        mbar_init(&bar_free1, 1); mbar_init(&bar_free2, 1); mbar_init(&bar_free, 1); mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
@@ -251,9 +252,13 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 const bool has_next = item + (int)gridDim.x < n_items;
                 if (has_next) chunk_entry(p, nx, item + gridDim.x);
                 pend_qk = pend_vo = false;
-                // the trip is under way: Q, K of the next one (loaded late in this trip) -> L2
+                // the trip is under way: the inputs of the next one (loaded late in this trip) -> L2
                 if (!(lok = mbar_wait(&bar_ld0, ph))) break;
                 if (has_next) {
+                    for (int cb = 0; cb < 2; ++cb) {
+                        prefetch_l2_tma_2d(&P.tm_v, nx.hd * D + cb * 64, nx.tok0);
+                        if (bwd) prefetch_l2_tma_2d(&P.tm_do, nx.hd * D + cb * 64, nx.tok0);
+                    }
                     for (int cb = 0; cb < 2; ++cb) {
                         prefetch_l2_tma_2d(&P.tm_q, nx.hd * D + cb * 64, nx.tok0);
                         prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + cb * 64, nx.tok0);
@@ -267,15 +272,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 if (!(lok = mbar_wait(&bar_vofree, ph))) break;
                 bulk_wait_read<0>();
                 mbar_arrive(&bar_tfree);   // the T tile may be overwritten (by the staged Nm image)
-                bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
-                bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
-                bulk_commit();
-                if (has_next) {
+                if (has_next) {            // (the loads first: the next trip starts with them, the stores have time)
                     mbar_expect_tx(&bar_vo, VO_BYTES);
                     pend_vo = true;
 #pragma unroll 1
                     for (int piece = 4; piece < 8; ++piece) load_piece(piece, nx);
                 }
+                bulk_store(p.ws + p.L.W + (size_t)x.ch * 16384, sm + WT, 16384);
+                bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
+                bulk_commit();
                 // phase 3 is done: Q, K have been read for the last time
                 if (!(lok = mbar_wait(&bar_ld1, ph))) break;
                 if (has_next) {
@@ -292,16 +297,24 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 #endif
                     }
                 }
-                // the three images are staged.  A store drains shared memory at some 32 bytes per cycle, so they leave in
-                // the order in which the next trip rewrites their tiles: E (fp32 scratch) and Nm (P) first, Bf last
+                // the three images are staged.  All CTAs store at about the same time, so the 96 KB drain at the rate of
+                // HBM (some 22 bytes per cycle and SM); they leave in the order in which the next trip rewrites their
+                // tiles: first the bytes under the fp32 A block (head of the E image) and under P (tail of the Nm image),
+                // then those under the fp32 T block (rest of E), last what the T tiles and the second readout overwrite
                 if (!(lok = mbar_wait(&bar_st, ph))) break;
-                if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + ES, 32768);
-                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + NMS, 32768);
+                constexpr uint32_t A_BYTES = XT - XA;
+                if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + ES, A_BYTES);
+                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768 + (PT - TT), sm + NMS + (PT - TT), 8192);
                 bulk_commit();
+                if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768 + A_BYTES, sm + ES + A_BYTES, 32768 - A_BYTES);
+                bulk_commit();
+                bulk_wait_read<1>();       // (issuing a store takes hundreds of cycles: the first group has drained by now)
+                mbar_arrive(&bar_free1);   // the fp32 A block and P may be written (and the scratch over W^T: its store is older)
+                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + NMS, PT - TT);
                 bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + BFS, 32768);
                 bulk_commit();
                 bulk_wait_read<1>();
-                mbar_arrive(&bar_free1);   // the E and Nm staging tiles may be rewritten
+                mbar_arrive(&bar_free2);   // the fp32 T block may be written
                 bulk_wait_read<0>();
                 mbar_arrive(&bar_free);    // every staging tile may be rewritten
             }
@@ -334,24 +347,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
             }
         }
     };
-    if (warp == 0) fetch_gates(xn);
-    // first trip: the inputs are loaded at once, one instruction per warp
-    if (issuer) { mbar_expect_tx(&bar_qk, 32768); mbar_expect_tx(&bar_vo, VO_BYTES); }
-    if (lane == 0 && warp < 8) load_piece(warp, xn);
-#pragma unroll 1
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-    const ChunkInfo x = xn;
-    const float g_now[2] = {ng[0], ng[1]}, b_now[2] = {nb[0], nb[1]};
-    const bool has_next = item + (int)gridDim.x < n_items;
-    const bool first = item == (int)blockIdx.x;
-    if (has_next) chunk_entry(p, xn, item + gridDim.x);
-    GDN_TICK(0, 0);
-    GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
-
-    // gates: erase gate b, write gate w, chunk-local cumulative decay gam (inclusive prefix sum of the 64 log decays),
-    // all by warp 0 in registers; the barrier before phase 1 publishes the arrays
-    if (warp == 0) {
-        float a = g_now[0], b = g_now[1];
+    // Warp 0 turns the fetched values into the gate arrays of chunk-head `ch` (set `set`): erase gate b, write gate w,
+    // chunk-local cumulative decay gam (inclusive prefix sum of the 64 log decays), in registers.
+    auto make_gates = [&](int set, int ch) {
+        float a = ng[0], b = ng[1];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float ua = __shfl_up_sync(0xffffffffu, a, o), ub = __shfl_up_sync(0xffffffffu, b, o);
@@ -360,18 +359,40 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         b += __shfl_sync(0xffffffffu, a, 31);
         const float gend = __shfl_sync(0xffffffffu, b, 31);
         const float gc[2] = {a, b};
+        float (*gs)[kC] = gate_sets[set];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int i = lane + 32 * h;
             const float G = expf(gc[h]);
-            gl[i] = gc[h] * kLog2e;
-            Gam[i] = G;
-            bb[i] = b_now[h]; ww[i] = b_now[h];
-            bgam[i] = b_now[h] * G;
-            ee[i] = expf(gend - gc[h]);
-            reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gc[h];
+            gs[0][i] = gc[h] * kLog2e;
+            gs[1][i] = G;
+            gs[2][i] = expf(gend - gc[h]);
+            gs[3][i] = nb[h];
+            gs[4][i] = nb[h];
+            gs[5][i] = nb[h] * G;
+            reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)ch * kC + i] = gc[h];
         }
-    }
+    };
+    if (warp == 0) { fetch_gates(xn); make_gates(0, xn.ch); }
+    // first trip: the inputs are loaded at once, one instruction per warp
+    if (issuer) { mbar_expect_tx(&bar_qk, 32768); mbar_expect_tx(&bar_vo, VO_BYTES); }
+    if (lane == 0 && warp < 8) load_piece(warp, xn);
+#pragma unroll 1
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
+    const ChunkInfo x = xn;
+    const bool has_next = item + (int)gridDim.x < n_items;
+    const bool first = item == (int)blockIdx.x;
+    if (has_next) chunk_entry(p, xn, item + gridDim.x);
+    GDN_TICK(0, 0);
+    GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
+
+    // this trip's gate arrays (written by warp 0 during the previous trip; the barrier before phase 1 publishes them)
+    const float* gl = gate_sets[in_phase][0];
+    const float* Gam = gate_sets[in_phase][1];
+    const float* ee = gate_sets[in_phase][2];
+    const float* bb = gate_sets[in_phase][3];
+    const float* ww = gate_sets[in_phase][4];
+    const float* bgam = gate_sets[in_phase][5];
     GDN_TICK(0, 20);
     if (ok) {
         ok = mbar_wait(&bar_vo, in_phase);
@@ -402,7 +423,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
     if (has_next && warp == 0) fetch_gates(xn);   // next trip's gates -> registers while the product runs
     GDN_WAIT_MMA(2)
-    if (ok && !first) {   // the previous trip's E and Nm stores have read their tiles (the fp32 scratch and P are next)
+    GDN_TICK(0, 23);
+    if (ok && !first) {   // the previous trip's stores have read what lies under the fp32 A block and under P
         ok = mbar_wait(&bar_free1, in_phase ^ 1);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 6);
     }
@@ -435,11 +457,13 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     cta_sync();
     GDN_TICK(0, 3);
     // ---- T = (I + A)^-1, blocked (see inv_diag8 ... inv_level).  All fp32.
-    inv_diag8(Af, Tf);
-    if (ok && !first) {   // every store of the previous trip has read its tile (the scratch S lies over W^T)
-        ok = mbar_wait(&bar_free, in_phase ^ 1);
-        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 5);
+    GDN_TICK(0, 24);
+    if (ok && !first) {   // ... and what lies under the fp32 T block
+        ok = mbar_wait(&bar_free2, in_phase ^ 1);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 8);
     }
+    GDN_TICK(0, 25);
+    inv_diag8(Af, Tf);
     cta_sync();
     inv_diag16(Af, Tf, Sf);
     cta_sync();
@@ -455,6 +479,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     inv_level<3, 4, 2>(Sf, Tf);
     cta_sync();
     GDN_TICK(0, 4);
+    if (ok && !first) {   // every store of the previous trip has read its tile (the T tiles and the second readout are next)
+        ok = mbar_wait(&bar_free, in_phase ^ 1);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 5);
+    }
     if (threadIdx.x < kC * 4) {   // T -> bf16 tiles T, T Diag(b Gam), T Diag(w): a thread scales two rows of one 8-column piece
         const int cch = threadIdx.x & 7;
         float gb[8], gw[8];
@@ -549,7 +577,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     } else if (threadIdx.x == 32) {
         mbar_arrive(&bar_vofree);   // W^T, U~^T are staged; V, dO were last read by phase 2 and the pass that formed R
     }
+    if (has_next && warp == 0) make_gates(in_phase ^ 1, xn.ch);   // the next trip's gate arrays, while the products run
     GDN_WAIT_MMA(4)
+    GDN_TICK(0, 26);
     if (ok) {   // the T tile, part of the Nm staging area, has left through its store
         ok = mbar_wait(&bar_tfree, in_phase);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 7);
