@@ -844,7 +844,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ __align__(16) float gl[kC], Gam[kC], ee[kC], bb[kC];
+    __shared__ __align__(16) float gate_sets[2][4][kC];   // two sets: a trip's gate arrays are written during the trip before
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
     __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
@@ -1002,6 +1002,13 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         ngend = gsrc[kC - 1];
         nb = ((int)threadIdx.x < c.len) ? p.beta[(size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd] : 0.f;
     };
+    auto make_gates = [&](int set) {   // threads 0..63: the fetched values -> gate arrays of set `set`
+        const int i = threadIdx.x;
+        gate_sets[set][0][i] = ng * kLog2e;
+        gate_sets[set][1][i] = expf(ng);
+        gate_sets[set][2][i] = expf(ngend - ng);
+        gate_sets[set][3][i] = nb;
+    };
     // dbeta and dg of the previous trip's chunk, from its token-wise partial sums (warps 0 and 1; see the trip's end)
     ChunkInfo xp = xn;
     bool have_prev = false;
@@ -1022,11 +1029,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // first trip: every group is loaded at once, one instruction per warp
     if (issuer) { mbar_expect_tx(&bar_k, K_BYTES); mbar_expect_tx(&bar_g1, G1_BYTES); mbar_expect_tx(&bar_g2, G2_BYTES); }
     if (lane == 0 && warp < 13) load_piece(warp, xn);
-    if (threadIdx.x < kC) fetch_gates(xn);
+    if (threadIdx.x < kC) { fetch_gates(xn); make_gates(0); }
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
     const ChunkInfo x = xn;
-    const float g_now = ng, gend_now = ngend, b_now = nb;
+    // this trip's gate arrays (the barrier before phase 1 publishes them)
+    const float* gl = gate_sets[in_phase][0];
+    const float* Gam = gate_sets[in_phase][1];
+    const float* ee = gate_sets[in_phase][2];
+    const float* bb = gate_sets[in_phase][3];
     const bool has_next = item + (int)gridDim.x < n_items;
     const bool first = item == (int)blockIdx.x;
     if (has_next) chunk_entry(p, xn, item + gridDim.x);
@@ -1039,13 +1050,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     sync_no = 0;
 #endif
 
-    if (threadIdx.x < kC) {
-        const int i = threadIdx.x;
-        gl[i] = g_now * kLog2e;
-        Gam[i] = expf(g_now);
-        ee[i] = expf(gend_now - g_now);
-        bb[i] = b_now;
-    }
     GDN_TICK(2, 19);
     if (ok) {
         ok = mbar_wait(&bar_g1, in_phase);
@@ -1195,6 +1199,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_commit(&bar_mma2);
     }
     GDN_TICK(2, 7);
+    if (has_next && threadIdx.x < kC) make_gates(in_phase ^ 1);   // the next trip's gate arrays, while the product runs
     GDN_WAIT_MMA(23)
     if (ok && worker) {   // dPD = scale tril(dO U^T) . D  (group B; the accumulator loads are warp-wide instructions)
         float v2[2][8];
