@@ -454,8 +454,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         }
     }
     tc_fence_before();
+    fence_async_smem();
     cta_sync();
     GDN_TICK(0, 3);
+    // (P^T dO)^T = dO^T P needs nothing of the inversion: it runs under it and is covered by phase 2's commit
+    if (ok && issuer && bwd) {
+        tc_fence_after();
+        mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
+    }
     // ---- T = (I + A)^-1, blocked (see inv_diag8 ... inv_level).  All fp32.
     GDN_TICK(0, 24);
     if (ok && !first) {   // ... and what lies under the fp32 T block
@@ -512,12 +518,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     cta_sync();
     GDN_TICK(0, 5);
 
-    // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T ; (P^T dO)^T = dO^T P
+    // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T
     if (ok && issuer) {
         tc_fence_after();
         mma_tile<128, 64, 64>(tmem + C_W, op_mn_major(sm + QK, 128, 64), op_k_major(sm + TP, 64), false);
         mma_tile<128, 64, 64>(tmem + C_U, op_mn_major(sm + VO, 128, 0), op_k_major(sm + TPP, 64), false);
-        if (bwd) mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
         mma_commit(&bar_mma);
     }
     if (threadIdx.x == 32) mbar_arrive(&bar_t);   // the loader stores the T tile
@@ -568,8 +573,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     // ---- phase 3: Nm = K^T (Diag(e) W) ; Bf = K^T (Diag(e) U~) ; E = Q^T R - W^T (P^T dO)
     if (ok && issuer) {
         tc_fence_after();
-        mma_tile<128, 128, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
-        mma_tile<128, 128, 64>(tmem + C_BF, op_mn_major(sm + QK, 128, 64), op_k_major(sm + UET, 128), false);
+        // Nm and Bf share the operand K^T; their other operands and their accumulators are neighbours: one N = 256 product
+        static_assert(UET == WET + 16384 && C_BF == C_NM + 128, "Nm | Bf as one product");
+        mma_tile<128, 256, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
