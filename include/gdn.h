@@ -161,8 +161,12 @@ gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* l
  * host memory as row-major float32, whatever the internal storage format:
  *   "gamma" [64]   "T" [64,64]   "W" [64,d_k]   "Ut" [64,d_v]   "Nm" [d_k,d_k]
  *   "Bf", "E", "hc", "dhn" [d_k,d_v]
+ * "Nm" and "Bf" are written only when the carries run in operator form (see below).
  * gdn_debug_force_family: 0 = automatic dispatch, 1 = always use the FFMA kernels (tests use this to
- * exercise both families on the same inputs).  Process-wide; affects workspace sizes as well. */
+ * exercise both families on the same inputs); 2 / 3 = automatic family, but the tcgen05 d = 128 kernels carry the
+ * state across chunks in operator form (one d x d matrix per chunk) / in low-rank form (two dependent products
+ * per chunk, no such matrix), whatever the shape; by default the shape decides.  Process-wide; 1 affects workspace
+ * sizes as well. */
 gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
                           float* host_out);
 gdn_status gdn_debug_force_family(int32_t family);

@@ -168,6 +168,8 @@ def gdn_stage_timing_read():
 
 
 def gdn_debug_force_family(family: int) -> None:
+    """0: automatic dispatch.  1: FFMA kernels.  2 / 3: the tcgen05 d = 128 kernels carry the state across chunks
+    in operator form / in low-rank form whatever the shape (by default the shape decides)."""
     s = lib().gdn_debug_force_family(int(family))
     if s != GDN_OK:
         raise GdnError(s, "gdn_debug_force_family")

@@ -50,6 +50,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 enum class Path { None, SimtF32, SimtBf16, TcBf16, Tc64Bf16 };
 
 int g_force_family = 0;
+}  // namespace
+int g_force_carries = 0;   // tcgen05 d = 128 family: 0 = by shape, 1 = operator form (Nm, Bf), 2 = low-rank form
+namespace {
 
 Path pick_path(const gdn_desc& d) {
     if (d.dtype == GDN_F32) return Path::SimtF32;
@@ -185,8 +188,9 @@ const char* gdn_status_string(gdn_status s) {
 }
 
 gdn_status gdn_debug_force_family(int32_t family) {
-    if (family != 0 && family != 1) return GDN_ERR_BAD_SHAPE;
-    g_force_family = family;
+    if (family < 0 || family > 3) return GDN_ERR_BAD_SHAPE;
+    g_force_family = family == 1 ? 1 : 0;
+    g_force_carries = family >= 2 ? family - 1 : 0;
     return GDN_OK;
 }
 

@@ -121,6 +121,7 @@ cudaError_t simt_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t 
 size_t simt_scratch_per_chunkhead(const gdn_desc& d);
 
 // tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
+extern int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank form
 bool tc_supported(const gdn_desc& d);
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);

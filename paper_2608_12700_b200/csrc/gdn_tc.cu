@@ -62,6 +62,7 @@ struct TcParams {
     CUtensorMap tm_dq, tm_dk, tm_dv;       // same geometry, for the gradient stores of full chunks
     int with_bwd;                          // prep: also produce E
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
+    int lowrank;                           // carries in low-rank form (tc_scan_lr): tc_prep makes no Nm, Bf
 };
 
 // Blocked inverse of I + A (unit lower triangular), fp32 in shared memory, rows of kLdi floats:
@@ -200,6 +201,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     const int n_items = n_chunks_of(p) * H;
     if ((int)blockIdx.x >= n_items) return;
     const bool bwd = P.with_bwd != 0;
+    const bool opform = P.lowrank == 0;   // the carries want the chunk operator Nm and the additive term Bf
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
@@ -304,14 +306,16 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 if (!(lok = mbar_wait(&bar_st, ph))) break;
                 constexpr uint32_t A_BYTES = XT - XA;
                 if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + ES, A_BYTES);
-                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768 + (PT - TT), sm + NMS + (PT - TT), 8192);
+                if (opform) bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768 + (PT - TT), sm + NMS + (PT - TT), 8192);
                 bulk_commit();
                 if (bwd) bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768 + A_BYTES, sm + ES + A_BYTES, 32768 - A_BYTES);
                 bulk_commit();
                 bulk_wait_read<1>();       // (issuing a store takes hundreds of cycles: the first group has drained by now)
                 mbar_arrive(&bar_free1);   // the fp32 A block and P may be written (and the scratch over W^T: its store is older)
-                bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + NMS, PT - TT);
-                bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + BFS, 32768);
+                if (opform) {
+                    bulk_store(p.ws + p.L.Nm + (size_t)x.ch * 32768, sm + NMS, PT - TT);
+                    bulk_store(p.ws + p.L.Bf + (size_t)x.ch * 32768, sm + BFS, 32768);
+                }
                 bulk_commit();
                 bulk_wait_read<1>();
                 mbar_arrive(&bar_free2);   // the fp32 T block may be written
@@ -551,13 +555,13 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
 #pragma unroll
             for (int i = 0; i < 8; ++i) ve[i] = v[i] * e8[i];
             chunk_store(sm + WT, 128, f, ib >> 3, v);
-            chunk_store(sm + WET, 128, f, ib >> 3, ve);
+            if (opform) chunk_store(sm + WET, 128, f, ib >> 3, ve);
             tmem_ld8(tmem + lane_base + C_U + ib, v);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 8; ++i) ve[i] = v[i] * e8[i];
             chunk_store(sm + UTT, 128, f, ib >> 3, v);
-            chunk_store(sm + UET, 128, f, ib >> 3, ve);
+            if (opform) chunk_store(sm + UET, 128, f, ib >> 3, ve);
             if (bwd) {
                 tmem_ld8(tmem + lane_base + C_PDO + ib, v);
                 tmem_wait_ld();
@@ -575,7 +579,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         tc_fence_after();
         // Nm and Bf share the operand K^T; their other operands and their accumulators are neighbours: one N = 256 product
         static_assert(UET == WET + 16384 && C_BF == C_NM + 128, "Nm | Bf as one product");
-        mma_tile<128, 256, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
+        if (opform) mma_tile<128, 256, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
         if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
@@ -598,12 +602,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         for (int part = 0; part < D / kGroups / 8; ++part) {
             const int cb = c0 + part * 8;
             float v[8];
-            tmem_ld8(tmem + lane_base + C_NM + cb, v);
-            tmem_wait_ld();
-            chunk_store(sm + NMS, 128, r, cb >> 3, v);
-            tmem_ld8(tmem + lane_base + C_BF + cb, v);
-            tmem_wait_ld();
-            chunk_store(sm + BFS, 128, r, cb >> 3, v);
+            if (opform) {
+                tmem_ld8(tmem + lane_base + C_NM + cb, v);
+                tmem_wait_ld();
+                chunk_store(sm + NMS, 128, r, cb >> 3, v);
+                tmem_ld8(tmem + lane_base + C_BF + cb, v);
+                tmem_wait_ld();
+                chunk_store(sm + BFS, 128, r, cb >> 3, v);
+            }
             if (bwd) {
                 tmem_ld8(tmem + lane_base + C_E + cb, v);
                 tmem_wait_ld();
@@ -793,6 +799,207 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, NS);
+}
+
+// ------------------------------------------------------------------------------------------------
+// tc_scan_lr: the same carries without the d x d operator of a chunk, for shapes whose carries are bound by HBM
+// bandwidth (one CTA per chain and direction fills the machine).  With e_j = exp(gam_e - gam_j):
+//   forward   h'  = Gam_e h   + K^T Diag(e) (U~ - W h)
+//   reverse   dh  = Gam_e dh' + E - W^T Diag(e) (K dh')
+// Two dependent products per step instead of one, but tc_prep neither forms nor writes Nm and Bf (64 KB per
+// chunk-head less to write and 16 KB less to read).  Per step a ring slot receives W^T, the K tile of the chunk and
+// U~^T (forward) or E (reverse); the first product leaves (W h)^T or (K dh')^T with features on TMEM lanes and tokens
+// on columns, the readout forms the scaled bf16 operand of the second product in the same orientation, the second
+// product yields the d_k x d_v increment of the state, which lives in fp32 registers as in tc_scan.
+// ------------------------------------------------------------------------------------------------
+namespace scanlr {
+constexpr int GE_CAP = 2048;
+constexpr int STAGES = 2;
+constexpr uint32_t WT = 0, KT = 16384, XT = 32768, STAGE_BYTES = 65536;   // ring slot: W^T | K | U~^T (16 KB) or E (32 KB)
+constexpr uint32_t HT = STAGES * STAGE_BYTES;      // two bf16 state tiles [128][128]
+constexpr uint32_t GT = HT + 2 * 32768;            // operand of the second product, [128 features][64 tokens]
+constexpr uint32_t SMEM_BYTES = GT + 16384 + 1024;
+constexpr uint32_t C_D1 = 0, C_D2 = 64;            // TMEM columns: first product (64), second product (128)
+static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budget");
+}  // namespace scanlr
+
+__global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_constant__ TcParams P) {
+    using namespace scanlr;
+    const int bid = (int)blockIdx.x;
+    const Problem& p = P.p;
+    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
+    if (hdr->status != GDN_OK) return;
+    const int reverse = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
+    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
+    const int H = p.d.H, n = chain / H, hd = chain % H;
+    const SeqGeom sg = seq_geom(p, n);
+    const int c0 = sg.c0, nsteps = sg.n_chunks, c1 = c0 + nsteps;
+
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* sm = align1024(smem_raw);
+    __shared__ float ge[GE_CAP];
+    __shared__ __align__(16) float ee2[2][kC];   // e_j of a step, made during the step before it
+    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ uint32_t tmem_slot;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q4 = warp & 3, hf = warp >> 2;
+    const int r = q4 * 32 + lane;              // TMEM lane of this thread: state row (d_k) or feature of the first product (d_v)
+    const int lc0 = hf * 64;                   // first of its 64 state columns
+    const int tk0 = hf * 32;                   // first of its 32 tokens in the first product
+    const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(&bar_full[s], 1);
+        mbar_init(&bar_mma, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    auto chunk_of = [&](int s) { return reverse ? (c1 - 1 - s) : (c0 + s); };
+    const char* w_base = p.ws + p.L.W;
+    const char* x_base = p.ws + (reverse ? p.L.E : p.L.Ut);
+    const uint32_t x_chunk = reverse ? 32768u : 16384u;
+    char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
+    const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
+    auto prefetch = [&](int s) {   // the ring gives a load one step of lead, less than an HBM round trip
+        const int c = chunk_of(s);
+        const size_t ch = (size_t)c * H + hd;
+        prefetch_l2_bulk(w_base + ch * 16384, 16384);
+        prefetch_l2_bulk(x_base + ch * x_chunk, x_chunk);
+        prefetch_l2_tma_2d(&P.tm_k, hd * D, sg.chunk_tok0(c));
+        prefetch_l2_tma_2d(&P.tm_k, hd * D + 64, sg.chunk_tok0(c));
+    };
+    auto fill = [&](int s) {   // thread 32: bring chunk step s into ring slot s % STAGES
+        const int stage = s % STAGES, c = chunk_of(s);
+        const size_t ch = (size_t)c * H + hd;
+        unsigned char* slot = sm + stage * STAGE_BYTES;
+        mbar_expect_tx(&bar_full[stage], 32768 + x_chunk);
+        bulk_load(slot + WT, w_base + ch * 16384, 16384, &bar_full[stage]);
+        tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
+        tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
+        bulk_load(slot + XT, x_base + ch * x_chunk, x_chunk, &bar_full[stage]);
+        if (s + STAGES + 1 < nsteps) prefetch(s + STAGES + 1);
+    };
+    if (threadIdx.x == 32) {
+        for (int s = STAGES; s < 2 * STAGES + 1 && s < nsteps; ++s) prefetch(s);
+        for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
+    }
+    for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
+        ge[s] = expf(gamma[((size_t)chunk_of(s) * H + hd) * kC + kC - 1]);
+    // e_j of the first step; the cumulative decays of the second are fetched now
+    auto gate_row = [&](int s) { return gamma + ((size_t)chunk_of(s) * H + hd) * kC; };
+    float gnext = 0.f, gend_next = 0.f;
+    if (threadIdx.x < kC && nsteps > 0) {
+        ee2[0][threadIdx.x] = expf(gate_row(0)[kC - 1] - gate_row(0)[threadIdx.x]);
+        if (nsteps > 1) { gnext = gate_row(1)[threadIdx.x]; gend_next = gate_row(1)[kC - 1]; }
+    }
+    float st[64];
+    {
+        const float* init = reverse ? p.dhT : p.h0;
+        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + lc0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            float4 v = init ? *reinterpret_cast<const float4*>(init + soff + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+            st[4 * k] = v.x; st[4 * k + 1] = v.y; st[4 * k + 2] = v.z; st[4 * k + 3] = v.w;
+        }
+    }
+    __syncthreads();
+    bool ok = true;
+    uint32_t mma_phase = 0;
+#pragma unroll 1
+    for (int s = 0; s < nsteps; ++s) {
+        unsigned char* Ht = sm + HT + (s & 1) * 32768;
+        const int c = chunk_of(s), stage = s % STAGES, len = sg.chunk_len(c);
+        const size_t ch = (size_t)c * H + hd;
+        unsigned char* ring = sm + stage * STAGE_BYTES;
+        const float* ee = ee2[s & 1];
+        const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
+        // state -> bf16: operand of the first product, and the per-chunk state the gradient stage reads
+#pragma unroll
+        for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
+        if (len < kC) {   // ragged tail: the K rows beyond the sequence belong to somebody else
+            ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
+            if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 12); break; }
+            zero_tail_rows(ring + KT, 64, 0, len, kThreads);
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
+            if (ok) {
+                tc_fence_after();
+                // forward (W h)^T = h^T W^T ; reverse (K dh')^T = dh'^T K^T : [d_v][tokens]
+                const Operand b = reverse ? op_k_major(ring + KT, 64) : op_mn_major(ring + WT, 128);
+                mma_tile<128, 64, 128>(tmem + C_D1, op_mn_major(Ht, 128), b, false);
+            } else {
+                report_timeout(p.ws, 10);
+            }
+            bulk_store(keep_base + ch * 32768, Ht, 32768);
+            bulk_commit();
+            bulk_wait_read<1>();   // (the store of the step before has read its tile: it is rewritten in the next step)
+            mma_commit(&bar_mma);
+        } else if (threadIdx.x == 32) {
+            if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
+        }
+        ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
+        if (ok) ok = mbar_wait(&bar_mma, mma_phase);
+        mma_phase ^= 1;
+        if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 11); break; }
+        tc_fence_after();
+        // operand of the second product: forward Diag(e)(U~ - W h), reverse Diag(e)(K dh'), transposed
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float d1[8], u[8], e8[8];
+            tmem_ld8(tmem + lane_base + C_D1 + tk0 + 8 * k, d1);
+            if (!reverse) chunk_load(ring + XT, 128, r, (tk0 >> 3) + k, u);
+            ld8s(ee + tk0 + 8 * k, e8);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) d1[j] = e8[j] * (reverse ? d1[j] : (u[j] - d1[j]));
+            chunk_store(sm + GT, 128, r, (tk0 >> 3) + k, d1);
+        }
+        tc_fence_before();
+        fence_async_smem();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            tc_fence_after();
+            if (reverse) mma_tile<128, 128, 64>(tmem + C_D2, op_k_major(ring + WT, 128), op_k_major(sm + GT, 128), false, /*neg_a=*/true);
+            else mma_tile<128, 128, 64>(tmem + C_D2, op_mn_major(ring + KT, 64), op_k_major(sm + GT, 128), false);
+            mma_commit(&bar_mma);
+        }
+        if (threadIdx.x < kC && s + 1 < nsteps) {   // e_j of the next step, while the product runs
+            ee2[(s + 1) & 1][threadIdx.x] = expf(gend_next - gnext);
+            if (s + 2 < nsteps) { gnext = gate_row(s + 2)[threadIdx.x]; gend_next = gate_row(s + 2)[kC - 1]; }
+        }
+        ok = mbar_wait(&bar_mma, mma_phase);
+        mma_phase ^= 1;
+        if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 13); break; }
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float d2[8], ad[8];
+            tmem_ld8(tmem + lane_base + C_D2 + lc0 + 8 * k, d2);
+            if (reverse) chunk_load(ring + XT, 128, r, (lc0 >> 3) + k, ad);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) st[8 * k + j] = fmaf(Ge, st[8 * k + j], reverse ? ad[j] + d2[j] : d2[j]);
+        }
+        tc_fence_before();
+    }
+    float* fin = reverse ? p.dh0 : p.hT;
+    if (fin && ok) {
+        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + lc0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
+    }
+    if (threadIdx.x == 0) bulk_wait_read<0>();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1541,10 +1748,15 @@ bool tc_supported(const gdn_desc& d) {
     return d.dtype == GDN_BF16 && d.d_k == 128 && d.d_v == 128 && d.delta_rule == 1 && d.chunk == kC;
 }
 
+static int sm_count();
 static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_dirs) {
     P.p = p;
     P.with_bwd = with_bwd ? 1 : 0;
     P.scan_dirs = scan_dirs;
+    // One CTA per (chain, direction) fills the machine: the carries are bound by HBM bandwidth, and the low-rank form
+    // moves less.  With fewer chains a step's latency counts, and the operator form needs one product per step.
+    const int ctas = p.d.N * p.d.H * (scan_dirs == 2 ? 2 : 1);
+    P.lowrank = g_force_carries ? (g_force_carries == 2) : (2 * ctas > sm_count());
     const uint64_t rows = (uint64_t)p.Ttot, cols = (uint64_t)p.d.H * D, pitch = cols * 2;
     if (!tc::make_tmap_bf16_2d(&P.tm_q, p.q, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
@@ -1592,6 +1804,10 @@ static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done;
     static SmemLimitOnce done2;
     const int ctas = P.p.d.N * P.p.d.H * (P.scan_dirs == 2 ? 2 : 1);
+    if (P.lowrank) {
+        static SmemLimitOnce done_lr;
+        return launch_chunk_kernel(tc_scan_lr_kernel, done_lr, scanlr::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
+    }
     // few chains: two CTAs per (chain, direction), each carrying half of the state columns
     if (2 * ctas <= sm_count())
         return launch_chunk_kernel(tc_scan_kernel<2>, done2, scan::Cfg<2>::SMEM_BYTES, ST_SCANS, 2 * ctas, kThreads, P, st);
