@@ -188,6 +188,7 @@ constexpr uint32_t SMEM_BYTES = TILES_END + 1024 /* alignment slack */;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 // TMEM columns (512 allocated): accumulators at fixed offsets, allocated once, released once.
 constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_NM = 256, C_BF = 384, C_E = 0;
+constexpr uint32_t C_E_LR = 256;   // low-rank mode (no Nm, Bf): E is started early, in columns of its own
 }  // namespace prep
 
 __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
@@ -270,6 +271,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 if (!(lok = mbar_wait(&bar_t, ph))) break;
                 bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
                 bulk_commit();
+                if (!opform) {   // low-rank mode: Q, K are dead after phase 2, before W^T, U~^T are staged
+                    if (!(lok = mbar_wait(&bar_ld1, ph))) break;
+                    if (has_next) {
+                        mbar_expect_tx(&bar_qk, 32768);
+                        pend_qk = true;
+#pragma unroll 1
+                        for (int piece = 0; piece < 4; ++piece) load_piece(piece, nx);
+                    }
+                }
                 // W^T, U~^T are staged and V, dO have been read for the last time
                 if (!(lok = mbar_wait(&bar_vofree, ph))) break;
                 bulk_wait_read<0>();
@@ -284,8 +294,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 bulk_store(p.ws + p.L.Ut + (size_t)x.ch * 16384, sm + UTT, 16384);
                 bulk_commit();
                 // phase 3 is done: Q, K have been read for the last time
-                if (!(lok = mbar_wait(&bar_ld1, ph))) break;
-                if (has_next) {
+                if (opform && !(lok = mbar_wait(&bar_ld1, ph))) break;
+                if (opform && has_next) {
 #ifdef GDN_PHASE_TIMING
                     if (blockIdx.x == 0) g_ticks[3][10] = clock64();
 #endif
@@ -426,6 +436,19 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     float* Tf = reinterpret_cast<float*>(sm + XT);   // [64][kLdi]  T
     float* Sf = reinterpret_cast<float*>(sm + WT);   // [64][kLdi]  scratch of the blocked inversion
     if (has_next && warp == 0) fetch_gates(xn);   // next trip's gates -> registers while the product runs
+    // R = Diag(Gam) dO (token-major tile) while the product runs.  In low-rank mode the tiles of Diag(e) W and
+    // Diag(e) U~ are never written, so R has a tile of its own from here on and Q^T R can run under the inversion.
+    auto form_R = [&](unsigned char* dst) {
+        for (int t = threadIdx.x; t < kC * 16; t += kIntraThreads) {
+            const int i = t >> 4, cch = t & 15;
+            float v[8];
+            chunk_load(sm + VO, 128, 64 + i, cch, v);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
+            chunk_store(dst, 64, i, cch, v);
+        }
+    };
+    if (bwd && !opform) form_R(sm + WET);
     GDN_WAIT_MMA(2)
     GDN_TICK(0, 23);
     if (ok && !first) {   // the previous trip's stores have read what lies under the fp32 A block and under P
@@ -465,6 +488,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     if (ok && issuer && bwd) {
         tc_fence_after();
         mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + VO, 128, 64), op_mn_major(sm + PT, 64), false);
+        // low-rank mode: so does the first half of E = Q^T R - W^T (P^T dO), into columns no other product uses
+        if (!opform) mma_tile<128, 128, 64>(tmem + C_E_LR, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + WET, 64), false);
     }
     // ---- T = (I + A)^-1, blocked (see inv_diag8 ... inv_level).  All fp32.
     GDN_TICK(0, 24);
@@ -528,19 +553,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         mma_tile<128, 64, 64>(tmem + C_W, op_mn_major(sm + QK, 128, 64), op_k_major(sm + TP, 64), false);
         mma_tile<128, 64, 64>(tmem + C_U, op_mn_major(sm + VO, 128, 0), op_k_major(sm + TPP, 64), false);
         mma_commit(&bar_mma);
+        if (!opform) mma_commit(&bar_ld1);   // low-rank mode: Q, K have been read for the last time
     }
     if (threadIdx.x == 32) mbar_arrive(&bar_t);   // the loader stores the T tile
-    // R = Diag(Gam) dO (token-major tile), while the MMAs run.  The fp32 A / T scratch is dead by now.
-    if (bwd) {
-        for (int t = threadIdx.x; t < kC * 16; t += kIntraThreads) {
-            const int i = t >> 4, cch = t & 15;
-            float v[8];
-            chunk_load(sm + VO, 128, 64 + i, cch, v);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
-            chunk_store(sm + XR, 64, i, cch, v);
-        }
-    }
+    // operator mode: R while the MMAs run, over the fp32 A / T scratch, which is dead by now
+    if (bwd && opform) form_R(sm + XR);
     GDN_WAIT_MMA(3)
     if (ok && worker) {
         const int f = q4 * 32 + lane, i0 = grp * kTG;
@@ -580,10 +597,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         // Nm and Bf share the operand K^T; their other operands and their accumulators are neighbours: one N = 256 product
         static_assert(UET == WET + 16384 && C_BF == C_NM + 128, "Nm | Bf as one product");
         if (opform) mma_tile<128, 256, 64>(tmem + C_NM, op_mn_major(sm + QK, 128, 64), op_k_major(sm + WET, 128), false);
-        if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
-        if (bwd) mma_tile<128, 128, 64>(tmem + C_E, op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
+        if (bwd && opform) mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + XR, 64), false);
+        if (bwd) mma_tile<128, 128, 64>(tmem + (opform ? C_E : C_E_LR), op_k_major(sm + WT, 128), op_k_major(sm + XPDO, 128), true, /*neg_a=*/true);
         mma_commit(&bar_mma);
-        mma_commit(&bar_ld1);   // Q, K have been read for the last time
+        if (opform) mma_commit(&bar_ld1);   // Q, K have been read for the last time
     } else if (threadIdx.x == 32) {
         mbar_arrive(&bar_vofree);   // W^T, U~^T are staged; V, dO were last read by phase 2 and the pass that formed R
     }
@@ -611,7 +628,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 chunk_store(sm + BFS, 128, r, cb >> 3, v);
             }
             if (bwd) {
-                tmem_ld8(tmem + lane_base + C_E + cb, v);
+                tmem_ld8(tmem + lane_base + (opform ? C_E : C_E_LR) + cb, v);
                 tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 8; ++k) v[k] *= sc;
