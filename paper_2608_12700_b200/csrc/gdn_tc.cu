@@ -438,14 +438,19 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     if (has_next && warp == 0) fetch_gates(xn);   // next trip's gates -> registers while the product runs
     // R = Diag(Gam) dO (token-major tile) while the product runs.  In low-rank mode the tiles of Diag(e) W and
     // Diag(e) U~ are never written, so R has a tile of its own from here on and Q^T R can run under the inversion.
-    auto form_R = [&](unsigned char* dst) {
-        for (int t = threadIdx.x; t < kC * 16; t += kIntraThreads) {
-            const int i = t >> 4, cch = t & 15;
-            float v[8];
-            chunk_load(sm + VO, 128, 64 + i, cch, v);
+    auto form_R = [&](unsigned char* dst) {   // the 512 worker threads, two 16-byte pieces each (both loads in flight)
+        if (worker) {
+            float v[2][8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
-            chunk_store(dst, 64, i, cch, v);
+            for (int it = 0; it < 2; ++it) chunk_load(sm + VO, 128, 64 + (threadIdx.x >> 4) + 32 * it, threadIdx.x & 15, v[it]);
+#pragma unroll
+            for (int it = 0; it < 2; ++it) {
+                const int i = (threadIdx.x >> 4) + 32 * it;
+                const float G = Gam[i];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) v[it][k] *= G;
+                chunk_store(dst, 64, i, threadIdx.x & 15, v[it]);
+            }
         }
     };
     if (bwd && !opform) form_R(sm + WET);
