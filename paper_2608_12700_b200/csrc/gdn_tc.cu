@@ -845,24 +845,18 @@ constexpr uint32_t C_D1 = 0, C_D2 = 64;            // TMEM columns: first produc
 static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budget");
 }  // namespace scanlr
 
-__global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_constant__ TcParams P) {
+// One direction of one chain (the direction is a compile-time constant: the two differ in operands and readouts).
+template <bool reverse>
+__device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, float* ge, float (*ee2)[kC], uint64_t* bar_full,
+                                              uint64_t& bar_mma, uint32_t& tmem_slot) {
     using namespace scanlr;
-    const int bid = (int)blockIdx.x;
     const Problem& p = P.p;
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    if (hdr->status != GDN_OK) return;
-    const int reverse = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
-    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
     const int H = p.d.H, n = chain / H, hd = chain % H;
     const SeqGeom sg = seq_geom(p, n);
     const int c0 = sg.c0, nsteps = sg.n_chunks, c1 = c0 + nsteps;
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float ge[GE_CAP];
-    __shared__ __align__(16) float ee2[2][kC];   // e_j of a step, made during the step before it
-    __shared__ uint64_t bar_full[STAGES], bar_mma;
-    __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, hf = warp >> 2;
     const int r = q4 * 32 + lane;              // TMEM lane of this thread: state row (d_k) or feature of the first product (d_v)
@@ -887,14 +881,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_co
     const uint32_t x_chunk = reverse ? 32768u : 16384u;
     char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
-    auto prefetch = [&](int s) {   // the ring gives a load one step of lead, less than an HBM round trip
-        const int c = chunk_of(s);
-        const size_t ch = (size_t)c * H + hd;
-        prefetch_l2_bulk(w_base + ch * 16384, 16384);
-        prefetch_l2_bulk(x_base + ch * x_chunk, x_chunk);
-        prefetch_l2_tma_2d(&P.tm_k, hd * D, sg.chunk_tok0(c));
-        prefetch_l2_tma_2d(&P.tm_k, hd * D + 64, sg.chunk_tok0(c));
-    };
+    // (L2 prefetches running ahead of the ring, as in tc_scan, made this kernel slower: 79.7 -> 78.5 us without)
     auto fill = [&](int s) {   // thread 32: bring chunk step s into ring slot s % STAGES
         const int stage = s % STAGES, c = chunk_of(s);
         const size_t ch = (size_t)c * H + hd;
@@ -904,10 +891,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_co
         tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
         tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
         bulk_load(slot + XT, x_base + ch * x_chunk, x_chunk, &bar_full[stage]);
-        if (s + STAGES + 1 < nsteps) prefetch(s + STAGES + 1);
     };
     if (threadIdx.x == 32) {
-        for (int s = STAGES; s < 2 * STAGES + 1 && s < nsteps; ++s) prefetch(s);
         for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
     }
     for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
@@ -1022,6 +1007,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_co
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_constant__ TcParams P) {
+    using namespace scanlr;
+    __shared__ float ge[GE_CAP];
+    __shared__ __align__(16) float ee2[2][kC];   // e_j of a step, made during the step before it
+    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ uint32_t tmem_slot;
+    const int bid = (int)blockIdx.x;
+    if (reinterpret_cast<const WsHeader*>(P.p.ws)->status != GDN_OK) return;
+    const int rev = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
+    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
+    if (rev) scan_lr_chain<true>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
+    else scan_lr_chain<false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
 }
 
 // ------------------------------------------------------------------------------------------------
