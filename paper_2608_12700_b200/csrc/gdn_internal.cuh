@@ -37,6 +37,7 @@ struct WsLayout {
     size_t fwd_end;        // bytes needed by the forward recompute
     size_t E;              // [CH, d_k, d_v]           scale (Gam Q - P W)^T dO
     size_t dhn;            // [CH, d_k, d_v]           gradient w.r.t. the state leaving the chunk
+    size_t Pm;             // [CH, 64, 64]             P = tril(Q K^T . D) (tcgen05 d = 128 family: made once, by tc_prep)
     size_t scratch;        // kernel-private staging, per chunk-head
     size_t scratch_per_ch; // bytes of scratch per chunk-head
     size_t total;
@@ -67,6 +68,7 @@ inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, siz
     L.fwd_end = o;
     L.E = take(elem_add * CH * d.d_k * d.d_v);
     L.dhn = take(elem * CH * d.d_k * d.d_v);
+    L.Pm = take(elem * CH * kC * kC);
     L.scratch_per_ch = scratch_per_ch;
     L.scratch = take(scratch_per_ch * CH);
     L.total = o;

@@ -270,6 +270,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 // T is staged
                 if (!(lok = mbar_wait(&bar_t, ph))) break;
                 bulk_store(p.ws + p.L.Tm + (size_t)x.ch * 8192, sm + TT, 8192);
+                if (bwd) bulk_store(p.ws + p.L.Pm + (size_t)x.ch * 8192, sm + PT, 8192);   // the gradient stage reads P from here
                 bulk_commit();
                 if (!opform) {   // low-rank mode: Q, K are dead after phase 2, before W^T, U~^T are staged
                     if (!(lok = mbar_wait(&bar_ld1, ph))) break;
@@ -1028,7 +1029,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_co
 //
 // Products (all on tcgen05, outputs transposed: features on TMEM lanes, tokens on columns, except the 64 x 64
 // token-token matrices which use M = 64):
-//   phase 1  S = Q K^T ; (W h)^T ; (K dh')^T                      -> P = tril(S . D)
+//   phase 1  (W h)^T ; (K dh')^T          (P = tril(Q K^T . D) comes from tc_prep, which forms it anyway)
 //   phase 2  (P^T dO)^T ; then, under the readout, dO h^T          -> U = U~ - W h ; dU = scale P^T dO + Diag(e) K dh'
 //   phase 3  dO U^T ; -(dU h^T)^T                                  -> dPD = scale tril(dO U^T) . D ; dW
 //   phase 4  (dPD K)^T ; (T^T dW)^T ; (T^T dU)^T ; (dPD^T Q)^T ; (U dh'^T)^T
@@ -1081,7 +1082,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     __shared__ __align__(16) float gate_sets[2][4][kC];   // two sets: a trip's gate arrays are written during the trip before
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
-    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
+    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_do, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
@@ -1098,7 +1099,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const bool loader = warp == 17;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bar_k, 1); mbar_init(&bar_g1, 1); mbar_init(&bar_g2, 1);
+        mbar_init(&bar_k, 1); mbar_init(&bar_g1, 1); mbar_init(&bar_g2, 1); mbar_init(&bar_do, 1);
         mbar_init(&bar_ld0, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_ld2, 1);
         mbar_init(&bar_st1, 1); mbar_init(&bar_st2, 1); mbar_init(&bar_kfree, 16); mbar_init(&bar_free, 1);
         mbar_init(&bar_mma, 1); mbar_init(&bar_mma2, 1);
@@ -1115,7 +1116,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     //   g1  Q, U~^T, dh', h, W   once the products of phase 5 are done       needed by phase 1
     //   g2  dO, T, V             once the products of phase 6 are done       needed from phase 2 on
     //   k   K                    once the last readout holds its K values    needed by phase 1
-    constexpr uint32_t K_BYTES = 16384, G1_BYTES = 16384 + 16384 + 32768 + 32768 + 16384, G2_BYTES = 16384 + 8192 + 16384;
+    constexpr uint32_t K_BYTES = 16384, G1_BYTES = 16384 + 16384 + 32768 + 32768 + 16384 + 8192, G2_BYTES = 8192 + 16384, DO_BYTES = 16384;
     auto load_piece = [&](int piece, const ChunkInfo& c) {
         const int cb = piece & 1, xq = c.hd * D + cb * 64;
         switch (piece) {
@@ -1125,9 +1126,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             case 5: bulk_load(sm + DH, p.ws + p.L.dhn + (size_t)c.ch * 32768, 32768, &bar_g1); break;
             case 6: bulk_load(sm + HH, p.ws + p.L.hc + (size_t)c.ch * 32768, 32768, &bar_g1); break;
             case 7: bulk_load(sm + WT, p.ws + p.L.W + (size_t)c.ch * 16384, 16384, &bar_g1); break;
-            case 8: case 9: tma_load_2d(sm + DO + cb * 8192, &P.tm_do, xq, c.tok0, &bar_g2); break;
+            case 8: case 9: tma_load_2d(sm + DO + cb * 8192, &P.tm_do, xq, c.tok0, &bar_do); break;
             case 10: case 11: tma_load_2d(sm + VT + cb * 8192, &P.tm_v, xq, c.tok0, &bar_g2); break;
             case 12: bulk_load(sm + TT, p.ws + p.L.Tm + (size_t)c.ch * 8192, 8192, &bar_g2); break;
+            case 13: bulk_load(sm + PT, p.ws + p.L.Pm + (size_t)c.ch * 8192, 8192, &bar_g1); break;
             default: break;
         }
     };
@@ -1135,7 +1137,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     if (loader) {
         if (lane == 0) {
             uint32_t ph = 0;
-            bool lok = true, pend_k = false, pend1 = false, pend2 = false;
+            bool lok = true, pend_k = false, pend1 = false, pend2 = false, pend_do = false;
 #pragma unroll 1
             for (int item = blockIdx.x; item < n_items && lok; item += gridDim.x, ph ^= 1) {
                 ChunkInfo x, nx;
@@ -1143,7 +1145,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 const bool has_next = item + (int)gridDim.x < n_items;
                 if (has_next) chunk_entry(p, nx, item + gridDim.x);
                 const bool full = x.len == kC;
-                pend_k = pend1 = pend2 = false;
+                pend_k = pend1 = pend2 = pend_do = false;
                 // the trip is under way (all its tiles have arrived): K of the next one, the only late load, -> L2
                 if (!(lok = mbar_wait(&bar_ld0, ph))) break;
                 if (has_next) {
@@ -1170,6 +1172,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     pend1 = true;
 #pragma unroll 1
                     for (int piece = 2; piece <= 7; ++piece) load_piece(piece, nx);
+                    load_piece(13, nx);
                 }
                 // phase 6 is done and the last readout holds its K values in registers: K first, the next trip starts with
                 // it; dO, T, V are not needed before its second phase (V goes where dv is staged, so that store must have
@@ -1181,11 +1184,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     pend_k = true;
                     load_piece(0, nx);
                     load_piece(1, nx);
+                    mbar_expect_tx(&bar_do, DO_BYTES);   // dO next: the second phase starts with it
+                    pend_do = true;
+                    load_piece(8, nx);
+                    load_piece(9, nx);
                     bulk_wait_read<0>();
                     mbar_expect_tx(&bar_g2, G2_BYTES);
                     pend2 = true;
 #pragma unroll 1
-                    for (int piece = 8; piece <= 12; ++piece) load_piece(piece, nx);
+                    for (int piece = 10; piece <= 12; ++piece) load_piece(piece, nx);
                 }
                 // dk is staged
                 if (!(lok = mbar_wait(&bar_st2, ph))) break;
@@ -1199,9 +1206,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     mbar_expect_tx(&bar_k, K_BYTES);
                     mbar_expect_tx(&bar_g1, G1_BYTES);
                     mbar_expect_tx(&bar_g2, G2_BYTES);
-                    pend_k = pend1 = pend2 = true;
+                    mbar_expect_tx(&bar_do, DO_BYTES);
+                    pend_k = pend1 = pend2 = pend_do = true;
 #pragma unroll 1
-                    for (int piece = 0; piece <= 12; ++piece) load_piece(piece, nx);
+                    for (int piece = 0; piece <= 13; ++piece) load_piece(piece, nx);
                 }
             }
             bulk_wait_read<0>();
@@ -1209,6 +1217,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 if (pend_k) (void)mbar_wait(&bar_k, ph ^ 1);
                 if (pend1) (void)mbar_wait(&bar_g1, ph ^ 1);
                 if (pend2) (void)mbar_wait(&bar_g2, ph ^ 1);
+                if (pend_do) (void)mbar_wait(&bar_do, ph ^ 1);
             }
         }
         return;
@@ -1261,8 +1270,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         }
     };
     // first trip: every group is loaded at once, one instruction per warp
-    if (issuer) { mbar_expect_tx(&bar_k, K_BYTES); mbar_expect_tx(&bar_g1, G1_BYTES); mbar_expect_tx(&bar_g2, G2_BYTES); }
-    if (lane == 0 && warp < 13) load_piece(warp, xn);
+    if (issuer) { mbar_expect_tx(&bar_k, K_BYTES); mbar_expect_tx(&bar_g1, G1_BYTES); mbar_expect_tx(&bar_g2, G2_BYTES); mbar_expect_tx(&bar_do, DO_BYTES); }
+    if (lane == 0 && warp < 14) load_piece(warp, xn);
     if (threadIdx.x < kC) { fetch_gates(xn); make_gates(0); }
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
@@ -1300,61 +1309,23 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     cta_sync();
     GDN_TICK(2, 1);
 
-    // ---- phase 1
+    // ---- phase 1: (W h)^T and (K dh')^T.  P = tril(Q K^T . D) is not formed here: tc_prep made it and it arrived
+    // with the first group of tiles.
     if (ok && issuer) {
         tc_fence_after();
-        mma_tile<64, 64, 128>(tmem + slot(0), op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
-        mma_commit(&bar_mma);   // the P readout needs only S; the two products below are covered by phase 2's commit
         mma_tile<128, 64, 128>(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
         mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
     }
-    if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // every tile of this trip has arrived
-    if (has_next && threadIdx.x < kC) fetch_gates(xn);
-    // <dh', h> over the whole state while the MMAs run (both tiles share one format, so offsets pair up); warps 0 and 1
-    // finish the previous chunk's gate gradients instead
-    float hh = 0.f;
-    if (ok && have_prev && warp < 2) finish_gates();
-#pragma unroll 1
-    for (int t = (int)threadIdx.x - 64; t >= 0 && t < 2048; t += kIntraThreads - 64) {
-        float a[8], b[8];
-        unpack8(*reinterpret_cast<const uint4*>(sm + HH + t * 16), a);
-        unpack8(*reinterpret_cast<const uint4*>(sm + DH + t * 16), b);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) hh = fmaf(a[k], b[k], hh);
-    }
     GDN_TICK(2, 2);
-    GDN_WAIT_MMA(21)
     GDN_TICK(2, 3);
-    const int mi = q4 * 16 + lane;     // row of an M = 64 accumulator held by this lane (lanes 0..15 only)
-    const int j0 = grp * kTG;
-    if (ok && worker) {   // P_ij = (q_i . k_j) D_ij for j <= i
-        float v2[2][8];
-        tmem_ld8(tmem + lane_base + slot(0) + j0, v2[0]);
-        tmem_ld8(tmem + lane_base + slot(0) + j0 + 8, v2[1]);
-        tmem_wait_ld();
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float (&v)[8] = v2[part];
-            const int jb = j0 + part * 8;
-            if (lane < 16) {
-                float g8[8];
-                ld8s(gl + jb, g8);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - g8[j]) : 0.f;
-                chunk_store(sm + PT, 64, mi, jb >> 3, v);
-            }
-        }
-    }
     if (ok) {
-        ok = mbar_wait(&bar_g2, in_phase);
+        ok = mbar_wait(&bar_do, in_phase);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 27);
     }
     if (ok && x.len < kC) {
-        zero_tail_rows(sm + VT, 64, 0, x.len, kIntraThreads);
         zero_tail_rows(sm + DO, 64, 0, x.len, kIntraThreads);
+        fence_async_smem();
     }
-    tc_fence_before();
-    fence_async_smem();
     cta_sync();
     GDN_TICK(2, 4);
 
@@ -1366,6 +1337,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         // dO h^T (token-major, group A of columns 384..511) is first read after phase 4: it runs under the readout
         mma_tile<64, 128, 128>(tmem + 384, op_k_major(sm + DO, 64), op_k_major(sm + HH, 128), false);
     }
+    if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // every tile of this trip has arrived
+    if (has_next && threadIdx.x < kC) fetch_gates(xn);
+    if (ok && have_prev && warp < 2) finish_gates();   // warps 0 and 1: the previous chunk's gate gradients
     GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
     if (ok && !first) {   // U^T and dU^T held the previous trip's staged dk and dq: their stores must have read them
@@ -1434,6 +1408,16 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     }
     GDN_TICK(2, 7);
     if (has_next && threadIdx.x < kC) make_gates(in_phase ^ 1);   // the next trip's gate arrays, while the product runs
+    // <dh', h> over the whole state, while the products run (both tiles share one format, so offsets pair up)
+    float hh = 0.f;
+#pragma unroll 1
+    for (int t = (int)threadIdx.x - 64; t >= 0 && t < 2048; t += kIntraThreads - 64) {
+        float a[8], b[8];
+        unpack8(*reinterpret_cast<const uint4*>(sm + HH + t * 16), a);
+        unpack8(*reinterpret_cast<const uint4*>(sm + DH + t * 16), b);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) hh = fmaf(a[k], b[k], hh);
+    }
     GDN_WAIT_MMA(23)
     if (ok && worker) {   // dPD = scale tril(dO U^T) . D  (group B; the accumulator loads are warp-wide instructions)
         float v2[2][8];
@@ -1466,6 +1450,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         chunk_store(sm + DWT, 128, f, i0 >> 3, w2[0]);              // dW^T = -(dU h^T)^T
         chunk_store(sm + DWT, 128, f, (i0 >> 3) + 1, w2[1]);
     }
+    if (ok) {   // V and T, the last tiles of this trip, are needed from phase 4 on
+        ok = mbar_wait(&bar_g2, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 31);
+    }
+    if (ok && x.len < kC) zero_tail_rows(sm + VT, 64, 0, x.len, kIntraThreads);
     tc_fence_before();
     fence_async_smem();
     cta_sync();
@@ -1484,11 +1473,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
     const bool full = x.len == kC;
-    const size_t rowp = (size_t)H * D;
-    const size_t gbase = ((size_t)x.tok0 * H + x.hd) * D;
-    __nv_bfloat16* gdq = reinterpret_cast<__nv_bfloat16*>(p.dq) + gbase;
-    __nv_bfloat16* gdk = reinterpret_cast<__nv_bfloat16*>(p.dk) + gbase;
-    __nv_bfloat16* gdv = reinterpret_cast<__nv_bfloat16*>(p.dv) + gbase;
+    // (addresses of the ragged-tail flushes are formed where they are used: nothing of them lives across the phases)
+    auto grad_rows = [&](void* base) { return reinterpret_cast<__nv_bfloat16*>(base) + ((size_t)x.tok0 * H + x.hd) * D; };
     if (ok && worker) {
         // The two lane groups hold different quantities but share one instruction stream where they can (a warp runs
         // both sides of a branch one after the other):
@@ -1541,8 +1527,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mbar_arrive(&bar_st1);
     }
     if (ok && !full) {   // ragged tail: rows beyond the sequence must not be written
-        flush_rows(sm + STG_A, gdq, rowp, x.len, kIntraThreads);
-        flush_rows(sm + STG_B, gdv, rowp, x.len, kIntraThreads);
+        flush_rows(sm + STG_A, grad_rows(p.dq), (size_t)H * D, x.len, kIntraThreads);
+        flush_rows(sm + STG_B, grad_rows(p.dv), (size_t)H * D, x.len, kIntraThreads);
     }
     GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
@@ -1632,7 +1618,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     cta_sync();
     GDN_TICK(2, 14);
     if (threadIdx.x == 32) mbar_arrive(&bar_st2);   // dk is staged: the loader stores it
-    if (ok && !full) flush_rows(sm + STG_K, gdk, rowp, x.len, kIntraThreads);
+    if (ok && !full) flush_rows(sm + STG_K, grad_rows(p.dk), (size_t)H * D, x.len, kIntraThreads);
     // The token-wise sums are complete; turning them into dbeta and dg is left to warps 0 and 1 during the next trip's
     // first products (finish_gates).  They keep what the next trip overwrites: this chunk's gates and place.
     if (threadIdx.x < kC) { bb_prev = bb[threadIdx.x]; Gam_last_prev = Gam[kC - 1]; }
