@@ -930,14 +930,14 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
 #pragma unroll
         for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
         if (len < kC) {   // ragged tail: the K rows beyond the sequence belong to somebody else
-            ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
+            ok = mbar_wait_inline(&bar_full[stage], (s / STAGES) & 1);
             if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 12); break; }
             zero_tail_rows(ring + KT, 64, 0, len, kThreads);
         }
         fence_async_smem();
         __syncthreads();
         if (threadIdx.x == 0) {
-            ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
+            ok = mbar_wait_inline(&bar_full[stage], (s / STAGES) & 1);
             if (ok) {
                 tc_fence_after();
                 // forward (W h)^T = h^T W^T ; reverse (K dh')^T = dh'^T K^T : [d_v][tokens]
@@ -953,8 +953,8 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         } else if (threadIdx.x == 32) {
             if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
         }
-        ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
-        if (ok) ok = mbar_wait(&bar_mma, mma_phase);
+        ok = mbar_wait_inline(&bar_full[stage], (s / STAGES) & 1);
+        if (ok) ok = mbar_wait_inline(&bar_mma, mma_phase);
         mma_phase ^= 1;
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 11); break; }
         tc_fence_after();
@@ -983,7 +983,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
             ee2[(s + 1) & 1][threadIdx.x] = expf(gend_next - gnext);
             if (s + 2 < nsteps) { gnext = gate_row(s + 2)[threadIdx.x]; gend_next = gate_row(s + 2)[kC - 1]; }
         }
-        ok = mbar_wait(&bar_mma, mma_phase);
+        ok = mbar_wait_inline(&bar_mma, mma_phase);
         mma_phase ^= 1;
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 13); break; }
         tc_fence_after();

@@ -12,6 +12,7 @@
 //             dgamma_i = <q_i,dq_i> - <k_i,dk_i>,  dgamma_63 += sum_j r_j + Gam_e <dh',h>,  dg = reverse cumsum.
 // Accumulators are 64 x 64 (M = 64: row i on TMEM lane i % 16 + 32 (i / 16)), token rows on lanes, so a thread owns
 // a token row: row dots are thread-local and gradient rows leave with 16-byte stores.  Two CTAs share an SM.
+#define GDN_INLINE_WAIT   // small kernels: the polling loops sit at the wait sites (see tc_ptx.cuh)
 #include "tc_common.cuh"
 
 namespace gdn {

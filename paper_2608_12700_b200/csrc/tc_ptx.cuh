@@ -69,8 +69,27 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
         if (global_ns() - t0 > 2000000000ull) return false;
     }
 }
+// The same wait with its polling loop at the wait site: no call, so nothing has to be saved around it.  For the small
+// kernels (the carries, the scalar-gate passes), where code size does not matter and a step is short.
+__device__ __forceinline__ bool mbar_wait_inline(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    uint64_t t0 = 0;
+#pragma unroll 1
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0) {
+            const uint64_t t = global_ns();
+            if (t0 == 0) t0 = t;
+            else if (t - t0 > 2000000000ull) return false;
+        }
+    }
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+#ifdef GDN_INLINE_WAIT
+    return mbar_wait_inline(bar, parity);
+#else
     return mbar_try_wait(bar, parity) || mbar_wait_slow(bar, parity);
+#endif
 }
 
 // ---------------------------------------------------------------- proxies and copies
