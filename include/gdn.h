@@ -124,7 +124,7 @@ const char* gdn_kernel_path(const gdn_desc* desc);
  * GPU that loads it, for the life of the process.  The call allocates and frees nothing.
  *   - Problems whose gdn_workspace_bytes() backward size exceeds GDN_NOALLOC_WORKSPACE_BYTES are refused
  *     with GDN_ERR_WORKSPACE_TOO_SMALL before anything is launched (at bf16, d_k = d_v = 128 the limit is
- *     about 160 chunk-heads, e.g. H = 4 and 2560 tokens).
+ *     about 155 chunk-heads, e.g. H = 4 and 2304 tokens).
  *   - The first call on a device looks up the array's device address (one-time set-up on the host); make
  *     that first call outside of any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents.  The call
