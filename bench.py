@@ -256,13 +256,16 @@ def stage_algorithmic_work(stage, wl, io_bytes, family=""):
         ndir = 2 if stage == "scans" else 1
         return ndir * chd * (dk * dk + 2 * dk * dv) * io_bytes, ndir * chd * 2.0 * dk * dk * dv
     if stage == "prep":
-        return th * ((dk + dv) * io_bytes + 4 * gates), chd * (2 * tri_k + tri_v + 2 * dense + 2 * 64 ** 3 / 3)
+        n_tri = 3 if family == "tcgen05_bf16" else 2
+        return th * ((dk + dv) * io_bytes + 4 * gates), chd * (n_tri * tri_k + tri_v + 2 * dense + 2 * 64 ** 3 / 3)
     if stage == "eprep":
         return th * ((2 * dk + dv) * io_bytes), chd * (2 * tri_k + dense)
     # intra (or a fused gradient stage): streams every input and writes every gradient
     byts = benchutil.path_alg_bytes(token_heads=th, chains=chains, d_k=dk, d_v=dv, io_bytes=io_bytes,
                                     delta_rule=wl.delta_rule, has_h0=False, has_dhT=False, writes_dh0=False)
-    flops = chd * ((7 * tri_k + 5 * tri_v + 5 * dense) if wl.delta_rule else (3 * tri_k + 2 * tri_v + 3 * dense))
+    # (in the tcgen05 d = 128 family P = tril(Q K^T . D) is formed by the prep stage and handed over: counted there)
+    n_tri_k = 6 if family == "tcgen05_bf16" else 7
+    flops = chd * ((n_tri_k * tri_k + 5 * tri_v + 5 * dense) if wl.delta_rule else (3 * tri_k + 2 * tri_v + 3 * dense))
     return byts, flops
 
 
