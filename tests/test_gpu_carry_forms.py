@@ -81,3 +81,17 @@ def test_many_chains_choose_the_low_rank_form_by_themselves():
         binding.gdn_debug_force_family(0)
     for name in ("dq", "dk", "dv", "dg", "dbeta", "dh0"):
         assert np.array_equal(auto[name], forced[name]), name
+
+
+def test_many_short_ragged_sequences_in_low_rank_form():
+    """80 chains of 1 to 200 tokens: most chunks are ragged tails, many chains have a single step."""
+    rng = np.random.default_rng(48)
+    lengths = [int(x) for x in rng.integers(1, 201, size=40)]
+    lengths[3], lengths[17] = 1, 64
+    wl = synth.make_workload("carry_short", dtype="bf16", lengths=lengths, H=2, d_k=128, d_v=128, states=True, seed=48)
+    check_against_oracle(wl, runner.backward(wl))
+    buf = runner.to_device(wl, want_o=True)
+    runner.run_fwd(buf)
+    got, ref = runner.fetch(buf), oracle_grads(wl)
+    assert rel(got["o"], ref["o"]) < TOL["bf16"]
+    assert rel(got["hT"], ref["hT"]) < TOL["bf16"]
