@@ -17,6 +17,7 @@ CASES = {
     "equal_lengths": dict(B=2, T=256, H=3, states=True, seed=42),
     "short_sequences_no_states": dict(lengths=[1, 63, 65, 130], H=1, states=False, seed=43),
     "one_long_chain": dict(B=1, T=1100, H=1, states=True, seed=44),
+    "with_empty_sequences": dict(lengths=[0, 70, 0, 130, 64, 0], H=2, states=True, seed=49),
 }
 
 
