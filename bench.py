@@ -35,6 +35,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used when profiling)")
+    ap.add_argument("--no-others", action="store_true", help="skip the save-forward arm and the other configurations")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
     return ap.parse_args()
 
@@ -89,6 +90,45 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def time_steps(fn, steps, barrier, stream):
+    """Device time of `steps` back-to-back calls of fn, nothing but the calls between the two events."""
+    import torch
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for _ in range(steps):
+        fn()
+    ev1.record(stream)
+    barrier()
+    return ev0.elapsed_time(ev1)
+
+
+def path_roofline(wl, peaks, ms_per_step):
+    from paper_2608_12700_b200 import benchutil
+    io_bytes = 2 if wl.dtype == "bf16" else 4
+    alg_bytes = benchutil.path_alg_bytes(token_heads=wl.T_total * wl.H, chains=wl.N * wl.H, d_k=wl.d_k, d_v=wl.d_v,
+                                         io_bytes=io_bytes, delta_rule=wl.delta_rule, has_h0=wl.h0 is not None,
+                                         has_dhT=wl.dhT is not None)
+    alg_flops = benchutil.path_alg_flops(chunk_heads=wl.n_chunks() * wl.H, d_k=wl.d_k, d_v=wl.d_v, delta_rule=wl.delta_rule)
+    t_hbm, t_tc = benchutil.roofline_times(alg_bytes, alg_flops, peaks, sustained=False)
+    return dict(algorithmic_bytes=alg_bytes, algorithmic_flops=alg_flops, t_hbm_us=t_hbm * 1e6, t_tensor_us=t_tc * 1e6,
+                bound="hbm" if t_hbm >= t_tc else "tensor", frac=max(t_hbm, t_tc) / (ms_per_step * 1e-3),
+                peak_source=peaks["source"])
+
+
+def stage_pass(buf, runner, binding, calls):
+    """Per-kernel durations from a separate, untimed-for-the-headline pass: every launch bracketed by events."""
+    import torch
+    binding.gdn_stage_timing_enable(1)
+    binding.gdn_stage_timing_read()
+    for _ in range(calls):
+        runner.run_bwd(buf)
+    torch.cuda.synchronize()
+    stages = binding.gdn_stage_timing_read()
+    binding.gdn_stage_timing_enable(False)
+    return {k: v[0] / v[1] for k, v in stages.items() if v[1] > 0}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -115,45 +155,50 @@ def run_ours(args):
     desc = buf.desc
     peaks = benchutil.load_peaks(ROOT)
     stream = torch.cuda.current_stream()
+    warmup = max(3, args.warmup)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---------------- device-resident timing ----------------
-    for _ in range(max(3, args.warmup)):
+    def check_status(b, where):
+        st = binding.gdn_last_device_status(b.workspace)
+        if st != binding.GDN_OK:
+            raise binding.GdnError(st, where)
+
+    # ---------------- device-resident timing: nothing but the K calls between the two events ----------------
+    for _ in range(warmup):
         runner.run_bwd(buf)
-    st = binding.gdn_last_device_status(buf.workspace)
-    if st != binding.GDN_OK:
-        raise binding.GdnError(st, "warm-up")
-    sampler = benchutil.ClockSampler(local)
-    # per-kernel durations are sampled inside the timed region: the kernels of every `period`-th step are bracketed
-    # by events (an event between two kernels costs the stream a few microseconds; bracketing every launch slows a
-    # 0.35 ms step by 5 %)
-    period = max(1, args.steps // 12)
-    binding.gdn_stage_timing_enable(period)
-    binding.gdn_stage_timing_read()
+    check_status(buf, "warm-up")
+    sampler = benchutil.ClockSampler(local, period_s=0.0005)
     launches0 = binding.gdn_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     sampler.start()
-    ev0.record(stream)
-    for _ in range(args.steps):
-        runner.run_bwd(buf)
-    ev1.record(stream)
-    barrier()
+    elapsed_ms = time_steps(lambda: runner.run_bwd(buf), args.steps, barrier, stream)
     sampler.stop()
-    elapsed_ms = ev0.elapsed_time(ev1)
     launches = binding.gdn_launch_count() - launches0
-    stages = binding.gdn_stage_timing_read()
-    binding.gdn_stage_timing_enable(False)
-    st = binding.gdn_last_device_status(buf.workspace)
-    if st != binding.GDN_OK:
-        raise binding.GdnError(st, "timed region")
+    check_status(buf, "timed region")
     elapsed_ms, tokens_all = benchutil.aggregate_over_ranks(elapsed_ms, wl.tokens * args.steps, dist if world > 1 else None, dev)
     value = tokens_all / (elapsed_ms * 1e-3)
     ms_per_step = elapsed_ms / args.steps
+
+    # ---------------- per-kernel durations: a pass of its own, outside the headline ----------------
+    stage_calls = max(3, min(args.steps, 10))
+    stage_ms = stage_pass(buf, runner, binding, stage_calls)
+
+    # ---------------- the arm that consumes a workspace saved by the forward (Section 4.5) ----------------
+    save_forward = None
+    if world == 1 and not args.no_others:
+        runner.run_fwd(buf)
+        for _ in range(warmup):
+            runner.run_bwd(buf, fresh=1)
+        sf_steps = max(3, min(args.steps, 20))
+        sf_ms = time_steps(lambda: runner.run_bwd(buf, fresh=1), sf_steps, barrier, stream) / sf_steps
+        fw_ms = time_steps(lambda: runner.run_fwd(buf), sf_steps, barrier, stream) / sf_steps
+        check_status(buf, "save-forward arm")
+        save_forward = {"ms_per_step": sf_ms, "tokens_per_s": wl.tokens / (sf_ms * 1e-3), "steps": sf_steps,
+                        "gdn_fwd_recompute_ms": fw_ms,
+                        "what": "gdn_bwd with workspace_is_fresh_from_fwd=1 on a workspace filled by gdn_fwd_recompute"}
 
     # ---------------- end to end: host buffers in, host buffers out ----------------
     # (the public host-buffer call: pinned host tensors in, pinned host tensors out; uploads, kernels and downloads of
@@ -161,76 +206,101 @@ def run_ours(args):
     host = None if args.no_e2e else runner.HostBackward(wl, dev)
     h2d = host.h2d_bytes if host else 0
     d2h = host.d2h_bytes if host else 0
-
-    def e2e_step():
-        host.step()
-
     e2e_steps = 0 if args.no_e2e else max(3, min(args.steps, 10))
     for _ in range(2 if e2e_steps else 0):
-        e2e_step()
-    barrier()
-    ev0.record(stream)
-    for _ in range(e2e_steps):
-        e2e_step()
-    ev1.record(stream)
-    barrier()
+        host.step()
+    e2e_raw = time_steps(host.step, e2e_steps, barrier, stream) if e2e_steps else 0.0
     if host:
         host.check()
-    e2e_ms, e2e_tokens = benchutil.aggregate_over_ranks(ev0.elapsed_time(ev1), wl.tokens * e2e_steps, dist if world > 1 else None, dev)
+    e2e_ms, e2e_tokens = benchutil.aggregate_over_ranks(e2e_raw, wl.tokens * e2e_steps, dist if world > 1 else None, dev)
     e2e_value = e2e_tokens / (e2e_ms * 1e-3) if e2e_steps else None
+    del host
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # ---------------- roofline ----------------
+    # ---------------- roofline: the whole path against its bound, the dominant kernel beside it ----------------
     io_bytes = 2 if wl.dtype == "bf16" else 4
-    token_heads, chains, chunk_heads = wl.T_total * wl.H, wl.N * wl.H, wl.n_chunks() * wl.H
-    alg_bytes = benchutil.path_alg_bytes(token_heads=token_heads, chains=chains, d_k=wl.d_k, d_v=wl.d_v, io_bytes=io_bytes,
-                                         delta_rule=wl.delta_rule, has_h0=wl.h0 is not None, has_dhT=wl.dhT is not None)
-    alg_flops = benchutil.path_alg_flops(chunk_heads=chunk_heads, d_k=wl.d_k, d_v=wl.d_v, delta_rule=wl.delta_rule)
-    t_hbm, t_tc = benchutil.roofline_times(alg_bytes, alg_flops, peaks, sustained=False)
-    stage_ms = {k: v[0] / max(1, v[1]) for k, v in stages.items() if v[1] > 0}
-    dom = max(stage_ms, key=stage_ms.get)
-    # The dominant kernel is charged with the whole path's algorithmic work when it is the kernel that
-    # streams the inputs and writes the gradients (the intra / fused gradient stage); a scan stage is
-    # charged with the state traffic it cannot avoid.  Stated per stage in the design doc.
-    dom_bytes, dom_flops = stage_algorithmic_work(dom, wl, io_bytes, binding.gdn_kernel_path(desc))
-    d_hbm, d_tc = benchutil.roofline_times(dom_bytes, dom_flops, peaks, sustained=False)
-    dom_s = stage_ms[dom] * 1e-3
-    if d_hbm >= d_tc:
-        roof = {"bound": "hbm", "achieved": dom_bytes / dom_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    family = binding.gdn_kernel_path(desc)
+    path = path_roofline(wl, peaks, ms_per_step)
+    step_s = ms_per_step * 1e-3
+    if path["bound"] == "hbm":
+        roof = {"bound": "hbm", "achieved": path["algorithmic_bytes"] / step_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     else:
-        roof = {"bound": "tensor", "achieved": dom_flops / dom_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        roof = {"bound": "tensor", "achieved": path["algorithmic_flops"] / step_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = recorded_traffic(dom, wl)
-    roof.update({"kernel": dom, "kernel_ms": stage_ms[dom], "peak_source": peaks["source"],
-                 "algorithmic_bytes": dom_bytes, "algorithmic_flops": dom_flops})
-    path_roof_s = max(t_hbm, t_tc)
+    traffic = [recorded_traffic(k, wl, family) for k in stage_ms]
+    roof["traffic"] = sum(traffic) if traffic and all(t is not None for t in traffic) else None
+    roof["traffic_over_algorithmic"] = roof["traffic"] / path["algorithmic_bytes"] if roof["traffic"] else None
+    dom = max(stage_ms, key=stage_ms.get)
+    dom_bytes, dom_flops = stage_algorithmic_work(dom, wl, io_bytes, family)
+    d_hbm, d_tc = benchutil.roofline_times(dom_bytes, dom_flops, peaks, sustained=False)
+    roof.update({
+        "scope": "whole gdn_bwd call (all kernels of a step): algorithmic bytes of the path / ms_per_step; this is the "
+                 "fraction the 50 % target is stated on",
+        "peak_source": peaks["source"], "algorithmic_bytes": path["algorithmic_bytes"],
+        "algorithmic_flops": path["algorithmic_flops"],
+        "kernel": dom, "kernel_ms": stage_ms[dom], "kernel_algorithmic_bytes": dom_bytes,
+        "kernel_algorithmic_flops": dom_flops, "kernel_traffic": recorded_traffic(dom, wl, family),
+        "kernel_frac": max(d_hbm, d_tc) / (stage_ms[dom] * 1e-3),
+        "kernel_bound": "hbm" if d_hbm >= d_tc else "tensor"})
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
         "config": workload_config(wl),
-        "kernel_path": binding.gdn_kernel_path(desc),
+        "kernel_path": family,
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / max(1, e2e_steps), "steps": e2e_steps},
         "gpu_launches": launches,
         "roofline": roof,
-        "path_roofline": {"algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops, "t_hbm_us": t_hbm * 1e6,
-                          "t_tensor_us": t_tc * 1e6, "bound": "hbm" if t_hbm >= t_tc else "tensor",
-                          "frac": path_roof_s / (ms_per_step * 1e-3), "peak_source": peaks["source"]},
+        "path_roofline": path,
         "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()},
-        "stage_timed_steps": max(v[1] for v in stages.values()),
+        "stage_timed_calls": stage_calls,
     }
+    if save_forward:
+        line["save_forward_arm"] = save_forward
+    del buf
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_others:
+        line["other_configs"] = time_other_configs(args, peaks, barrier, stream, dev)
     if not args.no_cpu_baseline and world == 1:
         v, cores, sample, used = time_oracle_sample(wl, args.cpu_seconds)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_other_configs(args, peaks, barrier, stream, dev):
+    """The other benchmark configurations, briefly (device-resident, same protocol as the headline), so that their
+    figures come from the same run on the same machine.  Not bench lines of their own."""
+    import torch
+    from paper_2608_12700_b200 import binding, runner, synth
+    out = {}
+    for idx in range(5):
+        if idx == args.config:
+            continue
+        wl = synth.config(idx)
+        buf = runner.to_device(wl, dev)
+        for _ in range(3):
+            runner.run_bwd(buf)
+        steps = 20 if idx == 0 else 10
+        ms = time_steps(lambda: runner.run_bwd(buf), steps, barrier, stream) / steps
+        st = binding.gdn_last_device_status(buf.workspace)
+        if st != binding.GDN_OK:
+            raise binding.GdnError(st, wl.name)
+        pr = path_roofline(wl, peaks, ms)
+        stage_ms = stage_pass(buf, runner, binding, 3)
+        out[wl.name] = {"ms_per_step": ms, "tokens_per_s": wl.tokens / (ms * 1e-3), "steps": steps, "tokens": wl.tokens,
+                        "path_frac": pr["frac"], "path_bound": pr["bound"], "kernel_path": binding.gdn_kernel_path(buf.desc),
+                        "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()}}
+        del buf, wl
+        torch.cuda.empty_cache()
+    return out
 
 
 def stage_algorithmic_work(stage, wl, io_bytes, family=""):
@@ -269,15 +339,22 @@ def stage_algorithmic_work(stage, wl, io_bytes, family=""):
     return byts, flops
 
 
-def recorded_traffic(stage, wl):
+def recorded_traffic(stage, wl, family=""):
     """DRAM bytes per launch of the stage from the ncu captures summarised under profiles/ (bytes per
     chunk-head measured on a small case, scaled by the chunk-heads of this workload), or None."""
-    path = os.path.join(ROOT, "paper_2608_12700_b200", "measured_traffic.json")
+    path = os.path.join(ROOT, "profiles", "measured_traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         rec = json.load(f)
     key = f"{stage}:{wl.dtype}:{wl.d_k}x{wl.d_v}:{wl.delta_rule}"
+    if family == "tcgen05_bf16" and stage in ("prep", "scans"):
+        from paper_2608_12700_b200 import binding, runner
+        # the d = 128 family runs its carries in one of two forms with different traffic; the workspace size tells which
+        desc = runner.desc_for(wl)
+        per_ch = binding.gdn_workspace_bytes(desc)[1] / max(1, (wl.T_total // 64 + wl.N) * wl.H)
+        if per_ch < 180 * 1024:
+            key = f"{stage}_low_rank:{wl.dtype}:{wl.d_k}x{wl.d_v}:{wl.delta_rule}"
     if key not in rec:
         return None
     return rec[key]["bytes_per_chunk_head"] * wl.n_chunks() * wl.H

@@ -72,7 +72,9 @@ typedef struct gdn_desc {
 } gdn_desc;
 
 /* Bytes of workspace needed by gdn_fwd_recompute (*fwd_bytes) and by gdn_bwd (*bwd_bytes >= *fwd_bytes;
- * the forward's workspace is a prefix of the backward's).  Either output pointer may be NULL. */
+ * the forward's workspace is a prefix of the backward's).  Either output pointer may be NULL.  Host-only
+ * bookkeeping of this library (the paper has no counterpart): the workspace holds the chunk table, the
+ * chunk-local factors of Section 4.2 and the per-chunk states between the stages. */
 gdn_status gdn_workspace_bytes(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
 
 /* Recompute stage of the backward (Section 4.2, "chunking"): chunk table, chunk-local cumulative decay,
@@ -104,10 +106,11 @@ gdn_status gdn_bwd(const gdn_desc* desc,
 
 /* Synchronises the stream, reads the device-side status word of the last call that used `workspace`
  * and returns it (GDN_OK, GDN_ERR_BAD_SEQLENS or GDN_ERR_DEVICE_TIMEOUT; GDN_ERR_CUDA if the stream
- * itself reports an error). */
+ * itself reports an error).  Error reporting of this library (the paper has no counterpart).  After
+ * a device-side error the kernels of that call stop early and leave the outputs unwritten. */
 gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream);
 
-/* Static, NUL-terminated description of a status code. */
+/* Static, NUL-terminated description of a status code (the paper has no counterpart). */
 const char* gdn_status_string(gdn_status s);
 
 /* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16",
@@ -124,15 +127,18 @@ const char* gdn_kernel_path(const gdn_desc* desc);
  * GPU that loads it, for the life of the process.  The call allocates and frees nothing.
  *   - Problems whose gdn_workspace_bytes() backward size exceeds GDN_NOALLOC_WORKSPACE_BYTES are refused
  *     with GDN_ERR_WORKSPACE_TOO_SMALL before anything is launched (at bf16, d_k = d_v = 128 the limit is
- *     about 155 chunk-heads, e.g. H = 4 and 2304 tokens).
+ *     about 225 chunk-heads, e.g. H = 4 and 3456 tokens).
  *   - The first call on a device looks up the array's device address (one-time set-up on the host); make
  *     that first call outside of any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents.  The call
  *     clears the part that must start from zero itself.  Two calls that overlap on the GPU (different
  *     streams, or a second call enqueued before the first has finished on another stream) race on it:
  *     keep such calls on one stream or synchronise between them.
- *   - Conditions that only the device can see (malformed cu_seqlens) are not reported by this variant;
- *     use gdn_bwd with gdn_last_device_status where that matters. */
+ *   - Conditions that only the device can see (malformed cu_seqlens contents, a bounded device-side wait
+ *     that ran out) make the kernels stop early: the call has returned GDN_OK by then and the outputs
+ *     stay unwritten.  gdn_noalloc_last_device_status(stream) synchronises the stream and returns the
+ *     status word the last gdn_bwd_noalloc on the current device left in the built-in scratch (GDN_OK,
+ *     GDN_ERR_BAD_SEQLENS or GDN_ERR_DEVICE_TIMEOUT); it allocates nothing either. */
 #define GDN_NOALLOC_WORKSPACE_BYTES (32u * 1024u * 1024u)
 gdn_status gdn_bwd_noalloc(const gdn_desc* desc,
                            const void* q, const void* k, const void* v,
@@ -141,6 +147,7 @@ gdn_status gdn_bwd_noalloc(const gdn_desc* desc,
                            const int32_t* cu_seqlens_dev,
                            void* dq, void* dk, void* dv, float* dg, float* dbeta, float* dh0,
                            void* cuda_stream);
+gdn_status gdn_noalloc_last_device_status(void* cuda_stream);
 
 /* ---- measurement hooks (not part of the method; the paper has no counterpart) -------------------
  * gdn_launch_count: number of kernels this library has launched in this process.
@@ -165,8 +172,9 @@ gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* l
  * gdn_debug_force_family: 0 = automatic dispatch, 1 = always use the FFMA kernels (tests use this to
  * exercise both families on the same inputs); 2 / 3 = automatic family, but the tcgen05 d = 128 kernels carry the
  * state across chunks in operator form (one d x d matrix per chunk) / in low-rank form (two dependent products
- * per chunk, no such matrix), whatever the shape; by default the shape decides.  Process-wide; 1 affects workspace
- * sizes as well. */
+ * per chunk, no such matrix), whatever the shape; by default the shape decides.  The setting belongs to the
+ * calling thread (other threads keep automatic dispatch) and changes what gdn_workspace_bytes returns to that thread,
+ * so size the workspace after setting it. */
 gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
                           float* host_out);
 gdn_status gdn_debug_force_family(int32_t family);

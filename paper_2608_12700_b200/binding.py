@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
-           "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc"]
+           "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc",
+           "gdn_noalloc_last_device_status"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -71,6 +72,8 @@ def lib():
         L.gdn_stage_timing_read.argtypes = [I, P, P, P, P]
         L.gdn_bwd_noalloc.restype = I
         L.gdn_bwd_noalloc.argtypes = [D] + [P] * 15 + [P]
+        L.gdn_noalloc_last_device_status.restype = I
+        L.gdn_noalloc_last_device_status.argtypes = [P]
         L.gdn_debug_read.restype = I
         L.gdn_debug_read.argtypes = [D, P, ctypes.c_char_p, I, I, P]
         L.gdn_debug_force_family.restype = I
@@ -200,3 +203,8 @@ def gdn_bwd_noalloc(desc, q, k, v, g, beta, h0, dO, dhT, cu_seqlens, dq, dk, dv,
     if check and s != GDN_OK:
         raise GdnError(s, "gdn_bwd_noalloc")
     return s
+
+
+def gdn_noalloc_last_device_status(stream=None) -> int:
+    """Device-side status of the last gdn_bwd_noalloc on the current device (synchronises the stream)."""
+    return lib().gdn_noalloc_last_device_status(_stream(stream))

@@ -18,12 +18,26 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
+STAMP = LIB + ".stamp"   # digest of everything the library was built from
+
+
+def _digest() -> str:
+    """Content hash of sources, headers and flags: the library is rebuilt whenever any of them differs from what it
+    was built from (file times say nothing after a checkout or a copy to another machine)."""
+    import hashlib
+    h = hashlib.sha256(" ".join(NVCC_FLAGS[:6]).encode())
+    for d in sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(INCLUDE, "*.h"))):
+        h.update(os.path.basename(d).encode())
+        with open(d, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB):
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(INCLUDE, "*.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    with open(STAMP) as f:
+        return f.read().strip() != _digest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -44,6 +58,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs)
     os.replace(tmp, LIB)
+    with open(STAMP, "w") as f:
+        f.write(_digest() + "\n")
     return LIB
 
 

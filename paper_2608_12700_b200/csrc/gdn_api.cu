@@ -49,9 +49,11 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 enum class Path { None, SimtF32, SimtBf16, TcBf16, Tc64Bf16 };
 
-int g_force_family = 0;
+// Debug overrides of the dispatch are per thread: a thread that forces a family cannot change the workspace size
+// another thread is computing at that moment.
+thread_local int g_force_family = 0;
 }  // namespace
-int g_force_carries = 0;   // tcgen05 d = 128 family: 0 = by shape, 1 = operator form (Nm, Bf), 2 = low-rank form
+thread_local int g_force_carries = 0;   // tcgen05 d = 128 family: 0 = by shape, 1 = operator form (Nm, Bf), 2 = low-rank form
 namespace {
 
 Path pick_path(const gdn_desc& d) {
@@ -78,7 +80,9 @@ gdn_status check_desc(const gdn_desc* d) {
 
 WsLayout layout_for(const gdn_desc& d) {
     // tcgen05 path: every factor, state and additive term of the carries is a bf16 tile image.
-    if (pick_path(d) == Path::TcBf16 || pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
+    // The d = 128 family keeps the chunk operator Nm and the additive term Bf only when its carries use them.
+    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0, !tc_carries_lowrank(d));
+    if (pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
     return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
 }
@@ -91,6 +95,24 @@ gdn_status check_seq(const gdn_desc& d, const int32_t* cu) {
 }
 
 }  // namespace
+}  // namespace gdn
+
+namespace gdn {
+gdn_status check_bwd_args(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const float* h0, const void* dO, const float* dhT, const int32_t* cu, void* dq, void* dk, void* dv,
+                          float* dg, float* dbeta, float* dh0, const void* workspace, size_t workspace_bytes) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
+    const bool empty = (long long)desc->B * desc->T == 0;   // no tokens: token tensors may be NULL
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    if (!empty && (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg)) return GDN_ERR_NULL_ARG;
+    if (!empty && desc->delta_rule && (!beta || !dbeta)) return GDN_ERR_NULL_ARG;
+    const void* ptrs[] = {q, k, v, g, beta, h0, dO, dhT, cu, dq, dk, dv, dg, dbeta, dh0, workspace};
+    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
+    if (workspace_bytes < layout_for(*desc).total) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    return GDN_OK;
+}
 }  // namespace gdn
 
 using namespace gdn;
@@ -137,20 +159,12 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
                    float* dg, float* dbeta, float* dh0, void* workspace, size_t workspace_bytes,
                    int32_t workspace_is_fresh_from_fwd, void* cuda_stream) {
     call_begin();
-    gdn_status s = check_desc(desc);
+    const gdn_status s = check_bwd_args(desc, q, k, v, g, beta, h0, dO, dhT, cu, dq, dk, dv, dg, dbeta, dh0, workspace, workspace_bytes);
     if (s != GDN_OK) return s;
-    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
-    const bool empty = (long long)desc->B * desc->T == 0;   // no tokens: token tensors may be NULL
-    if (!workspace) return GDN_ERR_NULL_ARG;
-    if (!empty && (!q || !k || !v || !g || !dO || !dq || !dk || !dv || !dg)) return GDN_ERR_NULL_ARG;
-    if (!empty && desc->delta_rule && (!beta || !dbeta)) return GDN_ERR_NULL_ARG;
-    const void* ptrs[] = {q, k, v, g, beta, h0, dO, dhT, cu, dq, dk, dv, dg, dbeta, dh0, workspace};
-    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
     Problem p{};
     p.d = *desc;
     p.Ttot = desc->B * desc->T;
     p.L = layout_for(*desc);
-    if (workspace_bytes < p.L.total) return GDN_ERR_WORKSPACE_TOO_SMALL;
     p.q = q; p.k = k; p.v = v; p.g = g; p.beta = beta; p.h0 = h0; p.dO = dO; p.dhT = dhT; p.cu = cu;
     p.dq = dq; p.dk = dk; p.dv = dv; p.dg = dg; p.dbeta = dbeta; p.dh0 = dh0;
     p.ws = static_cast<char*>(workspace);
@@ -213,6 +227,8 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
     const Q* q = nullptr;
     for (const Q& t : table) if (strcmp(t.name, what) == 0) q = &t;
     if (!q) return GDN_ERR_BAD_SHAPE;
+    if (!L.has_operator && (q->off == L.Nm || q->off == L.Bf) && (strcmp(what, "Nm") == 0 || strcmp(what, "Bf") == 0))
+        return GDN_ERR_BAD_SHAPE;   // not stored: the carries of this descriptor run in low-rank form
     if (cudaDeviceSynchronize() != cudaSuccess) return GDN_ERR_CUDA;
     const size_t n = (size_t)q->rows * q->cols;
     const char* base = static_cast<const char*>(workspace) + q->off;

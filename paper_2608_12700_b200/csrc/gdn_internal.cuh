@@ -31,8 +31,9 @@ struct WsLayout {
     size_t Tm;             // f32|bf16 [CH, 64, 64]    T = (I + A)^-1
     size_t W;              // [CH, 64, d_k]
     size_t Ut;             // [CH, 64, d_v]            U~ = T Diag(w) V
-    size_t Nm;             // [CH, d_k, d_k]           Kb^T W
-    size_t Bf;             // [CH, d_k, d_v]           Kb^T U~
+    size_t Nm;             // [CH, d_k, d_k]           Kb^T W        (these two only when the carries run in operator
+    size_t Bf;             // [CH, d_k, d_v]           Kb^T U~        form: has_operator; otherwise they take no space)
+    int has_operator;
     size_t hc;             // [CH, d_k, d_v]           state entering the chunk
     size_t fwd_end;        // bytes needed by the forward recompute
     size_t E;              // [CH, d_k, d_v]           scale (Gam Q - P W)^T dO
@@ -47,7 +48,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // elem = bytes per element of the chunk factors and stored states (T, W, U~, Nm, hc, dhn): 4 on the fp32
 // path, 2 for the bf16 tile images of the tcgen05 path.  elem_add = bytes per element of Bf and E.
-inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, size_t scratch_per_ch) {
+inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, size_t scratch_per_ch, bool with_operator = true) {
     WsLayout L{};
     const size_t Ttot = (size_t)d.B * (size_t)d.T;
     L.max_chunks = (int)((Ttot + kC - 1) / kC + (size_t)d.N);
@@ -62,8 +63,9 @@ inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, siz
     L.Tm = take(elem * CH * kC * kC);
     L.W = take(elem * CH * kC * d.d_k);
     L.Ut = take(elem * CH * kC * d.d_v);
-    L.Nm = take(elem * CH * d.d_k * d.d_k);
-    L.Bf = take(elem_add * CH * d.d_k * d.d_v);
+    L.has_operator = with_operator ? 1 : 0;
+    L.Nm = take(with_operator ? elem * CH * d.d_k * d.d_k : 0);
+    L.Bf = take(with_operator ? elem_add * CH * d.d_k * d.d_v : 0);
     L.hc = take(elem * CH * d.d_k * d.d_v);
     L.fwd_end = o;
     L.E = take(elem_add * CH * d.d_k * d.d_v);
@@ -115,6 +117,12 @@ struct SmemLimitOnce {
     }
 };
 
+// Host-side argument checks of gdn_bwd (everything that can be refused before a launch), shared with the entry point
+// that brings its own workspace.
+gdn_status check_bwd_args(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
+                          const float* h0, const void* dO, const float* dhT, const int32_t* cu, void* dq, void* dk, void* dv,
+                          float* dg, float* dbeta, float* dh0, const void* workspace, size_t workspace_bytes);
+
 // Kernel families (each defined in its own translation unit).  They enqueue on `st` and return the
 // first CUDA error seen.
 cudaError_t launch_table(const Problem& p, cudaStream_t st);
@@ -123,8 +131,11 @@ cudaError_t simt_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t 
 size_t simt_scratch_per_chunkhead(const gdn_desc& d);
 
 // tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
-extern int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank form
+extern thread_local int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank
 bool tc_supported(const gdn_desc& d);
+// Form of the carries for a descriptor: one rule for the forward, the backward and a backward that consumes a workspace
+// fresh from the forward, so that the layout of a workspace does not depend on which call sized it.
+bool tc_carries_lowrank(const gdn_desc& d);
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 

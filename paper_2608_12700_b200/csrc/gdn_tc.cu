@@ -22,27 +22,6 @@
 
 namespace gdn {
 
-// Optional phase timing (compile with -DGDN_PHASE_TIMING): thread 0 of CTA 0 stamps clock64() at phase borders.
-#ifdef GDN_PHASE_TIMING
-__device__ long long g_ticks[4][32];
-__device__ int g_tick_trip = 0;   // which trip of a persistent CTA is stamped
-__device__ int g_trip_now = 0;
-__device__ long long g_sync[16][18];   // intra: arrival time of every warp at each named barrier of one trip, [17] = release
-__device__ long long g_trip_ns[2][24];   // wall-clock (ns) at kernel entry [0], at each trip start [1 + trip], at exit
-__device__ __forceinline__ long long tick_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define GDN_TRIP(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (idx) < 24) g_trip_ns[kern][idx] = tick_ns(); } while (0)
-#ifdef GDN_NO_TICKS   // barrier arrival times only: the phase stamps would delay thread 0
-#define GDN_TICK(kern, idx) do { } while (0)
-#define GDN_TICKT(tid, kern, idx) do { } while (0)
-#else
-#define GDN_TICK(kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && (kern != 2 || g_trip_now == g_tick_trip)) g_ticks[kern][idx] = clock64(); } while (0)
-#define GDN_TICKT(tid, kern, idx) do { if (blockIdx.x == 0 && threadIdx.x == (tid)) g_ticks[kern][idx] = clock64(); } while (0)
-#endif
-#else
-#define GDN_TICK(kern, idx) do { } while (0)
-#define GDN_TICKT(tid, kern, idx) do { } while (0)
-#define GDN_TRIP(kern, idx) do { } while (0)
-#endif
 
 namespace {
 
@@ -192,7 +171,6 @@ constexpr uint32_t C_E_LR = 256;   // low-rank mode (no Nm, Bf): E is started ea
 }  // namespace prep
 
 __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __grid_constant__ TcParams P) {
-    GDN_TRIP(0, 0);
     using namespace prep;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...; the inputs of its next one
@@ -297,17 +275,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
                 // phase 3 is done: Q, K have been read for the last time
                 if (opform && !(lok = mbar_wait(&bar_ld1, ph))) break;
                 if (opform && has_next) {
-#ifdef GDN_PHASE_TIMING
-                    if (blockIdx.x == 0) g_ticks[3][10] = clock64();
-#endif
                     mbar_expect_tx(&bar_qk, 32768);
                     pend_qk = true;
 #pragma unroll 1
                     for (int piece = 0; piece < 4; ++piece) {
                         load_piece(piece, nx);
-#ifdef GDN_PHASE_TIMING
-                        if (blockIdx.x == 0) g_ticks[3][11 + piece] = clock64();
-#endif
                     }
                 }
                 // the three images are staged.  All CTAs store at about the same time, so the 96 KB drain at the rate of
@@ -398,8 +370,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     const bool has_next = item + (int)gridDim.x < n_items;
     const bool first = item == (int)blockIdx.x;
     if (has_next) chunk_entry(p, xn, item + gridDim.x);
-    GDN_TICK(0, 0);
-    GDN_TRIP(0, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
 
     // this trip's gate arrays (written by warp 0 during the previous trip; the barrier before phase 1 publishes them)
     const float* gl = gate_sets[in_phase][0];
@@ -408,12 +378,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     const float* bb = gate_sets[in_phase][3];
     const float* ww = gate_sets[in_phase][4];
     const float* bgam = gate_sets[in_phase][5];
-    GDN_TICK(0, 20);
     if (ok) {
         ok = mbar_wait(&bar_vo, in_phase);
-        GDN_TICK(0, 21);
         ok = ok && mbar_wait(&bar_qk, in_phase);
-        GDN_TICK(0, 22);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 1);
     }
     if (ok && x.len < kC) {   // identity padding of a ragged tail: rows beyond the sequence read as zero
@@ -424,7 +391,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         fence_async_smem();
     }
     cta_sync();
-    GDN_TICK(0, 1);
 
     // ---- phase 1: S1 = [Q; K] K^T  (rows 0..63: Q K^T, rows 64..127: K K^T)
     if (ok && issuer) {
@@ -456,12 +422,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     };
     if (bwd && !opform) form_R(sm + WET);
     GDN_WAIT_MMA(2)
-    GDN_TICK(0, 23);
     if (ok && !first) {   // the previous trip's stores have read what lies under the fp32 A block and under P
         ok = mbar_wait(&bar_free1, in_phase ^ 1);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 6);
     }
-    GDN_TICK(0, 2);
     if (ok && worker) {
         const int i = (q4 & 1) * 32 + lane, j0 = grp * kTG;
 #pragma unroll 1
@@ -489,7 +453,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(0, 3);
     // (P^T dO)^T = dO^T P needs nothing of the inversion: it runs under it and is covered by phase 2's commit
     if (ok && issuer && bwd) {
         tc_fence_after();
@@ -498,28 +461,22 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
         if (!opform) mma_tile<128, 128, 64>(tmem + C_E_LR, op_mn_major(sm + QK, 128, 0), op_mn_major(sm + WET, 64), false);
     }
     // ---- T = (I + A)^-1, blocked (see inv_diag8 ... inv_level).  All fp32.
-    GDN_TICK(0, 24);
     if (ok && !first) {   // ... and what lies under the fp32 T block
         ok = mbar_wait(&bar_free2, in_phase ^ 1);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 8);
     }
-    GDN_TICK(0, 25);
     inv_diag8(Af, Tf);
     cta_sync();
     inv_diag16(Af, Tf, Sf);
     cta_sync();
-    GDN_TICK(0, 16);
     inv_premul<2>(Af, Tf, Sf);   // Sf <- T_rr A_rk for every block below the diagonal
     cta_sync();
     inv_level<1, 1, 2>(Sf, Tf);
     cta_sync();
-    GDN_TICK(0, 17);
     inv_level<2, 2, 2>(Sf, Tf);
     cta_sync();
-    GDN_TICK(0, 18);
     inv_level<3, 4, 2>(Sf, Tf);
     cta_sync();
-    GDN_TICK(0, 4);
     if (ok && !first) {   // every store of the previous trip has read its tile (the T tiles and the second readout are next)
         ok = mbar_wait(&bar_free, in_phase ^ 1);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 5);
@@ -551,7 +508,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     }
     fence_async_smem();
     cta_sync();
-    GDN_TICK(0, 5);
 
     // ---- phase 2: W^T = K^T (T Diag(b Gam))^T ; U~^T = V^T (T Diag(w))^T
     if (ok && issuer) {
@@ -595,7 +551,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(0, 6);
 
     // ---- phase 3: Nm = K^T (Diag(e) W) ; Bf = K^T (Diag(e) U~) ; E = Q^T R - W^T (P^T dO)
     if (ok && issuer) {
@@ -612,12 +567,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     }
     if (has_next && warp == 0) make_gates(in_phase ^ 1, xn.ch);   // the next trip's gate arrays, while the products run
     GDN_WAIT_MMA(4)
-    GDN_TICK(0, 26);
     if (ok) {   // the T tile, part of the Nm staging area, has left through its store
         ok = mbar_wait(&bar_tfree, in_phase);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 7);
     }
-    GDN_TICK(0, 7);
     if (ok && worker) {   // Nm, Bf, E -> bf16 tile images staged over tiles that no MMA reads any more
         const int r = q4 * 32 + lane, c0 = grp * (D / kGroups);
         const float sc = p.d.scale;
@@ -646,10 +599,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     fence_async_smem();
     cta_sync();
     if (threadIdx.x == 32) mbar_arrive(&bar_st);   // the three images are staged: the loader stores them
-    GDN_TICK(0, 8);
     if (!ok) break;
     }
-    GDN_TRIP(0, 20);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -764,14 +715,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
         const size_t ch = (size_t)chunk_of(s) * p.d.H + hd;
         const int stage = s % STAGES;
         const unsigned char* ring = sm + stage * STAGE_BYTES;
-        if (s < 4) GDN_TICK(1, s * 5 + 0);
         const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
         // state -> bf16: operand tile of the MMA; the same bytes are the per-chunk state the gradient stage reads
 #pragma unroll
         for (int k = 0; k < NSH / 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
         fence_async_smem();
         __syncthreads();
-        if (s < 4) GDN_TICK(1, s * 5 + 1);
         if (threadIdx.x == 0) {
             ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
             if (ok) {
@@ -793,13 +742,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
             // to issue; a thread of another warp does it so that the MMA issue is not delayed.
             if (s >= 1 && s - 1 + STAGES < nsteps) fill(s - 1 + STAGES);
         }
-        if (s < 4) GDN_TICK(1, s * 5 + 2);
         ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);   // the additive term of this step is in shared memory
         if (ok) ok = mbar_wait(&bar_mma, mma_phase);
         mma_phase ^= 1;
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 11); break; }
         tc_fence_after();
-        if (s < 4) GDN_TICK(1, s * 5 + 3);
 #pragma unroll
         for (int k = 0; k < NSH / 8; ++k) {
             float dl[8], ad[8];
@@ -809,7 +756,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 #pragma unroll
             for (int j = 0; j < 8; ++j) st[8 * k + j] = fmaf(Ge, st[8 * k + j], ad[j] - dl[j]);
         }
-        if (s < 4) GDN_TICK(1, s * 5 + 4);
         tc_fence_before();
     }
     float* fin = reverse ? p.dh0 : p.hT;
@@ -1067,7 +1013,6 @@ __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eigh
 }  // namespace intra
 
 __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const __grid_constant__ TcParams P) {
-    GDN_TRIP(1, 0);
     using namespace intra;
     const Problem& p = P.p;
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
@@ -1223,17 +1168,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         return;
     }
 
-#ifdef GDN_PHASE_TIMING
-    int sync_no = 0;
-    auto cta_sync = [&] {
-        if (blockIdx.x == 0 && lane == 0 && g_trip_now == g_tick_trip && sync_no < 16) g_sync[sync_no][warp] = clock64();
-        asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory");
-        if (blockIdx.x == 0 && threadIdx.x == 0 && g_trip_now == g_tick_trip && sync_no < 16) g_sync[sync_no][17] = clock64();
-        ++sync_no;
-    };
-#else
     auto cta_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(kIntraThreads) : "memory"); };   // all warps but the loader
-#endif
     uint32_t mma_phase = 0, in_phase = 0;
     // chunk table entry and gates of a trip are fetched one trip ahead into registers (their latency would be exposed)
     ChunkInfo xn;
@@ -1284,21 +1219,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const bool has_next = item + (int)gridDim.x < n_items;
     const bool first = item == (int)blockIdx.x;
     if (has_next) chunk_entry(p, xn, item + gridDim.x);
-#ifdef GDN_PHASE_TIMING
-    if (blockIdx.x == 0 && threadIdx.x == 0) g_trip_now = (item - (int)blockIdx.x) / (int)gridDim.x;
-#endif
-    GDN_TICK(2, 0);
-    GDN_TRIP(1, 1 + (item - (int)blockIdx.x) / (int)gridDim.x);
-#ifdef GDN_PHASE_TIMING
-    sync_no = 0;
-#endif
 
-    GDN_TICK(2, 19);
     if (ok) {
         ok = mbar_wait(&bar_g1, in_phase);
-        GDN_TICK(2, 20);
         ok = ok && mbar_wait(&bar_k, in_phase);
-        GDN_TICK(2, 21);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 20);
     }
     if (ok && x.len < kC) {
@@ -1307,7 +1231,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         fence_async_smem();
     }
     cta_sync();
-    GDN_TICK(2, 1);
 
     // ---- phase 1: (W h)^T and (K dh')^T.  P = tril(Q K^T . D) is not formed here: tc_prep made it and it arrived
     // with the first group of tiles.
@@ -1316,8 +1239,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_tile<128, 64, 128>(tmem + slot(1), op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
         mma_tile<128, 64, 128>(tmem + slot(2), op_mn_major(sm + DH, 128), op_k_major(sm + QK, 128, 64), false);
     }
-    GDN_TICK(2, 2);
-    GDN_TICK(2, 3);
     if (ok) {
         ok = mbar_wait(&bar_do, in_phase);
         if (!ok && threadIdx.x == 0) report_timeout(p.ws, 27);
@@ -1327,7 +1248,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         fence_async_smem();
     }
     cta_sync();
-    GDN_TICK(2, 4);
 
     // ---- phase 2
     if (ok && issuer) {
@@ -1340,7 +1260,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     if (threadIdx.x == 32) mbar_arrive(&bar_ld0);   // every tile of this trip has arrived
     if (has_next && threadIdx.x < kC) fetch_gates(xn);
     if (ok && have_prev && warp < 2) finish_gates();   // warps 0 and 1: the previous chunk's gate gradients
-    GDN_TICK(2, 5);
     GDN_WAIT_MMA(22)
     if (ok && !first) {   // U^T and dU^T held the previous trip's staged dk and dq: their stores must have read them
         ok = mbar_wait(&bar_free, in_phase ^ 1);
@@ -1379,7 +1298,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(2, 6);
 
     // From here on the accumulators that become gradients are produced token-major (64 token rows x 128 features,
     // M = 64): a thread owns a token row, so row dots are thread-local and rows leave with 16-byte stores.  A 64-row
@@ -1406,7 +1324,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         // has looked, and a parity wait cannot tell a phase from the one two later)
         mma_commit(&bar_mma2);
     }
-    GDN_TICK(2, 7);
     if (has_next && threadIdx.x < kC) make_gates(in_phase ^ 1);   // the next trip's gate arrays, while the product runs
     // <dh', h> over the whole state, while the products run (both tiles share one format, so offsets pair up)
     float hh = 0.f;
@@ -1458,7 +1375,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(2, 8);
 
     // ---- phase 4
     if (ok && issuer) {
@@ -1470,7 +1386,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
         mma_tile<64, 128, 128>(tmem + 0, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);                // U dh'^T
     }
-    GDN_TICK(2, 9);
     GDN_WAIT_MMA(24)
     const bool full = x.len == kC;
     // (addresses of the ragged-tail flushes are formed where they are used: nothing of them lives across the phases)
@@ -1510,7 +1425,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(2, 10);
 
     // ---- phase 5
     if (ok && issuer) {
@@ -1530,7 +1444,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         flush_rows(sm + STG_A, grad_rows(p.dq), (size_t)H * D, x.len, kIntraThreads);
         flush_rows(sm + STG_B, grad_rows(p.dv), (size_t)H * D, x.len, kIntraThreads);
     }
-    GDN_TICK(2, 11);
     GDN_WAIT_MMA(25)
     if (ok && worker) {
         float v2[2][8];
@@ -1558,7 +1471,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     tc_fence_before();
     fence_async_smem();
     cta_sync();
-    GDN_TICK(2, 12);
 
     // ---- phase 6
     if (ok && issuer) {
@@ -1568,9 +1480,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         mma_commit(&bar_mma);
         mma_commit(&bar_ld2);   // dW^T (over dO) and T have been read for the last time
     }
-    GDN_TICK(2, 13);
     GDN_WAIT_MMA(26)
-    GDN_TICK(2, 16);
     if (worker) {   // this thread's K values leave shared memory now, so that the next trip's K can be loaded over them
         uint4 kraw[4];
 #pragma unroll
@@ -1578,7 +1488,6 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             kraw[part] = *reinterpret_cast<const uint4*>(sm + QK + tile_chunk_off(128, 64 + tr, (cb0 >> 3) + part));
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar_kfree);
-        GDN_TICK(2, 17);
         // Group A assembles dk = Diag(b)(G K + Gam dXk) + dk^col and both row dots with k; the lanes of group B hold
         // nothing of this phase (Diag(b) G K is a row scaling of G K, so one product serves dk and db).
         float acc_col = 0.f, acc_db = 0.f;   // <k, dk^col> ; db = <k, G K + Gam dXk>
@@ -1609,14 +1518,12 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         }
         if (ga) { red[2][grp][tr] = acc_db; red[3][grp][tr] = acc_col; }
     }
-    GDN_TICK(2, 18);
     // block totals of sum_j r_j and <dh', h>
     rs = warp_sum(rs);
     hh = warp_sum(hh);
     if (lane == 0) { scal[0][warp] = rs; scal[1][warp] = hh; }
     fence_async_smem();
     cta_sync();
-    GDN_TICK(2, 14);
     if (threadIdx.x == 32) mbar_arrive(&bar_st2);   // dk is staged: the loader stores it
     if (ok && !full) flush_rows(sm + STG_K, grad_rows(p.dk), (size_t)H * D, x.len, kIntraThreads);
     // The token-wise sums are complete; turning them into dbeta and dg is left to warps 0 and 1 during the next trip's
@@ -1626,11 +1533,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     have_prev = true;
     tc_fence_before();
     cta_sync();   // every reader of this trip's tiles and scratch is done
-    GDN_TICK(2, 15);
     if (!ok) break;
     }
     if (ok && have_prev && warp < 2) finish_gates();
-    GDN_TRIP(1, 20);
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
@@ -1756,14 +1661,19 @@ bool tc_supported(const gdn_desc& d) {
 }
 
 static int sm_count();
+// When one CTA per (chain, direction) of the backward fills more than half of the SMs the carries are bound by HBM
+// bandwidth, and the low-rank form moves less.  With fewer chains a step's latency counts, and the operator form needs one
+// product per step.  The rule looks at the chains only, so the forward, the backward and a backward on a workspace fresh
+// from the forward agree on the form (and on the workspace layout that follows from it).
+bool tc_carries_lowrank(const gdn_desc& d) {
+    if (g_force_carries) return g_force_carries == 2;
+    return 4 * (long long)d.N * d.H > sm_count();
+}
 static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_dirs) {
     P.p = p;
     P.with_bwd = with_bwd ? 1 : 0;
     P.scan_dirs = scan_dirs;
-    // One CTA per (chain, direction) fills the machine: the carries are bound by HBM bandwidth, and the low-rank form
-    // moves less.  With fewer chains a step's latency counts, and the operator form needs one product per step.
-    const int ctas = p.d.N * p.d.H * (scan_dirs == 2 ? 2 : 1);
-    P.lowrank = g_force_carries ? (g_force_carries == 2) : (2 * ctas > sm_count());
+    P.lowrank = tc_carries_lowrank(p.d) ? 1 : 0;
     const uint64_t rows = (uint64_t)p.Ttot, cols = (uint64_t)p.d.H * D, pitch = cols * 2;
     if (!tc::make_tmap_bf16_2d(&P.tm_q, p.q, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
@@ -1870,17 +1780,3 @@ cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st
 
 }  // namespace gdn
 
-#ifdef GDN_PHASE_TIMING
-extern "C" int gdn_debug_tick_trip(int trip) {
-    return (int)cudaMemcpyToSymbol(gdn::g_tick_trip, &trip, sizeof(int));
-}
-extern "C" int gdn_debug_trips(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, gdn::g_trip_ns, sizeof(long long) * 2 * 24);
-}
-extern "C" int gdn_debug_syncs(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, gdn::g_sync, sizeof(long long) * 16 * 18);
-}
-extern "C" int gdn_debug_ticks(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks, sizeof(long long) * 4 * 32);
-}
-#endif

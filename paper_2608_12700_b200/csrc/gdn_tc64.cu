@@ -17,13 +17,6 @@
 
 namespace gdn {
 
-// Optional phase timing (compile with -DGDN_PHASE_TIMING): thread 0 of CTA 0 stamps clock64() at phase borders of one step.
-#ifdef GDN_PHASE_TIMING
-__device__ long long g_ticks64[32];
-#define T64(idx) do { if (blockIdx.x == 0 && threadIdx.x == 0 && s == 5) g_ticks64[idx] = clock64(); } while (0)
-#else
-#define T64(idx) do { } while (0)
-#endif
 namespace {
 
 constexpr int D6 = 64;
@@ -375,11 +368,8 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
         if (s + 1 < nsteps) { len_n = cg.chunk_len(c - 1); tok0_n = cg.chunk_tok0(c - 1); }
         unsigned char* tiles = sm + stage * STAGE_BYTES;
         const float *gl = gl2[s & 1], *Gam = Gam2[s & 1], *ee = ee2[s & 1];
-        T64(0);
-        T64(1);
         ok = mbar_wait(&bar_full[stage], (s / STAGES) & 1);
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 50); break; }
-        T64(2);
         if (len < kC) {
             zero_tail_rows64(tiles + QT, len);
             zero_tail_rows64(tiles + KT, len);
@@ -400,7 +390,6 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
         fence_async_smem();
         cta_sync();
         const float Ge = Gam[kC - 1];
-        T64(3);
         // ---- phase 1: S = Q K^T ; dO V^T ; K dh' (group A) | dO h^T ; V dh'^T (group B)
         if (threadIdx.x == 0) {
             tc_fence_after();
@@ -411,14 +400,12 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
             mma_tile<64, 64, 64>(tmem + C2 + LB, op_k_major(tiles + VT, 64), op_k_major(sm + DH, 64), false);
             mma_commit(&bar_mma);
         }
-        T64(4);
         if (threadIdx.x < kC && s + 1 < nsteps) {
             make_gates((s + 1) & 1, gnext, gend_next);
             if (s + 2 < nsteps) { gnext = gate_row(s + 2)[threadIdx.x]; gend_next = gate_row(s + 2)[kC - 1]; }
         }
         GDN_WAIT_MMA(51)
         if (!ok) break;
-        T64(5);
         for (int t = threadIdx.x; t < kC * 8; t += kThreads64) {   // Diag(Gam) dO over the dh' tile, which no MMA reads any more
             const int i = t >> 3, cch = t & 7;
             float v[8];
@@ -427,7 +414,6 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
             for (int k = 0; k < 8; ++k) v[k] *= Gam[i];
             chunk_store(sm + DH, 64, i, cch, v);
         }
-        T64(6);
         float rs = 0.f;   // sum_j r_j, r_j = e_j <(K dh')_j, V_j>
 #pragma unroll 1
         for (int part = 0; part < 4; ++part) {
@@ -456,7 +442,6 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
         tc_fence_before();
         fence_async_smem();
         cta_sync();
-        T64(7);
         // ---- phase 2: P^T dO ; (Diag(Gam) Q)^T dO (group A) | (dP.D) K ; (dP.D)^T Q (group B)
         if (threadIdx.x == 0) {
             tc_fence_after();
@@ -466,10 +451,8 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
             mma_tile<64, 64, 64>(tmem + C3 + LB, op_mn_major(sm + DPD, 64), op_mn_major(tiles + QT, 64), false);
             mma_commit(&bar_mma);
         }
-        T64(8);
         GDN_WAIT_MMA(52)
         if (!ok) break;
-        T64(9);
         float dot = 0.f;   // group B: <q_r, dq_r> - <k_r, dk_r> over this thread's columns
         // Gradient rows are staged token-major in place over this step's input tiles (dv over V, which was last read in
         // phase 1; dk over K and dq over Q, where a thread overwrites exactly the piece it has just read) and leave by TMA
@@ -507,7 +490,6 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
                 chunk_store(tiles + QT, 64, r, jb >> 3, a);
             }
         }
-        T64(10);
         if (!ga) dgp[half][r] = dot;
         // group A: dh = Gam_e dh' + scale (Diag(Gam) Q)^T dO
 #pragma unroll
@@ -537,14 +519,12 @@ __global__ void __launch_bounds__(kThreads64 + 32, 2) tc64_bwd_kernel(const __gr
             }
             cta_sync();   // the ring slot is handed to the loader only after every row has been read
         }
-        T64(11);
         if (threadIdx.x == 32) mbar_arrive(&bar_st);
         if (warp == 0) {
             float rsum = 0.f, hsum = 0.f;
             for (int w = 0; w < kThreads64 / 32; ++w) { rsum += scal[0][w]; hsum += scal[1][w]; }
             write_dg_suffix(dgp[0], dgp[1], rsum + Ge * hsum, p.dg + (size_t)tok0 * H + hd, (size_t)H, len, lane);
         }
-        T64(12);
     }
     if (p.dh0 && ok && ga) {
 #pragma unroll
@@ -645,8 +625,3 @@ cudaError_t tc64_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t 
 
 }  // namespace gdn
 
-#ifdef GDN_PHASE_TIMING
-extern "C" int gdn_debug_ticks64(long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, gdn::g_ticks64, sizeof(long long) * 32);
-}
-#endif

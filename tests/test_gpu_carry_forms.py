@@ -96,3 +96,17 @@ def test_many_short_ragged_sequences_in_low_rank_form():
     got, ref = runner.fetch(buf), oracle_grads(wl)
     assert rel(got["o"], ref["o"]) < TOL["bf16"]
     assert rel(got["hT"], ref["hT"]) < TOL["bf16"]
+
+
+def test_operator_form_with_one_cta_per_chain():
+    """With 40 chains the shape rule takes the low-rank form, and below 38 chains the operator form splits a chain over
+    two CTAs; forcing the operator form here runs its one-CTA-per-(chain, direction) variant, which no shape selects by
+    itself on a machine of this size."""
+    wl = synth.make_workload("carry_operator_one_cta", dtype="bf16", B=1, T=192, H=40, d_k=128, d_v=128, states=True,
+                             seed=50)
+    try:
+        binding.gdn_debug_force_family(OPERATOR)
+        got = runner.backward(wl)
+    finally:
+        binding.gdn_debug_force_family(0)
+    check_against_oracle(wl, got)

@@ -1,6 +1,6 @@
 """Persistent-kernel edge cases of the tcgen05 families: numbers of chunk-heads around the number of SMs (a CTA makes
-zero, one or two trips; the last trip of some CTAs has no successor to load for), and the two scan variants (one or
-two CTAs per chain and direction) on both sides of their switch-over."""
+zero, one or two trips; the last trip of some CTAs has no successor to load for), and the number of chains around the
+point where the carries switch from the operator form (two CTAs per chain and direction) to the low-rank form."""
 import numpy as np
 import pytest
 import torch
@@ -33,7 +33,8 @@ def test_single_chunk_head_and_ragged_single_token():
 
 @pytest.mark.parametrize("chains", [36, 37, 38, 74, 75])
 def test_scan_variants_around_their_switch_over(chains):
-    # 2 directions x chains CTAs; the column-split variant is used while 4 x chains CTAs fit the SMs
+    # the operator form with a chain's state columns split over two CTAs is used while 4 x chains CTAs fit the SMs;
+    # beyond that the carries take the low-rank form with one CTA per (chain, direction)
     wl = synth.make_workload(f"edge_scan_{chains}", dtype="bf16", B=1, T=192, H=chains, d_k=128, d_v=128, states=True,
                              seed=700 + chains)
     check_against_oracle(wl, runner.backward(wl))

@@ -171,7 +171,7 @@ def test_zero_upstream_gradient_gives_zero():
         assert not np.any(got[n]), n
 
 
-def test_inputs_are_not_modified_and_padding_is_not_written():
+def test_inputs_are_not_modified():
     wl = small("readonly", lengths=[70], H=2, seed=18, states=True)
     buf = runner.to_device(wl)
     before = {k: v.clone() for k, v in buf.inputs.items() if v is not None}
@@ -181,6 +181,26 @@ def test_inputs_are_not_modified_and_padding_is_not_written():
         assert torch.equal(v, buf.inputs[k]), k
 
 
+@pytest.mark.parametrize("dtype,d,delta", [("f32", 64, 1), ("bf16", 128, 1), ("bf16", 64, 0)])
+def test_rows_outside_every_sequence_are_not_written(dtype, d, delta):
+    """cu_seqlens may end before the buffers do (and T in the descriptor with it): token rows past the last
+    sequence belong to the caller and must keep what they held; so must the rows of a ragged tail's padding."""
+    lengths = [70, 1, 130]
+    wl = small("padding", dtype=dtype, lengths=lengths, H=2, d_k=d, d_v=d, delta_rule=delta, seed=26, states=True)
+    buf = runner.to_device(wl)
+    extra = 100                                     # rows appended behind the last sequence
+    big = {}
+    for n in ("dq", "dk", "dv", "dg", "dbeta"):
+        t = buf.outputs[n]
+        if t is None:
+            continue
+        big[n] = torch.full((t.shape[0] + extra,) + tuple(t.shape[1:]), 7.0, dtype=t.dtype, device=t.device)
+        buf.outputs[n] = big[n][:t.shape[0]]        # same base address, the call sees T rows
+    runner.run_bwd(buf)
+    got = runner.fetch(buf)
+    check_against_oracle(wl, got)
+    for n, t in big.items():
+        assert torch.all(t[wl.T_total:] == 7.0), n
 def test_nan_in_v_propagates_within_its_chain_only():
     wl = small("nan", B=2, T=128, H=2, seed=19)
     wl.v[70, 1, 3] = np.nan        # batch row 0, token 70, head 1
@@ -204,19 +224,16 @@ def test_malformed_cu_seqlens_is_reported_not_faulted():
     assert binding.gdn_last_device_status(buf.workspace) == 0
 
 
-# ---- the benchmark configurations at full size: sampled (sequence, head) chains against the oracle ----
-@pytest.mark.parametrize("idx,heads", [(1, [0, 9]), (2, [5]), (3, [3]), (4, [0, 31])])
-def test_full_size_configs_sampled_chains(idx, heads):
+# ---- the benchmark configurations at full size, every (sequence, head) chain against the oracle ----
+# (the oracle does all of cfg1 in about two seconds on the GPU machine's host cores and the largest, cfg4, in well under
+# a minute, so nothing is sampled; the comparison is per tensor and per 64-token block of every head)
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_full_size_configs_all_chains(idx):
     wl = synth.config(idx)
     got = runner.backward(wl)
-    sub = wl.take_heads(heads)
-    ref = oracle_grads(sub)
-    got_sub = {n: (v[:, heads] if v.ndim >= 2 else v) for n, v in got.items()}
-    errs = check_against_oracle(sub, got_sub, ref=ref)
+    errs = check_against_oracle(wl, got)
     print(wl.name, errs)
-    for n, v in got.items():
-        assert np.isfinite(v).all(), n
     # the acceptance bound the paper sets for its own assembled bf16 backward against its fp64 oracle (Section 4.5)
     with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "paper_figures.json")) as f:
         bound = json.load(f)["assembled_backward_acceptance_bound"]["value"]
-    assert max(errs.values()) <= bound, errs
+    assert max(v for n, v in errs.items() if n != "worst_block") <= bound, errs

@@ -235,3 +235,62 @@ def test_threads_do_not_change_the_result():
     b = oracle.bwd(x["q"], x["k"], x["v"], x["g"], x["b"], x["w"], x["dO"], cu_seqlens=x["cu"], h0=x["h0"], dhT=x["dhT"], n_threads=7)
     for name in a:
         assert np.array_equal(a[name], b[name]), name
+
+
+# ---- the workload wrapper every GPU parity test goes through: its gate mapping and dbeta = db + dw ----
+def _tiny_workload(delta_rule, seed):
+    from paper_2608_12700_b200 import synth
+    return synth.make_workload("pin_wrapper", dtype="f32", lengths=[23, 70], H=2, d_k=6, d_v=5, seed=seed,
+                               delta_rule=delta_rule, states=True, scale=0.7)
+
+
+def _workload_loss(wl, beta):
+    """L as a function of beta itself: one array feeds both the erase and the write gate (Table 2, GDN row)."""
+    o, hT = oracle.fwd(wl.q, wl.k, wl.v, wl.g, beta, beta, cu_seqlens=wl.cu_seqlens, scale=wl.scale, h0=wl.h0)
+    return np.sum(o * wl.dO.astype(np.float64)) + np.sum(hT * wl.dhT.astype(np.float64))
+
+
+def test_workload_wrapper_dbeta_is_the_derivative_with_respect_to_beta():
+    wl = _tiny_workload(1, seed=70)
+    out = oracle.bwd_workload(wl)
+    beta = wl.beta.astype(np.float64)
+    rng = np.random.default_rng(71)
+    idx = rng.choice(beta.size, size=40, replace=False)
+    eps = 1e-6
+    num = np.zeros(len(idx))
+    for n, i in enumerate(idx):
+        bp = beta.copy().reshape(-1); bm = beta.copy().reshape(-1)
+        bp[i] += eps; bm[i] -= eps
+        num[n] = (_workload_loss(wl, bp.reshape(beta.shape)) - _workload_loss(wl, bm.reshape(beta.shape))) / (2 * eps)
+    assert rel(out["dbeta"].reshape(-1)[idx], num) < 1e-7
+    # and it is not the gradient of either gate alone
+    assert rel(out["db"].reshape(-1)[idx], num) > 1e-2 and rel(out["dw"].reshape(-1)[idx], num) > 1e-2
+
+
+def test_workload_wrapper_delta_rule_off_is_erase_zero_write_one():
+    wl = _tiny_workload(0, seed=72)
+    out = oracle.bwd_workload(wl)
+    assert "dbeta" not in out
+    zero, one = np.zeros_like(wl.g, dtype=np.float64), np.ones_like(wl.g, dtype=np.float64)
+    direct = oracle.bwd(wl.q, wl.k, wl.v, wl.g, zero, one, wl.dO, cu_seqlens=wl.cu_seqlens, scale=wl.scale,
+                        h0=wl.h0, dhT=wl.dhT)
+    for n in ("o", "hT", "dq", "dk", "dv", "dg", "dh0"):
+        assert np.array_equal(out[n], direct[n]), n
+    # the same thing as one masked matrix product per (sequence, head) (Table 2, the scalar-decay row):
+    # o = scale [ (Q K^T . D) V + Diag(Gam) Q h0 ],  D_ts = exp(cs_t - cs_s) for s <= t, Gam_t = exp(cs_t)
+    cu = wl.cu_seqlens
+    for n in range(wl.N):
+        s = slice(cu[n], cu[n + 1])
+        for hd in range(wl.H):
+            Q, K, V = (a[s, hd].astype(np.float64) for a in (wl.q, wl.k, wl.v))
+            dO = wl.dO[s, hd].astype(np.float64)
+            cs = np.cumsum(wl.g[s, hd].astype(np.float64))
+            Dm = np.tril(np.exp(cs[:, None] - cs[None, :]))
+            h0 = wl.h0[n, hd].astype(np.float64)
+            S = (Q @ K.T) * Dm
+            o = wl.scale * (S @ V + np.exp(cs)[:, None] * (Q @ h0))
+            assert np.allclose(out["o"][s, hd], o, rtol=1e-11, atol=1e-12)
+            # textbook gradient of that product with respect to V, plus the path through the final state
+            e = np.exp(cs[-1] - cs)
+            dv = wl.scale * (S.T @ dO) + e[:, None] * (K @ wl.dhT[n, hd].astype(np.float64))
+            assert np.allclose(out["dv"][s, hd], dv, rtol=1e-10, atol=1e-11)
