@@ -104,6 +104,36 @@ gdn_status gdn_bwd(const gdn_desc* desc,
                    void* workspace, size_t workspace_bytes, int32_t workspace_is_fresh_from_fwd,
                    void* cuda_stream);
 
+/* ---- channel-wise gates: the general recurrence of Eq. 1 as printed ---------------------------------
+ * Section 4.1, Eq. 1 and Table 2; Appendix A, "The GDN backward's two hard stages" ("the channel-wise path
+ * folds the per-channel decay Diag(e^{g_t}) inside those contractions").  Three gate VECTORS per (token, head):
+ *
+ *     h_t = (I - k_t (b_t . k_t)^T) Diag(e^{g_t}) h_{t-1} + k_t (w_t . v_t)^T ,     o_t = scale * h_t^T q_t
+ *
+ *     g, b, dg, db   dev [B, T, H, d_k] float32  (log-decay and erase gate per key channel)
+ *     w, dw          dev [B, T, H, d_v] float32  (write gate per value channel)
+ * Every other argument, the sequence description, ownership, execution and error behaviour are those of
+ * gdn_fwd_recompute / gdn_bwd; desc->delta_rule is not read (the gates say which family member runs: KDA is
+ * b = w = beta broadcast over the channels, GLA is b = 0, w = 1, the full GDN has independent vectors).  All three
+ * gate gradients are required outputs.  The workspace has its own size (gdn_workspace_bytes_channelwise) and
+ * layout; its status word is read with gdn_last_device_status.  These entry points run on fp32 FFMA kernels
+ * for either I/O dtype (bf16 I/O: inputs and dq, dk, dv are bf16, all arithmetic and the gate tensors are fp32). */
+gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
+gdn_status gdn_fwd_recompute_channelwise(const gdn_desc* desc,
+                                         const void* q, const void* k, const void* v,
+                                         const float* g, const float* b, const float* w, const float* h0,
+                                         const int32_t* cu_seqlens_dev,
+                                         void* o, float* hT,
+                                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+gdn_status gdn_bwd_channelwise(const gdn_desc* desc,
+                               const void* q, const void* k, const void* v,
+                               const float* g, const float* b, const float* w, const float* h0,
+                               const void* dO, const float* dhT,
+                               const int32_t* cu_seqlens_dev,
+                               void* dq, void* dk, void* dv, float* dg, float* db, float* dw, float* dh0,
+                               void* workspace, size_t workspace_bytes, int32_t workspace_is_fresh_from_fwd,
+                               void* cuda_stream);
+
 /* Synchronises the stream, reads the device-side status word of the last call that used `workspace`
  * and returns it (GDN_OK, GDN_ERR_BAD_SEQLENS or GDN_ERR_DEVICE_TIMEOUT; GDN_ERR_CUDA if the stream
  * itself reports an error).  Error reporting of this library (the paper has no counterpart).  After

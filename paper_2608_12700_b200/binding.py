@@ -23,7 +23,8 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
            "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc",
-           "gdn_noalloc_last_device_status"]
+           "gdn_noalloc_last_device_status", "gdn_workspace_bytes_channelwise", "gdn_fwd_recompute_channelwise",
+           "gdn_bwd_channelwise"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -72,6 +73,12 @@ def lib():
         L.gdn_stage_timing_read.argtypes = [I, P, P, P, P]
         L.gdn_bwd_noalloc.restype = I
         L.gdn_bwd_noalloc.argtypes = [D] + [P] * 15 + [P]
+        L.gdn_workspace_bytes_channelwise.restype = I
+        L.gdn_workspace_bytes_channelwise.argtypes = [D, ctypes.POINTER(Z), ctypes.POINTER(Z)]
+        L.gdn_fwd_recompute_channelwise.restype = I
+        L.gdn_fwd_recompute_channelwise.argtypes = [D] + [P] * 10 + [P, Z, P]
+        L.gdn_bwd_channelwise.restype = I
+        L.gdn_bwd_channelwise.argtypes = [D] + [P] * 17 + [P, Z, I, P]
         L.gdn_noalloc_last_device_status.restype = I
         L.gdn_noalloc_last_device_status.argtypes = [P]
         L.gdn_debug_read.restype = I
@@ -208,3 +215,33 @@ def gdn_bwd_noalloc(desc, q, k, v, g, beta, h0, dO, dhT, cu_seqlens, dq, dk, dv,
 def gdn_noalloc_last_device_status(stream=None) -> int:
     """Device-side status of the last gdn_bwd_noalloc on the current device (synchronises the stream)."""
     return lib().gdn_noalloc_last_device_status(_stream(stream))
+
+
+def gdn_workspace_bytes_channelwise(desc: gdn_desc):
+    """Returns (fwd_bytes, bwd_bytes) of the channel-wise entry points."""
+    f, b = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    s = lib().gdn_workspace_bytes_channelwise(ctypes.byref(desc), ctypes.byref(f), ctypes.byref(b))
+    if s != GDN_OK:
+        raise GdnError(s, "gdn_workspace_bytes_channelwise")
+    return f.value, b.value
+
+
+def gdn_fwd_recompute_channelwise(desc, q, k, v, g, b, w, h0, cu_seqlens, o, hT, workspace, workspace_bytes=None,
+                                  stream=None, check=True) -> int:
+    wb = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
+    s = lib().gdn_fwd_recompute_channelwise(ctypes.byref(desc), _p(q), _p(k), _p(v), _p(g), _p(b), _p(w), _p(h0),
+                                            _p(cu_seqlens), _p(o), _p(hT), _p(workspace), wb, _stream(stream))
+    if check and s != GDN_OK:
+        raise GdnError(s, "gdn_fwd_recompute_channelwise")
+    return s
+
+
+def gdn_bwd_channelwise(desc, q, k, v, g, b, w, h0, dO, dhT, cu_seqlens, dq, dk, dv, dg, db, dw, dh0, workspace,
+                        workspace_bytes=None, workspace_is_fresh_from_fwd=0, stream=None, check=True) -> int:
+    wb = workspace.numel() * workspace.element_size() if workspace_bytes is None else workspace_bytes
+    s = lib().gdn_bwd_channelwise(ctypes.byref(desc), _p(q), _p(k), _p(v), _p(g), _p(b), _p(w), _p(h0), _p(dO), _p(dhT),
+                                  _p(cu_seqlens), _p(dq), _p(dk), _p(dv), _p(dg), _p(db), _p(dw), _p(dh0), _p(workspace),
+                                  wb, int(workspace_is_fresh_from_fwd), _stream(stream))
+    if check and s != GDN_OK:
+        raise GdnError(s, "gdn_bwd_channelwise")
+    return s

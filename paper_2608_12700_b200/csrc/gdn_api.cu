@@ -26,8 +26,8 @@ cudaEvent_t take_event() {
     cudaEventCreate(&e);
     return e;
 }
-void call_begin() { g_timing = g_period > 0 && (g_calls++ % (uint64_t)g_period) == 0; }
 }  // namespace
+void call_begin() { g_timing = g_period > 0 && (g_calls++ % (uint64_t)g_period) == 0; }
 
 void stage_begin(Stage, cudaStream_t st) {
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -67,6 +67,19 @@ Path pick_path(const gdn_desc& d) {
     return Path::None;
 }
 
+WsLayout layout_for(const gdn_desc& d) {
+    // tcgen05 path: every factor, state and additive term of the carries is a bf16 tile image.
+    // The d = 128 family keeps the chunk operator Nm and the additive term Bf only when its carries use them.
+    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0, !tc_carries_lowrank(d));
+    if (pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
+    // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
+    return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
+}
+
+}  // namespace
+}  // namespace gdn
+
+namespace gdn {
 gdn_status check_desc(const gdn_desc* d) {
     if (!d) return GDN_ERR_NULL_ARG;
     if (d->B <= 0 || d->T < 0 || d->H <= 0 || d->N <= 0 || d->d_k <= 0 || d->d_v <= 0) return GDN_ERR_BAD_SHAPE;
@@ -78,15 +91,6 @@ gdn_status check_desc(const gdn_desc* d) {
     return GDN_OK;
 }
 
-WsLayout layout_for(const gdn_desc& d) {
-    // tcgen05 path: every factor, state and additive term of the carries is a bf16 tile image.
-    // The d = 128 family keeps the chunk operator Nm and the additive term Bf only when its carries use them.
-    if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0, !tc_carries_lowrank(d));
-    if (pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
-    // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
-    return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
-}
-
 // Sequences are described either by cu_seqlens (then B must be 1) or by B rows of T tokens (then N == B).
 gdn_status check_seq(const gdn_desc& d, const int32_t* cu) {
     if (cu) { if (d.B != 1) return GDN_ERR_BAD_SHAPE; }
@@ -94,10 +98,6 @@ gdn_status check_seq(const gdn_desc& d, const int32_t* cu) {
     return GDN_OK;
 }
 
-}  // namespace
-}  // namespace gdn
-
-namespace gdn {
 gdn_status check_bwd_args(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
                           const float* h0, const void* dO, const float* dhT, const int32_t* cu, void* dq, void* dk, void* dv,
                           float* dg, float* dbeta, float* dh0, const void* workspace, size_t workspace_bytes) {
@@ -174,6 +174,63 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     const cudaError_t e = path == Path::TcBf16 ? tc_launch_bwd(p, fresh, st)
                           : path == Path::Tc64Bf16 ? tc64_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+// ---- channel-wise entry points: Eq. 1 with gate vectors (FFMA family) ----
+gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes) {
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    const WsLayout L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
+    if (fwd_bytes) *fwd_bytes = L.fwd_end;
+    if (bwd_bytes) *bwd_bytes = L.total;
+    return GDN_OK;
+}
+
+gdn_status gdn_fwd_recompute_channelwise(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g,
+                                         const float* b, const float* w, const float* h0, const int32_t* cu, void* o,
+                                         float* hT, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    call_begin();
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
+    const bool empty = (long long)desc->B * desc->T == 0;
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    if (!empty && (!q || !k || !v || !g || !b || !w)) return GDN_ERR_NULL_ARG;
+    const void* ptrs[] = {q, k, v, g, b, w, h0, cu, o, hT, workspace};
+    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
+    Problem p{};
+    p.d = *desc;
+    p.Ttot = desc->B * desc->T;
+    p.L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
+    if (workspace_bytes < p.L.fwd_end) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    p.q = q; p.k = k; p.v = v; p.gv = g; p.bv = b; p.wv = w; p.h0 = h0; p.cu = cu; p.o = o; p.hT = hT;
+    p.ws = static_cast<char*>(workspace);
+    return vec_launch_fwd(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+}
+
+gdn_status gdn_bwd_channelwise(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g,
+                               const float* b, const float* w, const float* h0, const void* dO, const float* dhT,
+                               const int32_t* cu, void* dq, void* dk, void* dv, float* dg, float* db, float* dw, float* dh0,
+                               void* workspace, size_t workspace_bytes, int32_t workspace_is_fresh_from_fwd, void* cuda_stream) {
+    call_begin();
+    gdn_status s = check_desc(desc);
+    if (s != GDN_OK) return s;
+    if ((s = check_seq(*desc, cu)) != GDN_OK) return s;
+    const bool empty = (long long)desc->B * desc->T == 0;
+    if (!workspace) return GDN_ERR_NULL_ARG;
+    if (!empty && (!q || !k || !v || !g || !b || !w || !dO || !dq || !dk || !dv || !dg || !db || !dw)) return GDN_ERR_NULL_ARG;
+    const void* ptrs[] = {q, k, v, g, b, w, h0, dO, dhT, cu, dq, dk, dv, dg, db, dw, dh0, workspace};
+    for (const void* p : ptrs) if (!aligned16(p)) return GDN_ERR_MISALIGNED;
+    Problem p{};
+    p.d = *desc;
+    p.Ttot = desc->B * desc->T;
+    p.L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
+    if (workspace_bytes < p.L.total) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    p.q = q; p.k = k; p.v = v; p.gv = g; p.bv = b; p.wv = w; p.h0 = h0; p.dO = dO; p.dhT = dhT; p.cu = cu;
+    p.dq = dq; p.dk = dk; p.dv = dv; p.dgv = dg; p.dbv = db; p.dwv = dw; p.dh0 = dh0;
+    p.ws = static_cast<char*>(workspace);
+    return vec_launch_bwd(p, workspace_is_fresh_from_fwd != 0, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? GDN_OK : GDN_ERR_CUDA;
 }
 
 gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream) {

@@ -77,6 +77,34 @@ inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, siz
     return L;
 }
 
+// Layout of the channel-wise FFMA family: everything fp32; gamma is per channel ([CH, 64, d_k]), no chunk operator.
+inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
+    WsLayout L{};
+    const size_t Ttot = (size_t)d.B * (size_t)d.T;
+    L.max_chunks = (int)((Ttot + kC - 1) / kC + (size_t)d.N);
+    const size_t CH = (size_t)L.max_chunks * d.H;
+    size_t o = sizeof(WsHeader);
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    L.seq_first = take(4 * ((size_t)d.N + 1));
+    L.chunk_seq = take(4 * (size_t)L.max_chunks);
+    L.chunk_tok0 = take(4 * (size_t)L.max_chunks);
+    L.chunk_len = take(4 * (size_t)L.max_chunks);
+    L.gamma = take(4 * CH * kC * d.d_k);
+    L.Tm = take(4 * CH * kC * kC);
+    L.W = take(4 * CH * kC * d.d_k);
+    L.Ut = take(4 * CH * kC * d.d_v);
+    L.Nm = L.Bf = o;
+    L.hc = take(4 * CH * d.d_k * d.d_v);
+    L.fwd_end = o;
+    L.E = take(4 * CH * d.d_k * d.d_v);
+    L.dhn = take(4 * CH * d.d_k * d.d_v);
+    L.Pm = take(4 * CH * kC * kC);
+    L.scratch_per_ch = scratch_per_ch;
+    L.scratch = take(scratch_per_ch * CH);
+    L.total = o;
+    return L;
+}
+
 // Everything a kernel needs to know about one call.
 struct Problem {
     gdn_desc d;
@@ -86,6 +114,9 @@ struct Problem {
     const int32_t* cu;
     void *o, *dq, *dk, *dv;
     float *hT, *dg, *dbeta, *dh0;
+    // channel-wise entry points only: gate vectors g, b [.., d_k], w [.., d_v] and their gradients (g, dg above unused)
+    const float *gv, *bv, *wv;
+    float *dgv, *dbv, *dwv;
     char* ws;
     WsLayout L;
 };
@@ -117,6 +148,10 @@ struct SmemLimitOnce {
     }
 };
 
+gdn_status check_desc(const gdn_desc* d);                       // shape / dtype envelope
+gdn_status check_seq(const gdn_desc& d, const int32_t* cu);     // B, N against cu_seqlens
+void call_begin();                                              // stage-timing bookkeeping at the top of an entry point
+
 // Host-side argument checks of gdn_bwd (everything that can be refused before a launch), shared with the entry point
 // that brings its own workspace.
 gdn_status check_bwd_args(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g, const float* beta,
@@ -129,6 +164,11 @@ cudaError_t launch_table(const Problem& p, cudaStream_t st);
 cudaError_t simt_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t simt_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 size_t simt_scratch_per_chunkhead(const gdn_desc& d);
+
+// FFMA family for per-channel gates (Eq. 1 with gate vectors).
+cudaError_t vec_launch_fwd(const Problem& p, cudaStream_t st);
+cudaError_t vec_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
+size_t vec_scratch_per_chunkhead(const gdn_desc& d);
 
 // tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
 extern thread_local int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank

@@ -178,3 +178,43 @@ class HostBackward:
             st = binding.gdn_last_device_status(sl["ws"])
             if st != binding.GDN_OK:
                 raise binding.GdnError(st, "device status")
+
+
+# ---- entry points with per-channel gates ----
+def to_device_channelwise(wl: Workload, device="cuda:0", want_o: bool = False) -> DeviceBuffers:
+    io = _io_dtype(wl)
+    dev = torch.device(device)
+    t = lambda a, dt: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dt).to(dev)
+    inputs = dict(q=t(wl.q, io), k=t(wl.k, io), v=t(wl.v, io), dO=t(wl.dO, io), g=t(wl.gv, torch.float32),
+                  b=t(wl.bv, torch.float32), w=t(wl.wv, torch.float32), h0=t(wl.h0, torch.float32),
+                  dhT=t(wl.dhT, torch.float32), cu_seqlens=t(wl.cu_seqlens, torch.int32) if wl.varlen else None)
+    Tt, H, N = wl.T_total, wl.H, wl.N
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=dev)
+    outputs = dict(dq=z((Tt, H, wl.d_k), io), dk=z((Tt, H, wl.d_k), io), dv=z((Tt, H, wl.d_v), io),
+                   dg=z((Tt, H, wl.d_k), torch.float32), db=z((Tt, H, wl.d_k), torch.float32),
+                   dw=z((Tt, H, wl.d_v), torch.float32), dh0=z((N, H, wl.d_k, wl.d_v), torch.float32),
+                   o=z((Tt, H, wl.d_v), io) if want_o else None,
+                   hT=z((N, H, wl.d_k, wl.d_v), torch.float32) if want_o else None)
+    desc = desc_for(wl)
+    _, bwd_bytes = binding.gdn_workspace_bytes_channelwise(desc)
+    ws = torch.empty(bwd_bytes, dtype=torch.uint8, device=dev)
+    return DeviceBuffers(desc=desc, inputs=inputs, outputs=outputs, workspace=ws)
+
+
+def run_fwd_channelwise(buf: DeviceBuffers, stream=None) -> None:
+    i, o = buf.inputs, buf.outputs
+    binding.gdn_fwd_recompute_channelwise(buf.desc, i["q"], i["k"], i["v"], i["g"], i["b"], i["w"], i["h0"],
+                                          i["cu_seqlens"], o["o"], o["hT"], buf.workspace, stream=stream)
+
+
+def run_bwd_channelwise(buf: DeviceBuffers, fresh: int = 0, stream=None) -> None:
+    i, o = buf.inputs, buf.outputs
+    binding.gdn_bwd_channelwise(buf.desc, i["q"], i["k"], i["v"], i["g"], i["b"], i["w"], i["h0"], i["dO"], i["dhT"],
+                                i["cu_seqlens"], o["dq"], o["dk"], o["dv"], o["dg"], o["db"], o["dw"], o["dh0"],
+                                buf.workspace, workspace_is_fresh_from_fwd=fresh, stream=stream)
+
+
+def backward_channelwise(wl: Workload, device="cuda:0") -> Dict[str, np.ndarray]:
+    buf = to_device_channelwise(wl, device)
+    run_bwd_channelwise(buf)
+    return fetch(buf)

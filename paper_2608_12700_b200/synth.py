@@ -73,6 +73,10 @@ class Workload:
     beta: Optional[np.ndarray] = field(repr=False, default=None)
     h0: Optional[np.ndarray] = field(repr=False, default=None)
     dhT: Optional[np.ndarray] = field(repr=False, default=None)
+    # channel-wise workloads only: gate vectors g, b [T_total, H, d_k] and w [T_total, H, d_v] (float32)
+    gv: Optional[np.ndarray] = field(repr=False, default=None)
+    bv: Optional[np.ndarray] = field(repr=False, default=None)
+    wv: Optional[np.ndarray] = field(repr=False, default=None)
 
     @property
     def N(self) -> int:
@@ -102,7 +106,7 @@ class Workload:
             d_k=self.d_k, d_v=self.d_v, chunk=self.chunk, scale=self.scale, delta_rule=self.delta_rule,
             seed=self.seed, cu_seqlens=self.cu_seqlens, varlen=self.varlen,
             q=sl(self.q), k=sl(self.k), v=sl(self.v), dO=sl(self.dO), g=sl(self.g), beta=sl(self.beta),
-            h0=sl(self.h0), dhT=sl(self.dhT))
+            h0=sl(self.h0), dhT=sl(self.dhT), gv=sl(self.gv), bv=sl(self.bv), wv=sl(self.wv))
 
 
 def _softplus(z):
@@ -149,6 +153,34 @@ def make_workload(name: str, *, dtype: str, H: int, d_k: int, d_v: int, seed: in
     return Workload(name=name, dtype=dtype, B=B, T=T, H=H, d_k=d_k, d_v=d_v, chunk=chunk, scale=scale,
                     delta_rule=delta_rule, seed=seed, cu_seqlens=cu.astype(np.int32), varlen=varlen,
                     q=q, k=k, v=v, dO=dO, g=g, beta=beta if delta_rule else None, h0=h0, dhT=dhT)
+
+
+def make_channelwise(name: str, *, member: str = "gdn", gate_seed: int = 0, **kw) -> Workload:
+    """A workload for the entry points with per-channel gates: the tensors of make_workload plus gate vectors
+    gv, bv [T_total, H, d_k] and wv [T_total, H, d_v], drawn like their scalar counterparts (log-decay
+    -g_scale * softplus(N(0,1)) per channel, erase and write gates sigmoid(N(0,1))).  `member` picks the row of the
+    family table: "gdn" independent vectors, "kda" one beta per token broadcast to both gates, "gla" erase 0, write 1."""
+    g_scale = kw.get("g_scale", 0.1)
+    wl = make_workload(name, **kw)
+    rng = np.random.Generator(np.random.PCG64([wl.seed, 7919 + gate_seed]))
+    Tt, H = wl.T_total, wl.H
+    sig = lambda z: (1.0 / (1.0 + np.exp(-z.astype(np.float64)))).astype(np.float32)
+    wl.gv = (-g_scale * _softplus(rng.standard_normal((Tt, H, wl.d_k), dtype=np.float32).astype(np.float64))).astype(np.float32)
+    if member == "gdn":
+        wl.bv = sig(rng.standard_normal((Tt, H, wl.d_k), dtype=np.float32))
+        wl.wv = sig(rng.standard_normal((Tt, H, wl.d_v), dtype=np.float32))
+    elif member == "kda":
+        beta = sig(rng.standard_normal((Tt, H, 1), dtype=np.float32))
+        wl.bv = np.ascontiguousarray(np.broadcast_to(beta, (Tt, H, wl.d_k)))
+        wl.wv = np.ascontiguousarray(np.broadcast_to(beta, (Tt, H, wl.d_v)))
+    elif member == "gla":
+        wl.bv = np.zeros((Tt, H, wl.d_k), dtype=np.float32)
+        wl.wv = np.ones((Tt, H, wl.d_v), dtype=np.float32)
+    else:
+        raise ValueError(f"unknown family member {member!r}")
+    wl.g = None
+    wl.beta = None
+    return wl
 
 
 def draw_packed_lengths(seed: int, n_seq: int = 8, lo: int = 256, hi: int = 8192, total: int = 32768):
