@@ -127,7 +127,7 @@ def fit(member, io=torch.float32, d=64, steps=60):
         loss = F.mse_loss(student(x), target)
         loss.backward()
         opt.step()
-        losses.append(float(loss))
+        losses.append(float(loss.detach()))
     return losses
 
 
