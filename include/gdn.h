@@ -208,6 +208,14 @@ gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* l
 gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
                           float* host_out);
 gdn_status gdn_debug_force_family(int32_t family);
+/* gdn_debug_inject_timeout(1): the next gdn_bwd of the calling thread that runs on the tcgen05 d = 128 family (and
+ * recomputes the forward) exercises the library's failure path without faulting anything: for that one call the
+ * bounded device-side waits give up after a millisecond instead of two seconds, and the first chunk-level kernel
+ * leaves out one of its input loads, so the wait for it runs out.  The CTAs leave through their normal teardown
+ * (tensor memory released, no copy in flight), the remaining kernels of the call see the status word and write
+ * nothing, gdn_bwd itself returns GDN_OK and gdn_last_device_status reports GDN_ERR_DEVICE_TIMEOUT.  The next call
+ * is a normal one.  0 cancels a pending request. */
+gdn_status gdn_debug_inject_timeout(int32_t on);
 
 #ifdef __cplusplus
 }

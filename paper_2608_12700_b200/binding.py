@@ -24,7 +24,7 @@ EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_devi
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
            "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc",
            "gdn_noalloc_last_device_status", "gdn_workspace_bytes_channelwise", "gdn_fwd_recompute_channelwise",
-           "gdn_bwd_channelwise"]
+           "gdn_bwd_channelwise", "gdn_debug_inject_timeout"]
 
 
 class gdn_desc(ctypes.Structure):
@@ -85,6 +85,8 @@ def lib():
         L.gdn_debug_read.argtypes = [D, P, ctypes.c_char_p, I, I, P]
         L.gdn_debug_force_family.restype = I
         L.gdn_debug_force_family.argtypes = [I]
+        L.gdn_debug_inject_timeout.restype = I
+        L.gdn_debug_inject_timeout.argtypes = [I]
         _lib = L
     return _lib
 
@@ -245,3 +247,8 @@ def gdn_bwd_channelwise(desc, q, k, v, g, b, w, h0, dO, dhT, cu_seqlens, dq, dk,
     if check and s != GDN_OK:
         raise GdnError(s, "gdn_bwd_channelwise")
     return s
+
+
+def gdn_debug_inject_timeout(on=True) -> None:
+    """The next gdn_bwd of this thread on the tcgen05 d = 128 family makes one bounded device-side wait run out."""
+    lib().gdn_debug_inject_timeout(1 if on else 0)

@@ -265,6 +265,11 @@ gdn_status gdn_debug_force_family(int32_t family) {
     return GDN_OK;
 }
 
+gdn_status gdn_debug_inject_timeout(int32_t on) {
+    g_inject_timeout = on ? 1 : 0;
+    return GDN_OK;
+}
+
 gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const char* what, int32_t chunk, int32_t head,
                           float* host_out) {
     gdn_status s = check_desc(desc);

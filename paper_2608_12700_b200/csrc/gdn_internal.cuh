@@ -172,6 +172,7 @@ size_t vec_scratch_per_chunkhead(const gdn_desc& d);
 
 // tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
 extern thread_local int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank
+extern thread_local int g_inject_timeout;   // debugging hook: the next gdn_bwd of this family provokes a device-side time-out
 bool tc_supported(const gdn_desc& d);
 // Form of the carries for a descriptor: one rule for the forward, the backward and a backward that consumes a workspace
 // fresh from the forward, so that the layout of a workspace does not depend on which call sized it.

@@ -42,6 +42,8 @@ struct TcParams {
     int with_bwd;                          // prep: also produce E
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
     int lowrank;                           // carries in low-rank form (tc_scan_lr): tc_prep makes no Nm, Bf
+    int withhold;                          // debugging hook: tc_prep leaves out one of its first loads, so that the wait
+                                           // for it runs out (exercises the time-out path without any fault)
 };
 
 // Blocked inverse of I + A (unit lower triangular), fp32 in shared memory, rows of kLdi floats:
@@ -363,7 +365,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     if (warp == 0) { fetch_gates(xn); make_gates(0, xn.ch); }
     // first trip: the inputs are loaded at once, one instruction per warp
     if (issuer) { mbar_expect_tx(&bar_qk, 32768); mbar_expect_tx(&bar_vo, VO_BYTES); }
-    if (lane == 0 && warp < 8) load_piece(warp, xn);
+    if (lane == 0 && warp < 8 && !(P.withhold && warp == 0)) load_piece(warp, xn);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
     const ChunkInfo x = xn;
@@ -603,6 +605,8 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     }
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
+
+#include "tc_prep_split.cuh"
 
 // ------------------------------------------------------------------------------------------------
 // tc_scan: forward and reverse inter-chunk carries, one CTA per (chain, direction).
@@ -1018,6 +1022,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // Persistent: a CTA walks over chunk-heads blockIdx.x, blockIdx.x + gridDim.x, ...  While it works on one, the
     // tiles of its next one are loaded into the regions the current one has finished with.
     const int H = p.d.H;
+    if (reinterpret_cast<const WsHeader*>(p.ws)->status != GDN_OK) return;   // an earlier stage gave up: nothing is written
     const int n_items = n_chunks_of(p) * H;
     if ((int)blockIdx.x >= n_items) return;
     const float sc = p.d.scale;
@@ -1660,6 +1665,8 @@ bool tc_supported(const gdn_desc& d) {
     return d.dtype == GDN_BF16 && d.d_k == 128 && d.d_v == 128 && d.delta_rule == 1 && d.chunk == kC;
 }
 
+thread_local int g_inject_timeout = 0;   // set by gdn_debug_inject_timeout, consumed by the next gdn_bwd of this family
+
 static int sm_count();
 // When one CTA per (chain, direction) of the backward fills more than half of the SMs the carries are bound by HBM
 // bandwidth, and the low-rank form moves less.  With fewer chains a step's latency counts, and the operator form needs one
@@ -1674,6 +1681,7 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
     P.with_bwd = with_bwd ? 1 : 0;
     P.scan_dirs = scan_dirs;
     P.lowrank = tc_carries_lowrank(p.d) ? 1 : 0;
+    P.withhold = 0;
     const uint64_t rows = (uint64_t)p.Ttot, cols = (uint64_t)p.d.H * D, pitch = cols * 2;
     if (!tc::make_tmap_bf16_2d(&P.tm_q, p.q, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
@@ -1717,6 +1725,18 @@ static int sm_count() {
     return cached[dev];
 }
 
+// The two small preparation kernels, two CTAs per SM.
+static cudaError_t launch_factors(const TcParams& P, cudaStream_t st) {
+    static SmemLimitOnce done;
+    const int items = P.p.L.max_chunks * P.p.d.H, ctas = 2 * sm_count();
+    return launch_chunk_kernel(tc_factors_kernel, done, factors::SMEM_BYTES, ST_PREP, items < ctas ? items : ctas, split::kT, P, st);
+}
+static cudaError_t launch_eprep(const TcParams& P, cudaStream_t st) {
+    static SmemLimitOnce done;
+    const int items = P.p.L.max_chunks * P.p.d.H, ctas = 2 * sm_count();
+    return launch_chunk_kernel(tc_eprep_kernel, done, eprep::SMEM_BYTES, ST_EPREP, items < ctas ? items : ctas, split::kT, P, st);
+}
+
 static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done;
     static SmemLimitOnce done2;
@@ -1754,28 +1774,46 @@ static cudaError_t launch_table_if_needed(const Problem& p, cudaStream_t st) {
     return (p.cu || p.Ttot == 0) ? launch_table(p, st) : cudaSuccess;
 }
 
+// Carries in low-rank form take the chunk factors from tc_factors; in operator form they also need Nm and Bf, which
+// only the fused tc_prep makes.
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st) {
     TcParams P;
     cudaError_t e = launch_table_if_needed(p, st);
     if (e != cudaSuccess) return e;
     if (p.Ttot == 0) return empty_call(p, false, st);
     if (!fill_params(P, p, false, 0)) return cudaErrorUnknown;
-    if ((e = launch_prep(P, st)) != cudaSuccess) return e;
+    if ((e = P.lowrank ? launch_factors(P, st) : launch_prep(P, st)) != cudaSuccess) return e;
     if ((e = launch_scan(P, st)) != cudaSuccess) return e;
     return p.o ? launch_out(P, st) : cudaSuccess;
 }
 
-// With a workspace fresh from gdn_fwd_recompute the forward carry is not repeated; the chunk factors are
-// rebuilt together with E, which needs dO.
+// With a workspace fresh from gdn_fwd_recompute nothing of the forward is repeated: T, W, U~ and the per-chunk states
+// are taken from it, and only what needs dO is built (P, E; tc_eprep), followed by the reverse carry and the
+// gradient stage.
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st) {
     TcParams P;
     cudaError_t e = launch_table_if_needed(p, st);
     if (e != cudaSuccess) return e;
     if (p.Ttot == 0) return empty_call(p, true, st);
     if (!fill_params(P, p, true, skip_recompute ? 1 : 2)) return cudaErrorUnknown;
-    if ((e = launch_prep(P, st)) != cudaSuccess) return e;
+    const bool inject = g_inject_timeout && !skip_recompute;
+    if (inject) {   // debugging hook, this call only: a millisecond of patience, and tc_prep withholds one load
+        const unsigned long long ns = 1000000ull;
+        g_inject_timeout = 0;
+        P.withhold = 1;
+        if ((e = cudaMemcpyToSymbolAsync(g_wait_limit_ns, &ns, sizeof(ns), 0, cudaMemcpyHostToDevice, st)) != cudaSuccess) return e;
+    }
+    // (the closed arm keeps the fused kernel: it reads k once and never moves W through HBM on its way to E; measured on
+    // B = 4, T = 2048, H = 16: fused 100 us, tc_factors + tc_eprep 67 + 56 us)
+    if ((e = skip_recompute ? launch_eprep(P, st) : launch_prep(P, st)) != cudaSuccess) return e;
     if ((e = launch_scan(P, st)) != cudaSuccess) return e;
-    return launch_intra(P, st);
+    e = launch_intra(P, st);
+    if (inject) {
+        const unsigned long long ns = 2000000000ull;
+        const cudaError_t e2 = cudaMemcpyToSymbolAsync(g_wait_limit_ns, &ns, sizeof(ns), 0, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = e2;
+    }
+    return e;
 }
 
 }  // namespace gdn

@@ -53,6 +53,9 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
+// How long a bounded wait polls before it gives up (one copy per translation unit; two seconds unless the host-side
+// debugging hook that provokes a time-out has shortened it for one call).
+static __device__ unsigned long long g_wait_limit_ns = 2000000000ull;
 // Bounded wait: gives up after about two seconds and returns false; the caller records the failure and
 // leaves through its normal teardown (no trap, no endless spin).  Only the first probe is inlined at a wait site: a
 // kernel has dozens of them and the polling loop with its time-out would multiply the code size (the instruction
@@ -66,7 +69,7 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > 2000000000ull) return false;
+        if (global_ns() - t0 > g_wait_limit_ns) return false;
     }
 }
 // The same wait with its polling loop at the wait site: no call, so nothing has to be saved around it.  For the small
@@ -80,7 +83,7 @@ __device__ __forceinline__ bool mbar_wait_inline(uint64_t* bar, uint32_t parity)
         if ((i & 255u) == 0) {
             const uint64_t t = global_ns();
             if (t0 == 0) t0 = t;
-            else if (t - t0 > 2000000000ull) return false;
+            else if (t - t0 > g_wait_limit_ns) return false;
         }
     }
 }
