@@ -36,6 +36,9 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used when profiling)")
     ap.add_argument("--no-others", action="store_true", help="skip the save-forward arm and the other configurations")
+    ap.add_argument("--arm", default="closed", choices=["closed", "save_forward"],
+                    help="closed: gdn_bwd recomputes the forward (the headline); save_forward: every step is "
+                         "gdn_fwd_recompute followed by gdn_bwd on its workspace (used when profiling that arm)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="target CPU time of the oracle sample")
     return ap.parse_args()
 
@@ -116,13 +119,13 @@ def path_roofline(wl, peaks, ms_per_step):
                 peak_source=peaks["source"])
 
 
-def stage_pass(buf, runner, binding, calls):
+def stage_pass(buf, runner, binding, calls, step=None):
     """Per-kernel durations from a separate, untimed-for-the-headline pass: every launch bracketed by events."""
     import torch
     binding.gdn_stage_timing_enable(1)
     binding.gdn_stage_timing_read()
     for _ in range(calls):
-        runner.run_bwd(buf)
+        step() if step else runner.run_bwd(buf)
     torch.cuda.synchronize()
     stages = binding.gdn_stage_timing_read()
     binding.gdn_stage_timing_enable(False)
@@ -168,13 +171,20 @@ def run_ours(args):
             raise binding.GdnError(st, where)
 
     # ---------------- device-resident timing: nothing but the K calls between the two events ----------------
+    def step():
+        if args.arm == "closed":
+            runner.run_bwd(buf)
+        else:
+            runner.run_fwd(buf)
+            runner.run_bwd(buf, fresh=1)
+
     for _ in range(warmup):
-        runner.run_bwd(buf)
+        step()
     check_status(buf, "warm-up")
     sampler = benchutil.ClockSampler(local, period_s=0.0005)
     launches0 = binding.gdn_launch_count()
     sampler.start()
-    elapsed_ms = time_steps(lambda: runner.run_bwd(buf), args.steps, barrier, stream)
+    elapsed_ms = time_steps(step, args.steps, barrier, stream)
     sampler.stop()
     launches = binding.gdn_launch_count() - launches0
     check_status(buf, "timed region")
@@ -184,7 +194,7 @@ def run_ours(args):
 
     # ---------------- per-kernel durations: a pass of its own, outside the headline ----------------
     stage_calls = max(3, min(args.steps, 10))
-    stage_ms = stage_pass(buf, runner, binding, stage_calls)
+    stage_ms = stage_pass(buf, runner, binding, stage_calls, step)
 
     # ---------------- the arm that consumes a workspace saved by the forward (Section 4.5) ----------------
     save_forward = None
@@ -250,7 +260,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": workload_config(wl),
+        "config": dict(workload_config(wl), arm=args.arm),
         "kernel_path": family,
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -281,10 +291,15 @@ def time_other_configs(args, peaks, barrier, stream, dev):
     import torch
     from paper_2608_12700_b200 import binding, runner, synth
     out = {}
-    for idx in range(5):
+    # the five configurations, and the other shape of the paper's verification envelope (d_k = 128, d_v = 64; Section 4.5)
+    # at the batch and length of the headline
+    for idx in list(range(5)) + ["dk128_dv64"]:
         if idx == args.config:
             continue
-        wl = synth.config(idx)
+        if idx == "dk128_dv64":
+            wl = synth.make_workload("envelope_bf16_dk128_dv64", dtype="bf16", B=4, T=2048, H=16, d_k=128, d_v=64, seed=6, states=True)
+        else:
+            wl = synth.config(idx)
         buf = runner.to_device(wl, dev)
         for _ in range(3):
             runner.run_bwd(buf)

@@ -47,7 +47,7 @@ namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-enum class Path { None, SimtF32, SimtBf16, TcBf16, Tc64Bf16 };
+enum class Path { None, SimtF32, SimtBf16, TcBf16, Tc64Bf16, TcBf16Padded };
 
 // Debug overrides of the dispatch are per thread: a thread that forces a family cannot change the workspace size
 // another thread is computing at that moment.
@@ -62,6 +62,7 @@ Path pick_path(const gdn_desc& d) {
         if (g_force_family == 1) return Path::SimtBf16;
         if (tc_supported(d)) return Path::TcBf16;
         if (tc64_supported(d)) return Path::Tc64Bf16;
+        if (tc_padded_supported(d)) return Path::TcBf16Padded;
         return Path::SimtBf16;
     }
     return Path::None;
@@ -72,6 +73,14 @@ WsLayout layout_for(const gdn_desc& d) {
     // The d = 128 family keeps the chunk operator Nm and the additive term Bf only when its carries use them.
     if (pick_path(d) == Path::TcBf16) return make_layout(d, 2, 2, 0, !tc_carries_lowrank(d));
     if (pick_path(d) == Path::Tc64Bf16) return make_layout(d, 2, 2, 0);
+    if (pick_path(d) == Path::TcBf16Padded) {   // the widened problem's layout, then the padded copies; one size for both calls
+        const gdn_desc w = tc_padded_desc(d);
+        WsLayout L = make_layout(w, 2, 2, 0, !tc_carries_lowrank(w));
+        L.scratch = align_up(L.total, 256);
+        L.total = L.scratch + tc_padded_extra_bytes(d);
+        L.fwd_end = L.total;
+        return L;
+    }
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
     return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
 }
@@ -150,7 +159,13 @@ gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k,
     p.ws = static_cast<char*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const Path path = pick_path(*desc);
-    const cudaError_t e = path == Path::TcBf16 ? tc_launch_fwd(p, st) : path == Path::Tc64Bf16 ? tc64_launch_fwd(p, st) : simt_launch_fwd(p, st);
+    cudaError_t e;
+    if (path == Path::TcBf16Padded) {
+        const gdn_desc w = tc_padded_desc(*desc);
+        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), false, false, st);
+    } else {
+        e = path == Path::TcBf16 ? tc_launch_fwd(p, st) : path == Path::Tc64Bf16 ? tc64_launch_fwd(p, st) : simt_launch_fwd(p, st);
+    }
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
@@ -171,8 +186,14 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const bool fresh = workspace_is_fresh_from_fwd != 0;
     const Path path = pick_path(*desc);
-    const cudaError_t e = path == Path::TcBf16 ? tc_launch_bwd(p, fresh, st)
-                          : path == Path::Tc64Bf16 ? tc64_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
+    cudaError_t e;
+    if (path == Path::TcBf16Padded) {
+        const gdn_desc w = tc_padded_desc(*desc);
+        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), true, fresh, st);
+    } else {
+        e = path == Path::TcBf16 ? tc_launch_bwd(p, fresh, st)
+            : path == Path::Tc64Bf16 ? tc64_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
+    }
     return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
@@ -277,6 +298,7 @@ gdn_status gdn_debug_read(const gdn_desc* desc, const void* workspace, const cha
     if (!workspace || !what || !host_out) return GDN_ERR_NULL_ARG;
     const WsLayout L = layout_for(*desc);
     if (chunk < 0 || chunk >= L.max_chunks || head < 0 || head >= desc->H) return GDN_ERR_BAD_SHAPE;
+    if (pick_path(*desc) == Path::TcBf16Padded) return GDN_ERR_UNSUPPORTED_SHAPE;   // (stored as the widened problem)
     const bool tcp = pick_path(*desc) == Path::TcBf16 || pick_path(*desc) == Path::Tc64Bf16;
     const size_t ch = (size_t)chunk * desc->H + head;
     const int dk = desc->d_k, dv = desc->d_v;
@@ -349,6 +371,7 @@ const char* gdn_kernel_path(const gdn_desc* desc) {
         case Path::SimtBf16: return "simt_bf16";
         case Path::TcBf16: return "tcgen05_bf16";
         case Path::Tc64Bf16: return "tcgen05_bf16_scalar_gate";
+        case Path::TcBf16Padded: return "tcgen05_bf16_padded";
         default: return nullptr;
     }
 }

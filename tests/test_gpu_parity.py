@@ -123,7 +123,9 @@ def test_kernel_family_dispatch():
     mk = lambda **kw: binding.make_desc(**dict(dict(B=1, T=64, H=1, d_k=128, d_v=128, N=1, dtype="bf16"), **kw))
     assert binding.gdn_kernel_path(mk()) == "tcgen05_bf16"
     assert binding.gdn_kernel_path(mk(dtype="f32")) == "simt_f32"
-    assert binding.gdn_kernel_path(mk(d_k=64, d_v=64)) == "simt_bf16"
+    assert binding.gdn_kernel_path(mk(d_k=64, d_v=64)) == "tcgen05_bf16_padded"
+    assert binding.gdn_kernel_path(mk(d_k=128, d_v=64)) == "tcgen05_bf16_padded"
+    assert binding.gdn_kernel_path(mk(d_k=64, d_v=128)) == "tcgen05_bf16_padded"
     assert binding.gdn_kernel_path(mk(delta_rule=0)) == "simt_bf16"
     assert binding.gdn_kernel_path(mk(d_k=64, d_v=64, delta_rule=0)) == "tcgen05_bf16_scalar_gate"
 
