@@ -36,6 +36,11 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (used when profiling)")
     ap.add_argument("--no-others", action="store_true", help="skip the save-forward arm and the other configurations")
+    ap.add_argument("--shape", default=None, metavar="B,T,H",
+                    help="instead of a configuration: bf16 GDN, d_k = d_v = 128, B sequences of T tokens, H heads, with "
+                         "states (value distributions of cfg1); used for kernel studies, not a bench line of its own")
+    ap.add_argument("--carries", default="auto", choices=["auto", "operator", "lowrank"],
+                    help="form of the inter-chunk carries of the tcgen05 d = 128 family (default: chosen by shape)")
     ap.add_argument("--arm", default="closed", choices=["closed", "save_forward"],
                     help="closed: gdn_bwd recomputes the forward (the headline); save_forward: every step is "
                          "gdn_fwd_recompute followed by gdn_bwd on its workspace (used when profiling that arm)")
@@ -147,13 +152,20 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = synth.config(args.config)
+    if args.shape:
+        B_, T_, H_ = (int(x) for x in args.shape.split(","))
+        wl = synth.make_workload(f"shape_B{B_}_T{T_}_H{H_}_bf16_d128", dtype="bf16", B=B_, T=T_, H=H_, d_k=128, d_v=128,
+                                 seed=3, states=True)
+    else:
+        wl = synth.config(args.config)
+    binding.gdn_debug_force_family({"auto": 0, "operator": 2, "lowrank": 3}[args.carries])
     if rank:   # every rank its own batch of the same shape (heads permuted: chains are independent)
         import numpy as np
         rng = np.random.default_rng(1000 + rank)
         perm = rng.permutation(wl.H)
+        name = wl.name
         wl = wl.take_heads(list(perm))
-        wl.name = synth.CONFIG_NAMES[args.config]
+        wl.name = name
     buf = runner.to_device(wl, dev)
     desc = buf.desc
     peaks = benchutil.load_peaks(ROOT)
@@ -241,7 +253,7 @@ def run_ours(args):
     else:
         roof = {"bound": "tensor", "achieved": path["algorithmic_flops"] / step_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    traffic = [recorded_traffic(k, wl, family) for k in stage_ms]
+    traffic = [recorded_traffic(k, wl, family, args.arm) for k in stage_ms]
     roof["traffic"] = sum(traffic) if traffic and all(t is not None for t in traffic) else None
     roof["traffic_over_algorithmic"] = roof["traffic"] / path["algorithmic_bytes"] if roof["traffic"] else None
     dom = max(stage_ms, key=stage_ms.get)
@@ -253,14 +265,14 @@ def run_ours(args):
         "peak_source": peaks["source"], "algorithmic_bytes": path["algorithmic_bytes"],
         "algorithmic_flops": path["algorithmic_flops"],
         "kernel": dom, "kernel_ms": stage_ms[dom], "kernel_algorithmic_bytes": dom_bytes,
-        "kernel_algorithmic_flops": dom_flops, "kernel_traffic": recorded_traffic(dom, wl, family),
+        "kernel_algorithmic_flops": dom_flops, "kernel_traffic": recorded_traffic(dom, wl, family, args.arm),
         "kernel_frac": max(d_hbm, d_tc) / (stage_ms[dom] * 1e-3),
         "kernel_bound": "hbm" if d_hbm >= d_tc else "tensor"})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": dict(workload_config(wl), arm=args.arm),
+        "config": dict(workload_config(wl), arm=args.arm, carries=args.carries),
         "kernel_path": family,
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -275,6 +287,7 @@ def run_ours(args):
         line["save_forward_arm"] = save_forward
     del buf
     torch.cuda.empty_cache()
+    binding.gdn_debug_force_family(0)
     if world == 1 and not args.no_others:
         line["other_configs"] = time_other_configs(args, peaks, barrier, stream, dev)
     if not args.no_cpu_baseline and world == 1:
@@ -354,7 +367,7 @@ def stage_algorithmic_work(stage, wl, io_bytes, family=""):
     return byts, flops
 
 
-def recorded_traffic(stage, wl, family=""):
+def recorded_traffic(stage, wl, family="", arm="closed"):
     """DRAM bytes per launch of the stage from the ncu captures summarised under profiles/ (bytes per
     chunk-head measured on a small case, scaled by the chunk-heads of this workload), or None."""
     path = os.path.join(ROOT, "profiles", "measured_traffic.json")
@@ -363,7 +376,9 @@ def recorded_traffic(stage, wl, family=""):
     with open(path) as f:
         rec = json.load(f)
     key = f"{stage}:{wl.dtype}:{wl.d_k}x{wl.d_v}:{wl.delta_rule}"
-    if family == "tcgen05_bf16" and stage in ("prep", "scans"):
+    if family == "tcgen05_bf16" and stage == "prep" and arm == "save_forward":
+        key = f"factors:{wl.dtype}:{wl.d_k}x{wl.d_v}:{wl.delta_rule}"   # the forward's share of the preparation
+    elif family == "tcgen05_bf16" and stage in ("prep", "scans"):
         from paper_2608_12700_b200 import binding, runner
         # the d = 128 family runs its carries in one of two forms with different traffic; the workspace size tells which
         desc = runner.desc_for(wl)
