@@ -144,8 +144,8 @@ gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream);
 const char* gdn_status_string(gdn_status s);
 
 /* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16",
- * "tcgen05_bf16_scalar_gate", "tcgen05_bf16_padded": bf16 delta-rule shapes with a head dimension of 64,
- * zero-padded onto the d = 128 tensor-core kernels inside the workspace),
+ * "tcgen05_bf16_scalar_gate", "tcgen05_bf16_padded": bf16 shapes with one or both head dimensions at 64 that have no
+ * kernels of their own, zero-padded onto the d = 128 tensor-core kernels inside the workspace),
  * or NULL for an unsupported descriptor.  Diagnostic only. */
 const char* gdn_kernel_path(const gdn_desc* desc);
 

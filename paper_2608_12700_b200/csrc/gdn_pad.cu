@@ -60,7 +60,7 @@ PadPlan plan_for(const gdn_desc& d) {
 }  // namespace
 
 bool tc_padded_supported(const gdn_desc& d) {
-    return d.dtype == GDN_BF16 && d.delta_rule == 1 && d.chunk == kC && (d.d_k == 64 || d.d_k == 128) && (d.d_v == 64 || d.d_v == 128) &&
+    return d.dtype == GDN_BF16 && d.chunk == kC && (d.d_k == 64 || d.d_k == 128) && (d.d_v == 64 || d.d_v == 128) &&
            !(d.d_k == 128 && d.d_v == 128);
 }
 gdn_desc tc_padded_desc(const gdn_desc& d) {

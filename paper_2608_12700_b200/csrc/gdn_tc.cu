@@ -323,16 +323,18 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     ChunkInfo xn;
     chunk_entry(p, xn, blockIdx.x);
     // Warp 0 owns the gates: lane l holds g (0 when padded) and the erase gate b of tokens l and l + 32.
-    float ng[2] = {0.f, 0.f}, nb[2] = {0.f, 0.f};
+    float ng[2] = {0.f, 0.f}, nb[2] = {0.f, 0.f}, nw[2] = {0.f, 0.f};
+    const bool delta = p.d.delta_rule != 0;   // off: erase gate 0, write gate 1 (T = I, W = 0 fall out of the same products)
     auto fetch_gates = [&](const ChunkInfo& c) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int i = lane + 32 * h;
-            ng[h] = nb[h] = 0.f;
+            ng[h] = nb[h] = nw[h] = 0.f;
             if (i < c.len) {
                 const size_t idx = (size_t)(c.tok0 + i) * H + c.hd;
                 ng[h] = p.g[idx];
-                nb[h] = p.beta[idx];
+                nb[h] = delta ? p.beta[idx] : 0.f;
+                nw[h] = delta ? nb[h] : 1.f;
             }
         }
     };
@@ -357,7 +359,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
             gs[1][i] = G;
             gs[2][i] = expf(gend - gc[h]);
             gs[3][i] = nb[h];
-            gs[4][i] = nb[h];
+            gs[4][i] = nw[h];
             gs[5][i] = nb[h] * G;
             reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)ch * kC + i] = gc[h];
         }
@@ -1029,7 +1031,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ __align__(16) float gate_sets[2][4][kC];   // two sets: a trip's gate arrays are written during the trip before
+    __shared__ __align__(16) float gate_sets[2][5][kC];   // two sets: a trip's gate arrays are written during the trip before
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
     __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_do, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
@@ -1183,14 +1185,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         const float* gsrc = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)c.ch * kC;
         ng = gsrc[threadIdx.x];
         ngend = gsrc[kC - 1];
-        nb = ((int)threadIdx.x < c.len) ? p.beta[(size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd] : 0.f;
+        nb = ((int)threadIdx.x < c.len && p.d.delta_rule) ? p.beta[(size_t)(c.tok0 + (int)threadIdx.x) * H + c.hd] : 0.f;
     };
     auto make_gates = [&](int set) {   // threads 0..63: the fetched values -> gate arrays of set `set`
         const int i = threadIdx.x;
         gate_sets[set][0][i] = ng * kLog2e;
         gate_sets[set][1][i] = expf(ng);
         gate_sets[set][2][i] = expf(ngend - ng);
-        gate_sets[set][3][i] = nb;
+        gate_sets[set][3][i] = nb;                                                    // erase gate
+        gate_sets[set][4][i] = p.d.delta_rule ? nb : (i < xn.len ? 1.f : 0.f);        // write gate (delta rule off: 0 and 1)
     };
     // dbeta and dg of the previous trip's chunk, from its token-wise partial sums (warps 0 and 1; see the trip's end)
     ChunkInfo xp = xn;
@@ -1200,7 +1203,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         const int i = threadIdx.x;
         auto tot = [&](int w) { return (red[w][0][i] + red[w][1][i]) + (red[w][2][i] + red[w][3][i]); };
         const float qdq = tot(0), dw = tot(1), db = tot(2), kcol = tot(3);
-        if (i < xp.len) p.dbeta[(size_t)(xp.tok0 + i) * H + xp.hd] = db + dw;
+        if (i < xp.len && p.dbeta) p.dbeta[(size_t)(xp.tok0 + i) * H + xp.hd] = db + dw;
         dgam[i] = fmaf(bb_prev, db, qdq - kcol);
         asm volatile("bar.sync 2, 64;" ::: "memory");
         if (warp == 0) {
@@ -1401,7 +1404,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         //   group A: dq = scale Gam (dO h^T) + (dP.D) K, staged ; acc = <q, dq>
         //   group B: dXk, dXv -> operand tiles ; acc = <v, dXv> (dw partial) ; dv = w dXv, staged
         float acc = 0.f;
-        const float coef = sc * Gam[tr], outscale = ga ? 1.f : bb[tr];
+        const float coef = sc * Gam[tr], outscale = ga ? 1.f : gate_sets[in_phase][4][tr];
         const unsigned char* dot_tile = sm + (ga ? QK : VT);   // q rows (128-row tile) or v rows (64-row tile)
         unsigned char* stage = sm + (ga ? STG_A : STG_B);
 #pragma unroll
@@ -1662,7 +1665,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_consta
 // host side
 // ------------------------------------------------------------------------------------------------
 bool tc_supported(const gdn_desc& d) {
-    return d.dtype == GDN_BF16 && d.d_k == 128 && d.d_v == 128 && d.delta_rule == 1 && d.chunk == kC;
+    return d.dtype == GDN_BF16 && d.d_k == 128 && d.d_v == 128 && d.chunk == kC;
 }
 
 thread_local int g_inject_timeout = 0;   // set by gdn_debug_inject_timeout, consumed by the next gdn_bwd of this family

@@ -76,14 +76,15 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
             pending = true;
         }
         if (warp == 0) {   // gate arrays of the chunk: lane l owns tokens l and l + 32
-            float gg[2] = {0.f, 0.f}, gb[2] = {0.f, 0.f};
+            float gg[2] = {0.f, 0.f}, gb[2] = {0.f, 0.f}, gw[2] = {0.f, 0.f};   // log decay, erase gate, write gate
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int i = lane + 32 * h;
                 if (i < x.len) {
                     const size_t idx = (size_t)(x.tok0 + i) * H + x.hd;
                     gg[h] = p.g[idx];
-                    gb[h] = p.beta[idx];
+                    gb[h] = p.d.delta_rule ? p.beta[idx] : 0.f;   // delta rule off: erase 0, write 1
+                    gw[h] = p.d.delta_rule ? gb[h] : 1.f;
                 }
             }
             float a = gg[0], b = gg[1];
@@ -103,7 +104,7 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
                 gates[1][i] = G;
                 gates[2][i] = expf(gend - gc[h]);
                 gates[3][i] = gb[h];
-                gates[4][i] = gb[h];
+                gates[4][i] = gw[h];
                 gates[5][i] = gb[h] * G;
                 reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + i] = gc[h];
             }

@@ -66,6 +66,26 @@ def test_scalar_gate_recurrence_ragged_with_states(family):
     assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))
 
 
+@pytest.mark.parametrize("dk,dv", [(128, 128), (128, 64), (64, 128)])
+def test_scalar_gate_recurrence_at_wide_heads(dk, dv, family):
+    """Delta rule off at head dimensions the d = 64 scalar-gate kernels do not cover: the GDN kernels run with erase
+    gate 0 and write gate 1 (T = I and W = 0 fall out of the same products), both carry forms, ragged, with states."""
+    for lengths, H in (([65, 128, 0, 37, 300], 2), ([130] * 10, 4)):     # few chains: operator form; 40 chains: low-rank
+        wl = small(f"beta_off_wide_{dk}_{dv}_{H}", dtype="bf16", lengths=lengths, H=H, d_k=dk, d_v=dv, delta_rule=0,
+                   g_scale=0.05, states=True, scale=0.5, seed=27)
+        got = runner.backward(wl)
+        check_against_oracle(wl, got)
+        buf = runner.to_device(wl, want_o=True)
+        runner.run_fwd(buf)
+        f = runner.fetch(buf)
+        ref = oracle_grads(wl)
+        assert rel(f["o"], ref["o"]) < TOL["bf16"] and rel(f["hT"], ref["hT"]) < TOL["bf16"]
+        runner.run_bwd(buf, fresh=1)
+        fresh = runner.fetch(buf)
+        for n in ("dq", "dk", "dv", "dg", "dh0"):
+            assert np.array_equal(fresh[n], got[n]), n
+
+
 def test_scalar_gate_forward_outputs(family):
     wl = small("beta_off_fwd", dtype="bf16", lengths=[70, 130], H=2, d_k=64, d_v=64, delta_rule=0, states=True, seed=23)
     buf = runner.to_device(wl, want_o=True)
@@ -126,7 +146,8 @@ def test_kernel_family_dispatch():
     assert binding.gdn_kernel_path(mk(d_k=64, d_v=64)) == "tcgen05_bf16_padded"
     assert binding.gdn_kernel_path(mk(d_k=128, d_v=64)) == "tcgen05_bf16_padded"
     assert binding.gdn_kernel_path(mk(d_k=64, d_v=128)) == "tcgen05_bf16_padded"
-    assert binding.gdn_kernel_path(mk(delta_rule=0)) == "simt_bf16"
+    assert binding.gdn_kernel_path(mk(delta_rule=0)) == "tcgen05_bf16"
+    assert binding.gdn_kernel_path(mk(d_v=64, delta_rule=0)) == "tcgen05_bf16_padded"
     assert binding.gdn_kernel_path(mk(d_k=64, d_v=64, delta_rule=0)) == "tcgen05_bf16_scalar_gate"
 
 
