@@ -323,18 +323,16 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
     ChunkInfo xn;
     chunk_entry(p, xn, blockIdx.x);
     // Warp 0 owns the gates: lane l holds g (0 when padded) and the erase gate b of tokens l and l + 32.
-    float ng[2] = {0.f, 0.f}, nb[2] = {0.f, 0.f}, nw[2] = {0.f, 0.f};
-    const bool delta = p.d.delta_rule != 0;   // off: erase gate 0, write gate 1 (T = I, W = 0 fall out of the same products)
+    float ng[2] = {0.f, 0.f}, nb[2] = {0.f, 0.f};
     auto fetch_gates = [&](const ChunkInfo& c) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const int i = lane + 32 * h;
-            ng[h] = nb[h] = nw[h] = 0.f;
+            ng[h] = nb[h] = 0.f;
             if (i < c.len) {
                 const size_t idx = (size_t)(c.tok0 + i) * H + c.hd;
                 ng[h] = p.g[idx];
-                nb[h] = delta ? p.beta[idx] : 0.f;
-                nw[h] = delta ? nb[h] : 1.f;
+                if (p.d.delta_rule) nb[h] = p.beta[idx];   // delta rule off: erase gate 0 (T = I, W = 0 fall out of the same products)
             }
         }
     };
@@ -359,7 +357,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_prep_kernel(const __
             gs[1][i] = G;
             gs[2][i] = expf(gend - gc[h]);
             gs[3][i] = nb[h];
-            gs[4][i] = nw[h];
+            gs[4][i] = p.d.delta_rule ? nb[h] : (i < xn.len ? 1.f : 0.f);   // write gate (delta rule off: 1)
             gs[5][i] = nb[h] * G;
             reinterpret_cast<float*>(p.ws + p.L.gamma)[(size_t)ch * kC + i] = gc[h];
         }
@@ -1807,7 +1805,7 @@ cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st
         if ((e = cudaMemcpyToSymbolAsync(g_wait_limit_ns, &ns, sizeof(ns), 0, cudaMemcpyHostToDevice, st)) != cudaSuccess) return e;
     }
     // (the closed arm keeps the fused kernel: it reads k once and never moves W through HBM on its way to E; measured on
-    // B = 4, T = 2048, H = 16: fused 100 us, tc_factors + tc_eprep 67 + 56 us)
+    // B = 4, T = 2048, H = 16: fused 99 us, tc_factors + tc_eprep 62 + 45 us)
     if ((e = skip_recompute ? launch_eprep(P, st) : launch_prep(P, st)) != cudaSuccess) return e;
     if ((e = launch_scan(P, st)) != cudaSuccess) return e;
     e = launch_intra(P, st);

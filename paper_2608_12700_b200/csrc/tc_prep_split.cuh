@@ -5,8 +5,9 @@
 //
 // Each holds about 105 KB of shared memory and 256 columns of tensor memory, so that two CTAs share an SM: a CTA works
 // through the dependent phases of one chunk-head (product -> readout -> product ...) while its neighbour is in another
-// phase of another chunk-head, which is what keeps the tensor pipe and the load/store path busy.  There is no
-// look-ahead inside a CTA: the neighbour is the look-ahead.  A backward that consumes a workspace fresh from the
+// phase of another chunk-head, which is what keeps the tensor pipe and the load/store path busy.  A trip's inputs are
+// dead once its last product is done, so the next trip's are loaded right then, under the last readout and the stores
+// (look-ahead without a second buffer).  A backward that consumes a workspace fresh from the
 // forward runs tc_eprep alone (T, W, U~ are reused: no product, inversion or store of the forward is repeated).
 // The fused tc_prep kernel remains for carries in operator form, which also need Nm and Bf.
 #pragma once
@@ -62,31 +63,40 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
     float* Sf = reinterpret_cast<float*>(sm + WU);
     bool ok = true, pending = false;
     uint32_t mma_phase = 0, in_phase = 0;
+    // K and V of a trip are dead once its last product is done, so the next trip's are loaded right then, under the last
+    // readout and the stores; the gate values of the next trip are fetched into registers at the same moment.
+    auto issue_loads = [&](const ChunkInfo& c) {   // thread 0
+        mbar_expect_tx(&bar_in, 32768);
+        for (int cb = 0; cb < 2; ++cb) {
+            tma_load_2d(sm + KV + cb * 16384, &P.tm_k, c.hd * D + cb * 64, c.tok0, &bar_in);
+            tma_load_2d(sm + KV + cb * 16384 + 8192, &P.tm_v, c.hd * D + cb * 64, c.tok0, &bar_in);
+        }
+        pending = true;
+    };
+    float gg[2] = {0.f, 0.f}, gb[2] = {0.f, 0.f}, gw[2] = {0.f, 0.f};   // warp 0: log decay, erase gate, write gate of tokens lane, lane + 32
+    auto fetch_gates = [&](const ChunkInfo& c) {   // warp 0
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int i = lane + 32 * h;
+            gg[h] = gb[h] = gw[h] = 0.f;
+            if (i < c.len) {
+                const size_t idx = (size_t)(c.tok0 + i) * H + c.hd;
+                gg[h] = p.g[idx];
+                gb[h] = p.d.delta_rule ? p.beta[idx] : 0.f;   // delta rule off: erase 0, write 1
+                gw[h] = p.d.delta_rule ? gb[h] : 1.f;
+            }
+        }
+    };
+    ChunkInfo x;
+    chunk_entry(p, x, blockIdx.x);
+    if (threadIdx.x == 0) issue_loads(x);
+    if (warp == 0) fetch_gates(x);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-        ChunkInfo x;
-        chunk_entry(p, x, item);
-        if (threadIdx.x == 0) {
-            bulk_wait_read<0>();   // the previous trip's stores have read their tiles
-            mbar_expect_tx(&bar_in, 32768);
-            for (int cb = 0; cb < 2; ++cb) {
-                tma_load_2d(sm + KV + cb * 16384, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in);
-                tma_load_2d(sm + KV + cb * 16384 + 8192, &P.tm_v, x.hd * D + cb * 64, x.tok0, &bar_in);
-            }
-            pending = true;
-        }
-        if (warp == 0) {   // gate arrays of the chunk: lane l owns tokens l and l + 32
-            float gg[2] = {0.f, 0.f}, gb[2] = {0.f, 0.f}, gw[2] = {0.f, 0.f};   // log decay, erase gate, write gate
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int i = lane + 32 * h;
-                if (i < x.len) {
-                    const size_t idx = (size_t)(x.tok0 + i) * H + x.hd;
-                    gg[h] = p.g[idx];
-                    gb[h] = p.d.delta_rule ? p.beta[idx] : 0.f;   // delta rule off: erase 0, write 1
-                    gw[h] = p.d.delta_rule ? gb[h] : 1.f;
-                }
-            }
+        const bool has_next = item + (int)gridDim.x < n_items;
+        ChunkInfo xn = x;
+        if (has_next) chunk_entry(p, xn, item + gridDim.x);
+        if (warp == 0) {   // gate arrays of the chunk from the values fetched a trip ahead
             float a = gg[0], b = gg[1];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -126,7 +136,9 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
             mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + KV, 128, 0), op_k_major(sm + KV, 128, 0), false);
             mma_commit(&bar_mma);
         }
+        if (threadIdx.x == 0) bulk_wait_read<0>();   // the previous trip's stores have read their tiles (rewritten from here on)
         GDN_WAIT_MMA(22)
+        __syncthreads();
         if (ok && q4 < 2) {   // A_ij = b_i (k_i . k_j) exp(gam_i - gam_j), j < i (mask before exponentiating)
             const int i = q4 * 32 + lane, j0 = grp * 32;
 #pragma unroll 1
@@ -189,6 +201,10 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(23)
+        if (ok && has_next) {   // K, V have been read for the last time
+            if (threadIdx.x == 0) issue_loads(xn);
+            if (warp == 0) fetch_gates(xn);
+        }
         if (ok) {
             const int f = q4 * 32 + lane, i0 = grp * 32;
 #pragma unroll 1
@@ -213,6 +229,7 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
             bulk_commit();
         }
         if (!ok) break;
+        x = xn;
     }
     if (threadIdx.x == 0) {
         bulk_wait_read<0>();
@@ -227,12 +244,13 @@ __global__ void __launch_bounds__(split::kT, 2) tc_factors_kernel(const __grid_c
 // tc_eprep
 // ------------------------------------------------------------------------------------------------
 namespace eprep {
-constexpr uint32_t QK = 0;                  // [Q rows 0..63 ; K rows 64..127] x 128; finally the staged E image   32 KB
+constexpr uint32_t QK = 0;                  // [Q rows 0..63 ; K rows 64..127] x 128                            32 KB
 constexpr uint32_t DOT = 32768;             // dO [64][128]                                    16 KB
 constexpr uint32_t WT = DOT + 16384;        // W^T [128][64] (image from the workspace)         16 KB
 constexpr uint32_t PT = WT + 16384;         // P = tril(Q K^T . D)                              8 KB
-constexpr uint32_t RT = PT + 8192;          // R = Diag(Gam) dO [64][128]                       16 KB
-constexpr uint32_t PDOT = RT + 16384;       // (P^T dO)^T [128][64]                             16 KB
+constexpr uint32_t RT = PT + 8192;          // R = Diag(Gam) dO [64][128]                       16 KB  (these two: finally
+constexpr uint32_t PDOT = RT + 16384;       // (P^T dO)^T [128][64]                             16 KB   the staged E image)
+static_assert(RT % 1024 == 0 && PDOT == RT + 16384, "the E image [128][128] is two column blocks of 16 KB");
 constexpr uint32_t SMEM_BYTES = PDOT + 16384 + 1024 /* alignment slack */;
 constexpr uint32_t C_S1 = 0, C_PDO = 64, C_E = 128;   // TMEM columns (256 allocated)
 static_assert(2 * (SMEM_BYTES + 4096) <= 228 * 1024, "two CTAs per SM");
@@ -263,25 +281,34 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
     const float sc = p.d.scale;
     bool ok = true, pending = false;
     uint32_t mma_phase = 0, in_phase = 0;
+    // Q, K, dO and W of a trip are dead once its last product is done: the next trip's are loaded right then, under the
+    // readout of E and its store (E is staged over R and (P^T dO)^T, which are dead by then too, not over an input).
+    auto issue_loads = [&](const ChunkInfo& c) {   // thread 0
+        mbar_expect_tx(&bar_in, 65536);
+        for (int cb = 0; cb < 2; ++cb) {
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, c.hd * D + cb * 64, c.tok0, &bar_in);
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, c.hd * D + cb * 64, c.tok0, &bar_in);
+            tma_load_2d(sm + DOT + cb * 8192, &P.tm_do, c.hd * D + cb * 64, c.tok0, &bar_in);
+        }
+        bulk_load(sm + WT, p.ws + p.L.W + (size_t)c.ch * 16384, 16384, &bar_in);
+        pending = true;
+    };
+    float gnext = 0.f;   // threads 0..63: cumulative decay of the next trip's chunk, fetched a trip ahead
+    auto fetch_gamma = [&](const ChunkInfo& c) {
+        if (threadIdx.x < kC) gnext = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)c.ch * kC + threadIdx.x];
+    };
+    ChunkInfo x;
+    chunk_entry(p, x, blockIdx.x);
+    if (threadIdx.x == 0) issue_loads(x);
+    fetch_gamma(x);
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-        ChunkInfo x;
-        chunk_entry(p, x, item);
-        if (threadIdx.x == 0) {
-            bulk_wait_read<0>();   // the previous trip's stores have read the staged E image and P
-            mbar_expect_tx(&bar_in, 65536);
-            for (int cb = 0; cb < 2; ++cb) {
-                tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_in);
-                tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in);
-                tma_load_2d(sm + DOT + cb * 8192, &P.tm_do, x.hd * D + cb * 64, x.tok0, &bar_in);
-            }
-            bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in);
-            pending = true;
-        }
+        const bool has_next = item + (int)gridDim.x < n_items;
+        ChunkInfo xn = x;
+        if (has_next) chunk_entry(p, xn, item + gridDim.x);
         if (threadIdx.x < kC) {   // chunk-local cumulative decay, left in the workspace by the factor stage
-            const float gc = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + threadIdx.x];
-            gl[threadIdx.x] = gc * kLog2e;
-            Gam[threadIdx.x] = expf(gc);
+            gl[threadIdx.x] = gnext * kLog2e;
+            Gam[threadIdx.x] = expf(gnext);
         }
         if (ok) {
             ok = mbar_wait(&bar_in, in_phase);
@@ -301,7 +328,10 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
             mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
             mma_commit(&bar_mma);
         }
-        // R = Diag(Gam) dO while the product runs: four 16-byte pieces per thread
+        if (threadIdx.x == 0) bulk_wait_read<0>();   // the previous trip's stores have read P and the staged E image
+        GDN_WAIT_MMA(25)
+        __syncthreads();
+        // R = Diag(Gam) dO: four 16-byte pieces per thread
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
             const int i = (threadIdx.x >> 4) + 16 * it;
@@ -312,7 +342,6 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
             for (int k = 0; k < 8; ++k) v[k] *= G;
             chunk_store(sm + RT, 64, i, threadIdx.x & 15, v);
         }
-        GDN_WAIT_MMA(25)
         if (ok && q4 < 2) {   // P_ij = (q_i . k_j) exp(gam_i - gam_j), j <= i (mask before exponentiating)
             const int i = q4 * 32 + lane, j0 = grp * 32;
 #pragma unroll 1
@@ -359,7 +388,11 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(27)
-        if (ok) {   // E -> bf16 tile image over Q, K, which no product reads any more
+        if (ok && has_next) {   // every input tile has been read for the last time
+            if (threadIdx.x == 0) issue_loads(xn);
+            fetch_gamma(xn);
+        }
+        if (ok) {   // E -> bf16 tile image over R and (P^T dO)^T, which no product reads any more
             const int r = q4 * 32 + lane, c0 = grp * 64;
 #pragma unroll 1
             for (int part = 0; part < 8; ++part) {
@@ -369,7 +402,7 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
                 tmem_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 8; ++k) v[k] *= sc;
-                chunk_store(sm + QK, 128, r, cb >> 3, v);
+                chunk_store(sm + RT, 128, r, cb >> 3, v);
             }
         }
         tc_fence_before();
@@ -377,10 +410,11 @@ __global__ void __launch_bounds__(split::kT, 2) tc_eprep_kernel(const __grid_con
         __syncthreads();
         if (ok && threadIdx.x == 0) {
             bulk_store(p.ws + p.L.Pm + (size_t)x.ch * 8192, sm + PT, 8192);
-            bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + QK, 32768);
+            bulk_store(p.ws + p.L.E + (size_t)x.ch * 32768, sm + RT, 32768);
             bulk_commit();
         }
         if (!ok) break;
+        x = xn;
     }
     if (threadIdx.x == 0) {
         bulk_wait_read<0>();
