@@ -328,6 +328,20 @@ def time_other_configs(args, peaks, barrier, stream, dev):
                         "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()}}
         del buf, wl
         torch.cuda.empty_cache()
+    # the entry points with per-channel gates (FFMA kernels): KDA gate setting, a quarter of the headline's heads
+    wl = synth.make_channelwise("channelwise_kda_bf16_B4_T2048_H4_d128", member="kda", dtype="bf16", B=4, T=2048, H=4,
+                                d_k=128, d_v=128, seed=7, states=True)
+    buf = runner.to_device_channelwise(wl, dev)
+    for _ in range(2):
+        runner.run_bwd_channelwise(buf)
+    ms = time_steps(lambda: runner.run_bwd_channelwise(buf), 3, barrier, stream) / 3
+    st = binding.gdn_last_device_status(buf.workspace)
+    if st != binding.GDN_OK:
+        raise binding.GdnError(st, wl.name)
+    out[wl.name] = {"ms_per_step": ms, "tokens_per_s": wl.tokens / (ms * 1e-3), "steps": 3, "tokens": wl.tokens,
+                    "kernel_path": "simt_channelwise", "entry_point": "gdn_bwd_channelwise"}
+    del buf, wl
+    torch.cuda.empty_cache()
     return out
 
 

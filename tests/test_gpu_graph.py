@@ -14,6 +14,8 @@ CASES = {
     "tcgen05_scalar_gate_d64": dict(dtype="bf16", lengths=[200, 64, 130], H=2, d_k=64, d_v=64, delta_rule=0,
                                     g_scale=0.05, states=True, seed=32),
     "ffma_f32": dict(dtype="f32", B=2, T=160, H=2, d_k=64, d_v=64, states=True, seed=33),
+    "tcgen05_padded_dk128_dv64": dict(dtype="bf16", lengths=[200, 64, 130], H=2, d_k=128, d_v=64, states=True, seed=34),
+    "tcgen05_d128_low_rank": dict(dtype="bf16", lengths=[70, 130, 64, 1, 100], H=8, d_k=128, d_v=128, states=True, seed=35),
 }
 
 
@@ -72,3 +74,24 @@ def test_captured_forward_then_backward_on_its_workspace():
         assert torch.equal(got[name].view(torch.uint8), ref.view(torch.uint8)), name
     assert binding.gdn_last_device_status(buf.workspace) == binding.GDN_OK
     assert np.isfinite(got["o"].float().cpu().numpy()).all()
+
+
+def test_captured_channelwise_backward_replays_bit_exact():
+    wl = synth.make_channelwise("graph_channelwise", member="kda", dtype="bf16", lengths=[100, 64, 30], H=2, d_k=64, d_v=128,
+                                states=True, seed=36)
+    buf = runner.to_device_channelwise(wl)
+    runner.run_bwd_channelwise(buf)
+    eager = _snapshot(buf)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    _clear(buf)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        runner.run_bwd_channelwise(buf)
+    for _ in range(2):
+        _clear(buf)
+        graph.replay()
+        got = _snapshot(buf)
+        for name, ref in eager.items():
+            assert torch.equal(got[name].view(torch.uint8), ref.view(torch.uint8)), name
+    assert binding.gdn_last_device_status(buf.workspace) == binding.GDN_OK
