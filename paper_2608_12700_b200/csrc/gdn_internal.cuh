@@ -39,6 +39,9 @@ struct WsLayout {
     size_t E;              // [CH, d_k, d_v]           scale (Gam Q - P W)^T dO
     size_t dhn;            // [CH, d_k, d_v]           gradient w.r.t. the state leaving the chunk
     size_t Pm;             // [CH, 64, 64]             P = tril(Q K^T . D) (tcgen05 d = 128 family: made once, by tc_prep)
+    size_t img_W, img_U, img_K, img_E;   // channel-wise path with tensor-core carries: bf16 tile images of W^T, U~^T, the
+                                         // scaled keys Kb (16 KB per chunk-head each) and E (32 KB); else unused
+    int tc_scans;                        // ... and hc, dhn are bf16 tile images (32 KB per chunk-head) instead of fp32
     size_t scratch;        // kernel-private staging, per chunk-head
     size_t scratch_per_ch; // bytes of scratch per chunk-head
     size_t total;
@@ -78,6 +81,7 @@ inline WsLayout make_layout(const gdn_desc& d, size_t elem, size_t elem_add, siz
 }
 
 // Layout of the channel-wise FFMA family: everything fp32; gamma is per channel ([CH, 64, d_k]), no chunk operator.
+inline bool vec_tc_scans(const gdn_desc& d) { return d.dtype == GDN_BF16 && d.d_k == 128 && d.d_v == 128; }
 inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
     WsLayout L{};
     const size_t Ttot = (size_t)d.B * (size_t)d.T;
@@ -85,6 +89,7 @@ inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
     const size_t CH = (size_t)L.max_chunks * d.H;
     size_t o = sizeof(WsHeader);
     auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    L.tc_scans = vec_tc_scans(d) ? 1 : 0;
     L.seq_first = take(4 * ((size_t)d.N + 1));
     L.chunk_seq = take(4 * (size_t)L.max_chunks);
     L.chunk_tok0 = take(4 * (size_t)L.max_chunks);
@@ -93,12 +98,16 @@ inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
     L.Tm = take(4 * CH * kC * kC);
     L.W = take(4 * CH * kC * d.d_k);
     L.Ut = take(4 * CH * kC * d.d_v);
+    L.Pm = take(4 * CH * kC * kC);
     L.Nm = L.Bf = o;
-    L.hc = take(4 * CH * d.d_k * d.d_v);
+    L.img_W = take(L.tc_scans ? CH * 16384 : 0);
+    L.img_U = take(L.tc_scans ? CH * 16384 : 0);
+    L.img_K = take(L.tc_scans ? CH * 16384 : 0);
+    L.hc = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
     L.fwd_end = o;
     L.E = take(4 * CH * d.d_k * d.d_v);
-    L.dhn = take(4 * CH * d.d_k * d.d_v);
-    L.Pm = take(4 * CH * kC * kC);
+    L.img_E = take(L.tc_scans ? CH * 32768 : 0);
+    L.dhn = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
     L.scratch_per_ch = scratch_per_ch;
     L.scratch = take(scratch_per_ch * CH);
     L.total = o;
@@ -177,6 +186,7 @@ bool tc_supported(const gdn_desc& d);
 // Form of the carries for a descriptor: one rule for the forward, the backward and a backward that consumes a workspace
 // fresh from the forward, so that the layout of a workspace does not depend on which call sized it.
 bool tc_carries_lowrank(const gdn_desc& d);
+cudaError_t tc_launch_scan_channelwise(const Problem& p, int dirs, cudaStream_t st);   // carries of the channel-wise path
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 

@@ -15,7 +15,11 @@
 //            gradients per channel, and dg by a reverse cumulative sum inside the chunk
 // One CTA handles one (chunk, head) in the parallel stages and one (sequence, head) chain in the scans.  Every
 // reduction has a fixed order: results are bit-identical from run to run.
+// With bf16 I/O at d_k = d_v = 128 the two carries (the reverse one is the paper's K#1) run on the tensor cores instead
+// (tc_scan_cw in gdn_tc.cu): vprep and veprep then also leave bf16 tile images of W^T, U~^T, the scaled keys Kb and E in
+// the workspace, and the per-chunk states come back as bf16 tile images.
 #include "simt_common.cuh"
+#include "tc_ptx.cuh"
 
 namespace gdn {
 namespace {
@@ -37,6 +41,14 @@ __device__ __forceinline__ void mac_decay(float (&acc)[4][4], int i0, int j0, in
             for (int y = 0; y < 4; ++y)
                 if (j0 + y <= i0 + x - strict) acc[x][y] = fmaf(a[x] * b[y], expf(gi[x] - gj[y]), acc[x][y]);
     }
+}
+
+// Element (r, c) of a bf16 tile image with R rows (the operand format of the tensor-core kernels).
+__device__ __forceinline__ void img_put(char* img, int R, int r, int c, float x) {
+    *reinterpret_cast<__nv_bfloat16*>(img + tc::tile_off(R, r, c)) = __float2bfloat16_rn(x);
+}
+__device__ __forceinline__ float img_get(const char* img, int R, int r, int c) {
+    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(img + tc::tile_off(R, r, c)));
 }
 
 // Chunk-local cumulative log decay per channel into shared memory (pitch DK + 1); rows beyond the sequence repeat the
@@ -84,6 +96,7 @@ __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
     float* wsW = reinterpret_cast<float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
     float* wsU = reinterpret_cast<float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
 
+    const bool imgs = p.L.tc_scans != 0;
     cumulate_gates<DK>(p, x, gam);
     __syncthreads();
     for (int t = threadIdx.x; t < kC * DK; t += blockDim.x) wsG[t] = gam[(t / DK) * (DK + 1) + t % DK];
@@ -115,13 +128,26 @@ __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
         float acc[4][4] = {};
         mac(acc, i0, j0, kC, [&](int i, int m) { return Ti[i][m]; },
             [&](int m, int j) { return expf(gam[m * (DK + 1) + j]) * Bf(m, j) * Kf(m, j); });
-        for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) wsW[(i0 + a) * DK + j0 + b] = acc[a][b];
+        for (int a = 0; a < 4; ++a)
+            for (int b = 0; b < 4; ++b) {
+                wsW[(i0 + a) * DK + j0 + b] = acc[a][b];
+                if (imgs) img_put(p.ws + p.L.img_W + (size_t)x.ch * 16384, 128, j0 + b, i0 + a, acc[a][b]);   // W^T [d_k][tokens]
+            }
     });
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
         mac(acc, i0, j0, kC, [&](int i, int m) { return Ti[i][m]; }, [&](int m, int j) { return Wf(m, j) * Vf(m, j); });
-        for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) wsU[(i0 + a) * DV + j0 + b] = acc[a][b];
+        for (int a = 0; a < 4; ++a)
+            for (int b = 0; b < 4; ++b) {
+                wsU[(i0 + a) * DV + j0 + b] = acc[a][b];
+                if (imgs) img_put(p.ws + p.L.img_U + (size_t)x.ch * 16384, 128, j0 + b, i0 + a, acc[a][b]);   // U~^T [d_v][tokens]
+            }
     });
+    if (imgs)   // Kb_j = exp(gam_e - gam_j) . k_j, [tokens][d_k]; rows beyond the sequence are zero
+        for (int t = threadIdx.x; t < kC * DK; t += blockDim.x) {
+            const int i = t / DK, r = t % DK;
+            img_put(p.ws + p.L.img_K + (size_t)x.ch * 16384, 64, i, r, expf(gam[(kC - 1) * (DK + 1) + r] - gam[i * (DK + 1) + r]) * Kf(i, r));
+        }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -154,7 +180,11 @@ __global__ void __launch_bounds__(kThreads) veprep_kernel(Problem p) {
     tiles(DK, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
         mac(acc, i0, j0, kC, [&](int i, int m) { return X[m * DK + i]; }, Of);
-        for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) wsE[(i0 + a) * DV + j0 + b] = sc * acc[a][b];
+        for (int a = 0; a < 4; ++a)
+            for (int b = 0; b < 4; ++b) {
+                wsE[(i0 + a) * DV + j0 + b] = sc * acc[a][b];
+                if (p.L.tc_scans) img_put(p.ws + p.L.img_E + (size_t)x.ch * 32768, 128, i0 + a, j0 + b, sc * acc[a][b]);
+            }
     });
 }
 
@@ -238,18 +268,23 @@ __global__ void __launch_bounds__(kThreads) vout_kernel(Problem p) {
     const float* wsP = reinterpret_cast<const float*>(p.ws + p.L.Pm) + (size_t)x.ch * kC * kC;
     const float* wsW = reinterpret_cast<const float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
     const float* wsU = reinterpret_cast<const float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
-    const float* h = reinterpret_cast<const float*>(p.ws + p.L.hc) + (size_t)x.ch * DK * DV;
+    // the state entering the chunk: fp32 row-major, or the bf16 tile image the tensor-core carries leave
+    const char* hraw = p.ws + p.L.hc;
+    const bool img = p.L.tc_scans != 0;
+    auto Hf = [&](int m, int j) -> float {
+        return img ? img_get(hraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(hraw)[(size_t)x.ch * DK * DV + m * DV + j];
+    };
     float* U = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);  // [64, DV]
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
-        mac(acc, i0, j0, DK, [&](int i, int m) { return wsW[i * DK + m]; }, [&](int m, int j) { return h[m * DV + j]; });
+        mac(acc, i0, j0, DK, [&](int i, int m) { return wsW[i * DK + m]; }, Hf);
         for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) U[(i0 + a) * DV + j0 + b] = wsU[(i0 + a) * DV + j0 + b] - acc[a][b];
     });
     __syncthreads();
     const float sc = p.d.scale;
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
-        mac(acc, i0, j0, DK, [&](int i, int m) { return expf(wsG[i * DK + m]) * Qf(i, m); }, [&](int m, int j) { return h[m * DV + j]; });
+        mac(acc, i0, j0, DK, [&](int i, int m) { return expf(wsG[i * DK + m]) * Qf(i, m); }, Hf);
         mac(acc, i0, j0, kC, [&](int i, int m) { return wsP[i * kC + m]; }, [&](int m, int j) { return U[m * DV + j]; });
         for (int a = 0; a < 4; ++a)
             for (int b = 0; b < 4; ++b)
@@ -289,8 +324,16 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     const float* Pm = reinterpret_cast<const float*>(p.ws + p.L.Pm) + (size_t)x.ch * kC * kC;
     const float* W = reinterpret_cast<const float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
     const float* Ut = reinterpret_cast<const float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
-    const float* h = reinterpret_cast<const float*>(p.ws + p.L.hc) + (size_t)x.ch * DK * DV;
-    const float* dhn = reinterpret_cast<const float*>(p.ws + p.L.dhn) + (size_t)x.ch * DK * DV;
+    // per-chunk states: fp32 row-major, or the bf16 tile images the tensor-core carries leave
+    const bool img = p.L.tc_scans != 0;
+    const char* hraw = p.ws + p.L.hc;
+    const char* dhraw = p.ws + p.L.dhn;
+    auto Hs = [&](int m, int j) -> float {   // h[m][j]
+        return img ? img_get(hraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(hraw)[(size_t)x.ch * DK * DV + m * DV + j];
+    };
+    auto DHs = [&](int m, int j) -> float {  // dh'[m][j]
+        return img ? img_get(dhraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(dhraw)[(size_t)x.ch * DK * DV + m * DV + j];
+    };
     float* scr = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);
     float* U = scr;                    // [64, DV]
     float* dU = U + kC * DV;           // [64, DV]
@@ -306,9 +349,9 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     // (1) U = Ut - W h ;  dU = scale P^T dO + Kb dh'
     tiles(kC, DV, [&](int i0, int j0) {
         float a0[4][4] = {}, a1[4][4] = {}, a2[4][4] = {};
-        mac(a0, i0, j0, DK, [&](int i, int m) { return W[i * DK + m]; }, [&](int m, int j) { return h[m * DV + j]; });
+        mac(a0, i0, j0, DK, [&](int i, int m) { return W[i * DK + m]; }, Hs);
         mac(a1, i0, j0, DK, [&](int i, int m) { return expf(wsG[(kC - 1) * DK + m] - wsG[i * DK + m]) * Kf(i, m); },
-            [&](int m, int j) { return dhn[m * DV + j]; });
+            DHs);
         mac(a2, i0, j0, kC, [&](int i, int m) { return Pm[m * kC + i]; }, Of);
         for (int a = 0; a < 4; ++a)
             for (int b = 0; b < 4; ++b) {
@@ -327,9 +370,9 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     });
     tiles(kC, DK, [&](int i0, int j0) {
         float a1[4][4] = {}, a2[4][4] = {}, a3[4][4] = {};
-        mac(a1, i0, j0, DV, Of, [&](int m, int j) { return h[j * DV + m]; });
-        mac(a2, i0, j0, DV, [&](int i, int m) { return dU[i * DV + m]; }, [&](int m, int j) { return h[j * DV + m]; });
-        mac(a3, i0, j0, DV, [&](int i, int m) { return U[i * DV + m]; }, [&](int m, int j) { return dhn[j * DV + m]; });
+        mac(a1, i0, j0, DV, Of, [&](int m, int j) { return Hs(j, m); });
+        mac(a2, i0, j0, DV, [&](int i, int m) { return dU[i * DV + m]; }, [&](int m, int j) { return Hs(j, m); });
+        mac(a3, i0, j0, DV, [&](int i, int m) { return U[i * DV + m]; }, [&](int m, int j) { return DHs(j, m); });
         for (int a = 0; a < 4; ++a)
             for (int b = 0; b < 4; ++b) {
                 const int t = (i0 + a) * DK + j0 + b;
@@ -405,7 +448,7 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
         float extra = 0.f, hh = 0.f;
         const float ge = G(kC - 1, r);
         for (int j = 0; j < kC; ++j) extra = fmaf(Kf(j, r) * expf(ge - G(j, r)), UdH[j * DK + r], extra);
-        for (int c = 0; c < DV; ++c) hh = fmaf(dhn[r * DV + c], h[r * DV + c], hh);
+        for (int c = 0; c < DV; ++c) hh = fmaf(DHs(r, c), Hs(r, c), hh);
         float run = extra + expf(ge) * hh;
         for (int i = kC - 1; i >= 0; --i) {
             run += dgam[i * DK + r];
@@ -415,17 +458,23 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
 }
 
 template <typename IO, int DK, int DV>
-cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st) {
+cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st, bool with_scan = true) {
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
     launch_table(p, st);
     const size_t smp = sizeof(float) * (kC * (DK + 1) + 2 * kC * (kC + 1));
     cudaError_t e = cudaFuncSetAttribute(vprep_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smp);
     if (e != cudaSuccess) return e;
     if (CH > 0) { StageScope t(ST_PREP, st); vprep_kernel<IO, DK, DV><<<CH, kThreads, smp, st>>>(p); }
-    const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
-    e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    if (e != cudaSuccess) return e;
-    if (chains > 0) { StageScope t(ST_FSCAN, st); vscan_kernel<IO, DK, DV, false><<<chains, kThreads, sm, st>>>(p); }
+    if (with_scan) {
+        if (p.L.tc_scans) {
+            if (chains > 0 && (e = tc_launch_scan_channelwise(p, 0, st)) != cudaSuccess) return e;
+        } else {
+            const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
+            e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+            if (e != cudaSuccess) return e;
+            if (chains > 0) { StageScope t(ST_FSCAN, st); vscan_kernel<IO, DK, DV, false><<<chains, kThreads, sm, st>>>(p); }
+        }
+    }
     if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
     return cudaGetLastError();
 }
@@ -433,16 +482,21 @@ cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st) {
 template <typename IO, int DK, int DV>
 cudaError_t vlaunch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st) {
     cudaError_t e;
+    const bool tcs = p.L.tc_scans != 0;   // tensor-core carries: both directions in one launch, after E is there
     if (!skip_recompute) {
-        e = vlaunch_fwd_t<IO, DK, DV>(p, st);
+        e = vlaunch_fwd_t<IO, DK, DV>(p, st, /*with_scan=*/!tcs);
         if (e != cudaSuccess) return e;
     }
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
     if (CH > 0) { StageScope t(ST_EPREP, st); veprep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
-    const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
-    e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    if (e != cudaSuccess) return e;
-    if (chains > 0) { StageScope t(ST_RSCAN, st); vscan_kernel<IO, DK, DV, true><<<chains, kThreads, sm, st>>>(p); }
+    if (tcs) {
+        if (chains > 0 && (e = tc_launch_scan_channelwise(p, skip_recompute ? 1 : 2, st)) != cudaSuccess) return e;
+    } else {
+        const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
+        e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+        if (e != cudaSuccess) return e;
+        if (chains > 0) { StageScope t(ST_RSCAN, st); vscan_kernel<IO, DK, DV, true><<<chains, kThreads, sm, st>>>(p); }
+    }
     const size_t smi = sizeof(float) * (kC * (DK + 1) + 2 * kC * (kC + 1));
     e = cudaFuncSetAttribute(vintra_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smi);
     if (e != cudaSuccess) return e;

@@ -797,7 +797,11 @@ static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budge
 }  // namespace scanlr
 
 // One direction of one chain (the direction is a compile-time constant: the two differ in operands and readouts).
-template <bool reverse>
+// CW = carries of the channel-wise path (per-channel gates): the decay of the state is a vector (one factor per state
+// row, i.e. per thread), and the key tile arrives already scaled, Kb_j = exp(gam_e - gam_j) . k_j, as a tile image from the
+// workspace together with images of W^T, U~^T and E (written by the channel-wise preparation kernels), so the readout of the
+// first product applies no per-token factor.
+template <bool reverse, bool CW>
 __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, float* ge, float (*ee2)[kC], uint64_t* bar_full,
                                               uint64_t& bar_mma, uint32_t& tmem_slot) {
     using namespace scanlr;
@@ -827,8 +831,8 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
     const uint32_t tmem = tmem_slot;
 
     auto chunk_of = [&](int s) { return reverse ? (c1 - 1 - s) : (c0 + s); };
-    const char* w_base = p.ws + p.L.W;
-    const char* x_base = p.ws + (reverse ? p.L.E : p.L.Ut);
+    const char* w_base = p.ws + (CW ? p.L.img_W : p.L.W);
+    const char* x_base = p.ws + (reverse ? (CW ? p.L.img_E : p.L.E) : (CW ? p.L.img_U : p.L.Ut));
     const uint32_t x_chunk = reverse ? 32768u : 16384u;
     char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
@@ -839,19 +843,24 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         unsigned char* slot = sm + stage * STAGE_BYTES;
         mbar_expect_tx(&bar_full[stage], 32768 + x_chunk);
         bulk_load(slot + WT, w_base + ch * 16384, 16384, &bar_full[stage]);
-        tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
-        tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
+        if constexpr (CW) {
+            bulk_load(slot + KT, p.ws + p.L.img_K + ch * 16384, 16384, &bar_full[stage]);
+        } else {
+            tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
+            tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
+        }
         bulk_load(slot + XT, x_base + ch * x_chunk, x_chunk, &bar_full[stage]);
     };
     if (threadIdx.x == 32) {
         for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
     }
-    for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
-        ge[s] = expf(gamma[((size_t)chunk_of(s) * H + hd) * kC + kC - 1]);
+    if constexpr (!CW)
+        for (int s = threadIdx.x; s < nsteps && s < GE_CAP; s += blockDim.x)
+            ge[s] = expf(gamma[((size_t)chunk_of(s) * H + hd) * kC + kC - 1]);
     // e_j of the first step; the cumulative decays of the second are fetched now
     auto gate_row = [&](int s) { return gamma + ((size_t)chunk_of(s) * H + hd) * kC; };
     float gnext = 0.f, gend_next = 0.f;
-    if (threadIdx.x < kC && nsteps > 0) {
+    if (!CW && threadIdx.x < kC && nsteps > 0) {
         ee2[0][threadIdx.x] = expf(gate_row(0)[kC - 1] - gate_row(0)[threadIdx.x]);
         if (nsteps > 1) { gnext = gate_row(1)[threadIdx.x]; gend_next = gate_row(1)[kC - 1]; }
     }
@@ -875,11 +884,12 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         const size_t ch = (size_t)c * H + hd;
         unsigned char* ring = sm + stage * STAGE_BYTES;
         const float* ee = ee2[s & 1];
-        const float Ge = s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]);
+        // decay of the state over the chunk: a scalar, or (channel-wise) the factor of this thread's state row
+        const float Ge = CW ? expf(gamma[(ch * kC + kC - 1) * D + r]) : (s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]));
         // state -> bf16: operand of the first product, and the per-chunk state the gradient stage reads
 #pragma unroll
         for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
-        if (len < kC) {   // ragged tail: the K rows beyond the sequence belong to somebody else
+        if (!CW && len < kC) {   // ragged tail: the K rows beyond the sequence belong to somebody else
             ok = mbar_wait_inline(&bar_full[stage], (s / STAGES) & 1);
             if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 12); break; }
             zero_tail_rows(ring + KT, 64, 0, len, kThreads);
@@ -917,7 +927,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
             ld8s(ee + tk0 + 8 * k, e8);
             tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 8; ++j) d1[j] = e8[j] * (reverse ? d1[j] : (u[j] - d1[j]));
+            for (int j = 0; j < 8; ++j) d1[j] = (CW ? 1.f : e8[j]) * (reverse ? d1[j] : (u[j] - d1[j]));
             chunk_store(sm + GT, 128, r, (tk0 >> 3) + k, d1);
         }
         tc_fence_before();
@@ -929,7 +939,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
             else mma_tile<128, 128, 64>(tmem + C_D2, op_mn_major(ring + KT, 64), op_k_major(sm + GT, 128), false);
             mma_commit(&bar_mma);
         }
-        if (threadIdx.x < kC && s + 1 < nsteps) {   // e_j of the next step, while the product runs
+        if (!CW && threadIdx.x < kC && s + 1 < nsteps) {   // e_j of the next step, while the product runs
             ee2[(s + 1) & 1][threadIdx.x] = expf(gend_next - gnext);
             if (s + 2 < nsteps) { gnext = gate_row(s + 2)[threadIdx.x]; gend_next = gate_row(s + 2)[kC - 1]; }
         }
@@ -970,8 +980,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_co
     if (reinterpret_cast<const WsHeader*>(P.p.ws)->status != GDN_OK) return;
     const int rev = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
     const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
-    if (rev) scan_lr_chain<true>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
-    else scan_lr_chain<false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
+    if (rev) scan_lr_chain<true, false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
+    else scan_lr_chain<false, false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
+}
+
+// The carries of the channel-wise path (per-channel gates, d_k = d_v = 128, bf16 I/O) on the same machinery.
+__global__ void __launch_bounds__(kThreads, 1) tc_scan_cw_kernel(const __grid_constant__ TcParams P) {
+    using namespace scanlr;
+    __shared__ __align__(16) float ee2[2][kC];   // (unused: the key tile arrives scaled)
+    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ uint32_t tmem_slot;
+    const int bid = (int)blockIdx.x;
+    if (reinterpret_cast<const WsHeader*>(P.p.ws)->status != GDN_OK) return;
+    const int rev = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
+    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
+    if (rev) scan_lr_chain<true, true>(P, chain, nullptr, ee2, bar_full, bar_mma, tmem_slot);
+    else scan_lr_chain<false, true>(P, chain, nullptr, ee2, bar_full, bar_mma, tmem_slot);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1759,6 +1783,18 @@ static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done;
     return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, kThreads, P, st);
+}
+
+// Carries of the channel-wise path: dirs = 0 forward, 1 reverse, 2 both in one launch.  Needs the tile images the
+// channel-wise preparation kernels leave in the workspace; no tensor map is used.
+cudaError_t tc_launch_scan_channelwise(const Problem& p, int dirs, cudaStream_t st) {
+    static SmemLimitOnce done;
+    TcParams P{};
+    P.p = p;
+    P.scan_dirs = dirs;
+    P.lowrank = 1;
+    const int ctas = p.d.N * p.d.H * (dirs == 2 ? 2 : 1);
+    return launch_chunk_kernel(tc_scan_cw_kernel, done, scanlr::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
 }
 
 // A call with no tokens still owes the pass-through of the states.

@@ -39,6 +39,27 @@ def test_family_members_ragged_with_states(dtype, member):
     assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))   # empty sequence: pass-through
 
 
+@pytest.mark.parametrize("member", ["gdn", "kda", "gla"])
+def test_tensor_core_carries_bf16_d128(member):
+    """bf16 I/O at d_k = d_v = 128: the forward and the reverse carry (K#1) run on the tcgen05 kernels, fed with tile
+    images by the preparation kernels; ragged, with states and an empty sequence; forward outputs and the
+    save-forward arm as well."""
+    wl = synth.make_channelwise(f"cw_tc_{member}", member=member, dtype="bf16", lengths=[65, 128, 0, 37, 300], H=2,
+                                d_k=128, d_v=128, states=True, seed=68, scale=0.5)
+    got = runner.backward_channelwise(wl)
+    errs, ref = check(wl, got)
+    print(wl.name, errs)
+    assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))
+    buf = runner.to_device_channelwise(wl, want_o=True)
+    runner.run_fwd_channelwise(buf)
+    f = runner.fetch(buf)
+    assert rel(f["o"], ref["o"]) < TOL["bf16"] and rel(f["hT"], ref["hT"]) < TOL["bf16"]
+    runner.run_bwd_channelwise(buf, fresh=1)
+    fresh = runner.fetch(buf)
+    for n in GRADS:
+        assert np.array_equal(fresh[n], got[n]), n
+
+
 @pytest.mark.parametrize("dk,dv", [(128, 128), (128, 64), (64, 128)])
 def test_shapes(dk, dv):
     wl = synth.make_channelwise(f"cw_shape_{dk}_{dv}", dtype="f32", B=2, T=192, H=2, d_k=dk, d_v=dv, states=True, seed=62)
