@@ -28,6 +28,7 @@ namespace {
 template <int DK, class FA, class FB>
 __device__ __forceinline__ void mac_decay(float (&acc)[4][4], int i0, int j0, int strict, const float* gam, FA fa, FB fb) {
     if (j0 > i0 + 3 - strict) return;
+#pragma unroll 2
     for (int m = 0; m < DK; ++m) {
         float a[4], b[4], gi[4], gj[4];
 #pragma unroll

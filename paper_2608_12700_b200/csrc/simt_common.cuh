@@ -23,6 +23,7 @@ __device__ __forceinline__ void tiles(int M, int N, Body body) {
 // acc[a][b] += sum_m fa(i0 + a, m) * fb(m, j0 + b)
 template <class FA, class FB>
 __device__ __forceinline__ void mac(float (&acc)[4][4], int i0, int j0, int K, FA fa, FB fb) {
+#pragma unroll 4
     for (int m = 0; m < K; ++m) {
         float a[4], b[4];
 #pragma unroll
