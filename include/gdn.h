@@ -55,7 +55,9 @@ typedef enum gdn_status {
     GDN_ERR_BAD_SEQLENS = 5,        /* device-side: cu_seqlens not starting at 0 / decreasing / != T   */
     GDN_ERR_WORKSPACE_TOO_SMALL = 6,
     GDN_ERR_CUDA = 7,               /* a CUDA runtime call or launch failed                            */
-    GDN_ERR_DEVICE_TIMEOUT = 8      /* device-side: a bounded wait gave up                             */
+    GDN_ERR_DEVICE_TIMEOUT = 8,     /* device-side: a bounded wait gave up                             */
+    GDN_ERR_DECAY_RANGE = 9         /* device-side, channel-wise calls on the tensor cores: the cumulative log  */
+                                    /* decay of a chunk leaves [-80, 80] (or is not a number)                   */
 } gdn_status;
 
 typedef enum gdn_dtype { GDN_F32 = 0, GDN_BF16 = 1 } gdn_dtype;
@@ -116,8 +118,12 @@ gdn_status gdn_bwd(const gdn_desc* desc,
  * gdn_fwd_recompute / gdn_bwd; desc->delta_rule is not read (the gates say which family member runs: KDA is
  * b = w = beta broadcast over the channels, GLA is b = 0, w = 1, the full GDN has independent vectors).  All three
  * gate gradients are required outputs.  The workspace has its own size (gdn_workspace_bytes_channelwise) and
- * layout; its status word is read with gdn_last_device_status.  These entry points run on fp32 FFMA kernels
- * for either I/O dtype (bf16 I/O: inputs and dq, dk, dv are bf16, all arithmetic and the gate tensors are fp32). */
+ * layout; its status word is read with gdn_last_device_status.  With bf16 I/O at d_k = d_v = 128 these calls run on
+ * the tensor cores (tcgen05): keys and queries are scaled by the chunk-local cumulative decay element by element, which
+ * requires |sum of g over any prefix of a 64-token chunk| <= 80 per channel; a call whose gates leave that range
+ * reports GDN_ERR_DECAY_RANGE through the status word and writes no output (the fp32 dtype has no such limit).  Every
+ * other shape and dtype runs on fp32 FFMA kernels (bf16 I/O: inputs and dq, dk, dv are bf16, all arithmetic and the
+ * gate tensors are fp32). */
 gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
 gdn_status gdn_fwd_recompute_channelwise(const gdn_desc* desc,
                                          const void* q, const void* k, const void* v,

@@ -18,7 +18,7 @@ GDN_OK = 0
 GDN_F32, GDN_BF16 = 0, 1
 STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "GDN_ERR_UNSUPPORTED_SHAPE",
                 4: "GDN_ERR_MISALIGNED", 5: "GDN_ERR_BAD_SEQLENS", 6: "GDN_ERR_WORKSPACE_TOO_SMALL",
-                7: "GDN_ERR_CUDA", 8: "GDN_ERR_DEVICE_TIMEOUT"}
+                7: "GDN_ERR_CUDA", 8: "GDN_ERR_DEVICE_TIMEOUT", 9: "GDN_ERR_DECAY_RANGE"}
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
            "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",

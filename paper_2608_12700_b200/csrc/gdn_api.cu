@@ -260,7 +260,8 @@ gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream) {
     int32_t word = 0;
     if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return GDN_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return GDN_ERR_CUDA;
-    if (word == GDN_OK || word == GDN_ERR_BAD_SEQLENS || word == GDN_ERR_DEVICE_TIMEOUT) return (gdn_status)word;
+    if (word == GDN_OK || word == GDN_ERR_BAD_SEQLENS || word == GDN_ERR_DEVICE_TIMEOUT || word == GDN_ERR_DECAY_RANGE)
+        return (gdn_status)word;
     return GDN_ERR_CUDA;
 }
 
@@ -275,6 +276,7 @@ const char* gdn_status_string(gdn_status s) {
         case GDN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case GDN_ERR_CUDA: return "a CUDA call failed";
         case GDN_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+        case GDN_ERR_DECAY_RANGE: return "cumulative log decay of a chunk outside [-80, 80] (channel-wise call on the tensor cores)";
     }
     return "unknown status";
 }

@@ -39,9 +39,10 @@ struct WsLayout {
     size_t E;              // [CH, d_k, d_v]           scale (Gam Q - P W)^T dO
     size_t dhn;            // [CH, d_k, d_v]           gradient w.r.t. the state leaving the chunk
     size_t Pm;             // [CH, 64, 64]             P = tril(Q K^T . D) (tcgen05 d = 128 family: made once, by tc_prep)
-    size_t img_W, img_U, img_K, img_E;   // channel-wise path with tensor-core carries: bf16 tile images of W^T, U~^T, the
-                                         // scaled keys Kb (16 KB per chunk-head each) and E (32 KB); else unused
-    int tc_scans;                        // ... and hc, dhn are bf16 tile images (32 KB per chunk-head) instead of fp32
+    size_t img_W, img_U, img_K, img_E;   // channel-wise path on the tensor cores (bf16, d = 128): bf16 tile images of W^T,
+                                         // U~^T, the scaled keys Kb (16 KB per chunk-head each) and E (32 KB); else unused
+    size_t img_QKp, img_Km, img_Vt, img_dO;   // ... of [Q~; K+] (32 KB), K-, V~ and scale dO (16 KB each)
+    int tc_scans;                        // ... and T, P, hc, dhn are bf16 tile images as well (8, 8, 32, 32 KB)
     size_t scratch;        // kernel-private staging, per chunk-head
     size_t scratch_per_ch; // bytes of scratch per chunk-head
     size_t total;
@@ -103,10 +104,14 @@ inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
     L.img_W = take(L.tc_scans ? CH * 16384 : 0);
     L.img_U = take(L.tc_scans ? CH * 16384 : 0);
     L.img_K = take(L.tc_scans ? CH * 16384 : 0);
+    L.img_QKp = take(L.tc_scans ? CH * 32768 : 0);
+    L.img_Km = take(L.tc_scans ? CH * 16384 : 0);
+    L.img_Vt = take(L.tc_scans ? CH * 16384 : 0);
     L.hc = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
     L.fwd_end = o;
     L.E = take(4 * CH * d.d_k * d.d_v);
     L.img_E = take(L.tc_scans ? CH * 32768 : 0);
+    L.img_dO = take(L.tc_scans ? CH * 16384 : 0);
     L.dhn = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
     L.scratch_per_ch = scratch_per_ch;
     L.scratch = take(scratch_per_ch * CH);
@@ -178,6 +183,9 @@ size_t simt_scratch_per_chunkhead(const gdn_desc& d);
 cudaError_t vec_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t vec_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 size_t vec_scratch_per_chunkhead(const gdn_desc& d);
+// ... and its tensor-core route (bf16 I/O, d_k = d_v = 128; gdn_tc_cw.cu): forward (bwd = false) or backward.
+cudaError_t cw_tc_launch(const Problem& p, bool bwd, bool skip_recompute, cudaStream_t st);
+size_t cw_tc_scratch_per_chunkhead();
 
 // tcgen05 family (bf16 I/O, d_k = d_v = 128, delta rule on).
 extern thread_local int g_force_carries;   // form of the inter-chunk carries: 0 = chosen by shape, 1 = operator form, 2 = low-rank

@@ -15,9 +15,8 @@
 //            gradients per channel, and dg by a reverse cumulative sum inside the chunk
 // One CTA handles one (chunk, head) in the parallel stages and one (sequence, head) chain in the scans.  Every
 // reduction has a fixed order: results are bit-identical from run to run.
-// With bf16 I/O at d_k = d_v = 128 the two carries (the reverse one is the paper's K#1) run on the tensor cores instead
-// (tc_scan_cw in gdn_tc.cu): vprep and veprep then also leave bf16 tile images of W^T, U~^T, the scaled keys Kb and E in
-// the workspace, and the per-chunk states come back as bf16 tile images.
+// With bf16 I/O at d_k = d_v = 128 the whole path runs on the tensor cores instead (gdn_tc_cw.cu and tc_scan_cw in
+// gdn_tc.cu); only the optional forward output is formed here, from the bf16 tile images those kernels leave.
 #include "simt_common.cuh"
 #include "tc_ptx.cuh"
 
@@ -266,27 +265,35 @@ __global__ void __launch_bounds__(kThreads) vout_kernel(Problem p) {
     const size_t rk = (size_t)H * DK, rv = (size_t)H * DV;
     auto Qf = [&](int i, int m) -> float { return i < x.len ? ldf(qp + i * rk + m) : 0.f; };
     const float* wsG = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC * DK;
-    const float* wsP = reinterpret_cast<const float*>(p.ws + p.L.Pm) + (size_t)x.ch * kC * kC;
-    const float* wsW = reinterpret_cast<const float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
-    const float* wsU = reinterpret_cast<const float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
-    // the state entering the chunk: fp32 row-major, or the bf16 tile image the tensor-core carries leave
+    const bool img = p.L.tc_scans != 0;   // tensor-core route: the factors and states are bf16 tile images
+    auto Pf = [&](int i, int m) -> float {
+        return img ? img_get(p.ws + p.L.Pm + (size_t)x.ch * 8192, 64, i, m)
+                   : reinterpret_cast<const float*>(p.ws + p.L.Pm)[(size_t)x.ch * kC * kC + i * kC + m];
+    };
+    auto Wm = [&](int i, int m) -> float {   // W[i][m]
+        return img ? img_get(p.ws + p.L.img_W + (size_t)x.ch * 16384, 128, m, i)
+                   : reinterpret_cast<const float*>(p.ws + p.L.W)[(size_t)x.ch * kC * DK + i * DK + m];
+    };
+    auto Um = [&](int i, int j) -> float {   // U~[i][j]
+        return img ? img_get(p.ws + p.L.img_U + (size_t)x.ch * 16384, 128, j, i)
+                   : reinterpret_cast<const float*>(p.ws + p.L.Ut)[(size_t)x.ch * kC * DV + i * DV + j];
+    };
     const char* hraw = p.ws + p.L.hc;
-    const bool img = p.L.tc_scans != 0;
     auto Hf = [&](int m, int j) -> float {
         return img ? img_get(hraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(hraw)[(size_t)x.ch * DK * DV + m * DV + j];
     };
     float* U = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);  // [64, DV]
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
-        mac(acc, i0, j0, DK, [&](int i, int m) { return wsW[i * DK + m]; }, Hf);
-        for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) U[(i0 + a) * DV + j0 + b] = wsU[(i0 + a) * DV + j0 + b] - acc[a][b];
+        mac(acc, i0, j0, DK, Wm, Hf);
+        for (int a = 0; a < 4; ++a) for (int b = 0; b < 4; ++b) U[(i0 + a) * DV + j0 + b] = Um(i0 + a, j0 + b) - acc[a][b];
     });
     __syncthreads();
     const float sc = p.d.scale;
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
         mac(acc, i0, j0, DK, [&](int i, int m) { return expf(wsG[i * DK + m]) * Qf(i, m); }, Hf);
-        mac(acc, i0, j0, kC, [&](int i, int m) { return wsP[i * kC + m]; }, [&](int m, int j) { return U[m * DV + j]; });
+        mac(acc, i0, j0, kC, Pf, [&](int m, int j) { return U[m * DV + j]; });
         for (int a = 0; a < 4; ++a)
             for (int b = 0; b < 4; ++b)
                 if (i0 + a < x.len) stf(op + (i0 + a) * rv + j0 + b, sc * acc[a][b]);
@@ -461,6 +468,12 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st, bool with_scan = true) {
     const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
+    if (p.L.tc_scans) {   // bf16 I/O at d = 128: scaled operand images, tcgen05 preparation and carry
+        cudaError_t e = cw_tc_launch(p, /*bwd=*/false, false, st);
+        if (e != cudaSuccess) return e;
+        if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
+        return cudaGetLastError();
+    }
     launch_table(p, st);
     const size_t smp = sizeof(float) * (kC * (DK + 1) + 2 * kC * (kC + 1));
     cudaError_t e = cudaFuncSetAttribute(vprep_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smp);
@@ -483,7 +496,8 @@ cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st, bool with_scan = tr
 template <typename IO, int DK, int DV>
 cudaError_t vlaunch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st) {
     cudaError_t e;
-    const bool tcs = p.L.tc_scans != 0;   // tensor-core carries: both directions in one launch, after E is there
+    if (p.L.tc_scans) return cw_tc_launch(p, /*bwd=*/true, skip_recompute, st);   // bf16 I/O at d = 128: all on tcgen05
+    const bool tcs = false;
     if (!skip_recompute) {
         e = vlaunch_fwd_t<IO, DK, DV>(p, st, /*with_scan=*/!tcs);
         if (e != cudaSuccess) return e;
