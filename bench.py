@@ -328,18 +328,25 @@ def time_other_configs(args, peaks, barrier, stream, dev):
                         "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()}}
         del buf, wl
         torch.cuda.empty_cache()
-    # the entry points with per-channel gates (FFMA kernels): KDA gate setting, a quarter of the headline's heads
-    wl = synth.make_channelwise("channelwise_kda_bf16_B4_T2048_H4_d128", member="kda", dtype="bf16", B=4, T=2048, H=4,
+    # the entry points with per-channel gates (tensor-core route): KDA gate setting on the shape of the headline
+    wl = synth.make_channelwise("channelwise_kda_bf16_B4_T2048_H16_d128", member="kda", dtype="bf16", B=4, T=2048, H=16,
                                 d_k=128, d_v=128, seed=7, states=True)
     buf = runner.to_device_channelwise(wl, dev)
-    for _ in range(2):
+    for _ in range(3):
         runner.run_bwd_channelwise(buf)
-    ms = time_steps(lambda: runner.run_bwd_channelwise(buf), 3, barrier, stream) / 3
+    ms = time_steps(lambda: runner.run_bwd_channelwise(buf), 10, barrier, stream) / 10
     st = binding.gdn_last_device_status(buf.workspace)
     if st != binding.GDN_OK:
         raise binding.GdnError(st, wl.name)
-    out[wl.name] = {"ms_per_step": ms, "tokens_per_s": wl.tokens / (ms * 1e-3), "steps": 3, "tokens": wl.tokens,
-                    "kernel_path": "simt_channelwise", "entry_point": "gdn_bwd_channelwise"}
+    binding.gdn_stage_timing_enable(1)
+    binding.gdn_stage_timing_read()
+    for _ in range(3):
+        runner.run_bwd_channelwise(buf)
+    torch.cuda.synchronize()
+    stg = {k: round(v[0] / v[1], 5) for k, v in binding.gdn_stage_timing_read().items() if v[1] > 0}
+    binding.gdn_stage_timing_enable(False)
+    out[wl.name] = {"ms_per_step": ms, "tokens_per_s": wl.tokens / (ms * 1e-3), "steps": 10, "tokens": wl.tokens,
+                    "kernel_path": "tcgen05_bf16_channelwise", "entry_point": "gdn_bwd_channelwise", "stage_ms_per_launch": stg}
     del buf, wl
     torch.cuda.empty_cache()
     return out

@@ -137,7 +137,7 @@ struct Problem {
 
 // Launch bookkeeping: every kernel launch goes through stage_begin / stage_end so that launches can be
 // counted and, when enabled, timed per stage with CUDA events on the launching stream.
-enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_SCANS, ST_COUNT };
+enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_SCANS, ST_SCALE, ST_POST, ST_COUNT };
 void stage_begin(Stage s, cudaStream_t st);
 void stage_end(Stage s, cudaStream_t st);
 struct StageScope {

@@ -47,9 +47,9 @@ __device__ __forceinline__ bool chunk_ctx(const Problem& p, ChunkCtx& x) {
     return true;
 }
 
-// Per chunk-head scratch between cw_intra and cw_post (fp32): dQ~, dK+, dK-, U dh''^T [64][128] each, dXv^T [128][64],
+// Per chunk-head scratch between cw_intra and cw_post (fp32): dQ~, dK+, dK-, U dh''^T, dXv [64][128] each,
 // rowdot(dh'', h) [128].
-constexpr size_t S_DQ = 0, S_DKP = 32768, S_DKM = 65536, S_UDH = 98304, S_DXVT = 131072, S_HH = 163840, S_BYTES = 164352;
+constexpr size_t S_DQ = 0, S_DKP = 32768, S_DKM = 65536, S_UDH = 98304, S_DXV = 131072, S_HH = 163840, S_BYTES = 164352;
 
 // ------------------------------------------------------------------------------------------------
 // cw_scale
@@ -522,9 +522,8 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
                 tmem_ld8(tmem + lane_base + C_A + ib, v);
                 tmem_wait_ld();
                 chunk_store(sm + DXVT, 128, f, ib >> 3, v);
-                float* dst = scr + S_DXVT / 4 + f * kC + ib;
-                *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-                *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) scr[S_DXV / 4 + (ib + j) * D + f] = v[j];   // token-major: a warp writes 128 contiguous bytes
             }
 #pragma unroll 1
             for (int part = 0; part < 8; ++part) {   // dXk: operand tile (the accumulator goes on collecting dK+)
@@ -620,37 +619,65 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
     const float* wsG = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC * D;
     const float* scr = reinterpret_cast<const float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);
     const float *dQ = scr + S_DQ / 4, *dKp = scr + S_DKP / 4, *dKm = scr + S_DKM / 4, *udh = scr + S_UDH / 4;
-    const float *dXvT = scr + S_DXVT / 4, *hh = scr + S_HH / 4;
-    for (int t = threadIdx.x; t < kC * D; t += kT) {
-        const int i = t / D, r = t % D;
+    const float *dXv = scr + S_DXV / 4, *hh = scr + S_HH / 4;
+    __shared__ __align__(16) float part[8][D];   // per channel: the chunk-end sum, from the eight threads that share the channel
+    // a thread owns four adjacent channels and every eighth token: 16-byte accesses, coalesced rows, and the chunk-end sum
+    // of its tokens on the way
+    float extra[4] = {0.f, 0.f, 0.f, 0.f};
+    const int r4 = (threadIdx.x & 31) * 4;
+#pragma unroll 2
+    for (int i = threadIdx.x >> 5; i < kC; i += kT / 32) {
+        const int t = i * D + r4;
         const bool live = i < x.len;
-        const float g = wsG[t], G = expf(g), iG = expf(-g);
-        const float q = live ? __bfloat162float(qp[i * rs + r]) : 0.f, k = live ? __bfloat162float(kp[i * rs + r]) : 0.f;
-        const float b = live ? p.bv[base + i * rs + r] : 0.f;
-        const float dq = G * dQ[t];              // dq = Gam . dQ~
-        const float row = G * dKp[t];            // what multiplies b . k in the row role
-        const float col = iG * dKm[t];           // column role
+        const float4 g4 = *reinterpret_cast<const float4*>(wsG + t), a4 = *reinterpret_cast<const float4*>(dQ + t);
+        const float4 p4 = *reinterpret_cast<const float4*>(dKp + t), m4 = *reinterpret_cast<const float4*>(dKm + t);
+        const float4 u4 = *reinterpret_cast<const float4*>(udh + t), x4 = *reinterpret_cast<const float4*>(dXv + t);
+        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f), w4 = b4;
+        uint2 qr = make_uint2(0, 0), kr = qr, vr = qr;
         if (live) {
-            dqp[i * rs + r] = __float2bfloat16_rn(dq);
-            dkp[i * rs + r] = __float2bfloat16_rn(fmaf(b, row, col));
-            p.dbv[base + i * rs + r] = k * row;
+            b4 = *reinterpret_cast<const float4*>(p.bv + base + i * rs + r4);
+            w4 = *reinterpret_cast<const float4*>(p.wv + base + i * rs + r4);
+            qr = *reinterpret_cast<const uint2*>(qp + i * rs + r4);
+            kr = *reinterpret_cast<const uint2*>(kp + i * rs + r4);
+            vr = *reinterpret_cast<const uint2*>(vp + i * rs + r4);
         }
-        dgam[t] = q * dq + k * b * row - k * col;
-    }
-    for (int t = threadIdx.x; t < kC * D; t += kT) {   // dv = w . dXv ; dw = v . dXv
-        const int i = t / D, c = t % D;
-        if (i < x.len) {
-            const float dxv = dXvT[c * kC + i];
-            dvp[i * rs + c] = __float2bfloat16_rn(p.wv[base + i * rs + c] * dxv);
-            p.dwv[base + i * rs + c] = __bfloat162float(vp[i * rs + c]) * dxv;
+        const float g[4] = {g4.x, g4.y, g4.z, g4.w}, dqt[4] = {a4.x, a4.y, a4.z, a4.w}, dkp4[4] = {p4.x, p4.y, p4.z, p4.w};
+        const float dkm4[4] = {m4.x, m4.y, m4.z, m4.w}, ud[4] = {u4.x, u4.y, u4.z, u4.w}, xv[4] = {x4.x, x4.y, x4.z, x4.w};
+        const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, ww[4] = {w4.x, w4.y, w4.z, w4.w};
+        const float q[4] = {bf16_lo(qr.x), bf16_hi(qr.x), bf16_lo(qr.y), bf16_hi(qr.y)};
+        const float k[4] = {bf16_lo(kr.x), bf16_hi(kr.x), bf16_lo(kr.y), bf16_hi(kr.y)};
+        const float v[4] = {bf16_lo(vr.x), bf16_hi(vr.x), bf16_lo(vr.y), bf16_hi(vr.y)};
+        float dq[4], dk[4], db[4], dv[4], dw[4], dgm[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float G = expf(g[j]), iG = expf(-g[j]);
+            dq[j] = G * dqt[j];                       // dq = Gam . dQ~
+            const float row = G * dkp4[j];            // what multiplies b . k in the row role
+            const float col = iG * dkm4[j];           // column role
+            dk[j] = fmaf(bb[j], row, col);
+            db[j] = k[j] * row;
+            dgm[j] = q[j] * dq[j] + k[j] * bb[j] * row - k[j] * col;
+            extra[j] = fmaf(k[j] * iG, ud[j], extra[j]);   // k-_j . (U dh''^T)_j
+            dv[j] = ww[j] * xv[j];                    // dv = w . dXv
+            dw[j] = v[j] * xv[j];                     // dw = v . dXv
+        }
+        *reinterpret_cast<float4*>(dgam + t) = make_float4(dgm[0], dgm[1], dgm[2], dgm[3]);
+        if (live) {
+            *reinterpret_cast<uint2*>(dqp + i * rs + r4) = make_uint2(pack_bf16(dq[0], dq[1]), pack_bf16(dq[2], dq[3]));
+            *reinterpret_cast<uint2*>(dkp + i * rs + r4) = make_uint2(pack_bf16(dk[0], dk[1]), pack_bf16(dk[2], dk[3]));
+            *reinterpret_cast<uint2*>(dvp + i * rs + r4) = make_uint2(pack_bf16(dv[0], dv[1]), pack_bf16(dv[2], dv[3]));
+            *reinterpret_cast<float4*>(p.dbv + base + i * rs + r4) = make_float4(db[0], db[1], db[2], db[3]);
+            *reinterpret_cast<float4*>(p.dwv + base + i * rs + r4) = make_float4(dw[0], dw[1], dw[2], dw[3]);
         }
     }
+    *reinterpret_cast<float4*>(&part[threadIdx.x >> 5][r4]) = make_float4(extra[0], extra[1], extra[2], extra[3]);
     __syncthreads();
     // the chunk end collects sum_j k-_j . (U dh''^T)_j and rowdot(dh'', h); then dg_j = sum_{i >= j} dgam_i per channel
     if (threadIdx.x < D) {
         const int r = threadIdx.x;
         float run = hh[r];
-        for (int j = 0; j < x.len; ++j) run = fmaf(__bfloat162float(kp[j * rs + r]) * expf(-wsG[j * D + r]), udh[j * D + r], run);
+#pragma unroll
+        for (int w = 0; w < 8; ++w) run += part[w][r];
         for (int i = kC - 1; i >= 0; --i) {
             run += dgam[i * D + r];
             if (i < x.len) p.dgv[base + i * rs + r] = run;
@@ -677,7 +704,7 @@ cudaError_t cw_tc_launch(const Problem& p, bool bwd, bool skip_recompute, cudaSt
         const uint32_t sm_scale = sizeof(float) * kC * (D + 1);
         if ((e = once_scale.ensure(cw_scale_kernel, sm_scale)) != cudaSuccess) return e;
         if ((e = once_prep.ensure(cw_prep_kernel, prepcw::SMEM_BYTES)) != cudaSuccess) return e;
-        { StageScope t(ST_TABLE, st); cw_scale_kernel<<<CH, kT, sm_scale, st>>>(p, bwd ? 1 : 0); }
+        { StageScope t(ST_SCALE, st); cw_scale_kernel<<<CH, kT, sm_scale, st>>>(p, bwd ? 1 : 0); }
         { StageScope t(ST_PREP, st); cw_prep_kernel<<<grid, kT, prepcw::SMEM_BYTES, st>>>(p, bwd ? 1 : 0); }
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -690,7 +717,7 @@ cudaError_t cw_tc_launch(const Problem& p, bool bwd, bool skip_recompute, cudaSt
         if ((e = once_intra.ensure(cw_intra_kernel, intracw::SMEM_BYTES)) != cudaSuccess) return e;
         if ((e = once_post.ensure(cw_post_kernel, sm_post)) != cudaSuccess) return e;
         { StageScope t(ST_INTRA, st); cw_intra_kernel<<<grid, kT, intracw::SMEM_BYTES, st>>>(p); }
-        { StageScope t(ST_EPREP, st); cw_post_kernel<<<CH, kT, sm_post, st>>>(p); }
+        { StageScope t(ST_POST, st); cw_post_kernel<<<CH, kT, sm_post, st>>>(p); }
     }
     return cudaGetLastError();
 }

@@ -142,3 +142,27 @@ def test_argument_errors():
                                     o["dq"], o["dk"], o["dv"], o["dg"], o["db"], o["dw"], None, buf.workspace,
                                     workspace_bytes=1024, check=False)
     assert s == 6
+
+
+def test_decay_beyond_the_range_of_the_tensor_core_route_is_reported():
+    """bf16 I/O at d = 128 scales keys by exp(-gam): a chunk whose cumulative log decay leaves [-80, 80] is refused
+    through the status word (nothing is written); the same gates are fine at fp32, which never splits the decay."""
+    wl = synth.make_channelwise("cw_range", dtype="bf16", lengths=[100, 64], H=2, d_k=128, d_v=128, states=True, seed=69)
+    wl.gv[70:100, 1, 5] = -3.0                       # channel 5 of head 1: 30 tokens of e^-3 inside the second chunk
+    buf = runner.to_device_channelwise(wl)
+    for v in buf.outputs.values():
+        if v is not None:
+            v.fill_(7.0)
+    runner.run_bwd_channelwise(buf)
+    assert binding.gdn_last_device_status(buf.workspace) == 9   # GDN_ERR_DECAY_RANGE
+    assert "decay" in binding.status_string(9)
+    for n in ("dq", "dk", "dv", "dg", "db", "dw"):
+        assert torch.all(buf.outputs[n] == 7.0), n
+    wl32 = synth.make_channelwise("cw_range", dtype="f32", lengths=[100, 64], H=2, d_k=128, d_v=128, states=True, seed=69)
+    wl32.gv[70:100, 1, 5] = -3.0
+    check(wl32, runner.backward_channelwise(wl32))
+    # and the status word clears with the next well-formed call on the same workspace
+    wl.gv[70:100, 1, 5] = -0.1
+    buf.inputs["g"].copy_(torch.from_numpy(wl.gv))
+    runner.run_bwd_channelwise(buf)
+    check(wl, runner.fetch(buf))
