@@ -41,6 +41,9 @@ def parse():
                          "states (value distributions of cfg1); used for kernel studies, not a bench line of its own")
     ap.add_argument("--carries", default="auto", choices=["auto", "operator", "lowrank"],
                     help="form of the inter-chunk carries of the tcgen05 d = 128 family (default: chosen by shape)")
+    ap.add_argument("--channelwise", default=None, choices=["gdn", "kda", "gla"],
+                    help="time gdn_bwd_channelwise (per-channel gate vectors; the named gate setting) on --shape "
+                         "(default 4,2048,16) instead of the headline call; a kernel study, not the bench line")
     ap.add_argument("--arm", default="closed", choices=["closed", "save_forward"],
                     help="closed: gdn_bwd recomputes the forward (the headline); save_forward: every step is "
                          "gdn_fwd_recompute followed by gdn_bwd on its workspace (used when profiling that arm)")
@@ -298,6 +301,37 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_channelwise(args):
+    """gdn_bwd_channelwise on one GPU: device-resident timing, per-kernel times, roofline of its own algorithmic bytes
+    (q, k, v, dO and dq, dk, dv in bf16; g, b, dg, db [.., d_k] and w, dw [.., d_v] in fp32; states)."""
+    import torch
+    from paper_2608_12700_b200 import benchutil, binding, runner, synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B_, T_, H_ = (int(x) for x in (args.shape or "4,2048,16").split(","))
+    wl = synth.make_channelwise(f"channelwise_{args.channelwise}_bf16_B{B_}_T{T_}_H{H_}_d128", member=args.channelwise, dtype="bf16",
+                                B=B_, T=T_, H=H_, d_k=128, d_v=128, seed=7, states=True)
+    buf = runner.to_device_channelwise(wl, dev)
+    stream = torch.cuda.current_stream()
+    step = lambda: runner.run_bwd_channelwise(buf)
+    for _ in range(max(3, args.warmup)):
+        step()
+    ms = time_steps(step, args.steps, torch.cuda.synchronize, stream) / args.steps
+    st = binding.gdn_last_device_status(buf.workspace)
+    if st != binding.GDN_OK:
+        raise binding.GdnError(st, wl.name)
+    stage_ms = stage_pass(buf, runner, binding, 3, step)
+    peaks = benchutil.load_peaks(ROOT)
+    th, chains = wl.T_total * wl.H, wl.N * wl.H
+    alg = th * ((2 * 128 + 2 * 128) * 2 + (2 * 128 + 128) * 4 + (2 * 128 + 128) * 2 + (2 * 128 + 128) * 4) + chains * 3 * 128 * 128 * 4
+    print(json.dumps({"metric": "gdn_bwd_channelwise_tokens_per_sec", "value": wl.tokens / (ms * 1e-3), "unit": UNIT,
+                      "ms_per_step": ms, "steps": args.steps, "config": workload_config(wl),
+                      "stage_ms_per_launch": {k: round(v, 5) for k, v in stage_ms.items()},
+                      "roofline": {"bound": "hbm", "algorithmic_bytes": alg, "achieved": alg / (ms * 1e-3) / 1e9,
+                                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": alg / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   "peak_source": peaks["source"]}}))
+
+
 def time_other_configs(args, peaks, barrier, stream, dev):
     """The other benchmark configurations, briefly (device-resident, same protocol as the headline), so that their
     figures come from the same run on the same machine.  Not bench lines of their own."""
@@ -415,5 +449,7 @@ if __name__ == "__main__":
     a = parse()
     if a.impl == "reference":
         run_reference(a)
+    elif a.channelwise:
+        run_channelwise(a)
     else:
         run_ours(a)
