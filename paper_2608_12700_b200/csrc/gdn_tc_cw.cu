@@ -342,12 +342,12 @@ constexpr uint32_t WT = DOT + 16384;        // W^T  [128][64]                   
 constexpr uint32_t UTT = WT + 16384;        // U~^T [128][64]                                   16 KB
 constexpr uint32_t TT = UTT + 16384;        // T [64][64]; later dA                              8 KB
 constexpr uint32_t PT = TT + 8192;          // P [64][64]; later dP                              8 KB
-constexpr uint32_t HH = PT + 8192;          // h [128][128]; later dXk [64][128] and dXv^T [128][64]    32 KB
+constexpr uint32_t HH = PT + 8192;          // h [128][128]                                     32 KB
 constexpr uint32_t DH = HH + 32768;         // dh'' = Diag(Gam_e) dh' [128][128]                32 KB
-constexpr uint32_t UT = DH + 32768;         // U^T  [128][64]                                   16 KB
-constexpr uint32_t DUT = UT + 16384;        // dU^T [128][64]                                   16 KB
+constexpr uint32_t UT = DH + 32768;         // U^T  [128][64]; later dXk [64][128]              16 KB
+constexpr uint32_t DUT = UT + 16384;        // dU^T [128][64]; later dXv^T [128][64]            16 KB
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = HH, DXVT = HH + 16384;
+constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = UT, DXVT = DUT;   // (dXk over U^T, dXv^T over dU^T: the state tiles are free after round 2)
 // TMEM columns (512 allocated, fixed offsets).  Accumulators with features on the lanes use all 128 lanes (M = 128);
 // token-major ones (M = 64) occupy lanes 0..15 of each lane quadrant.
 //   0..63     (W h)^T  -> dW^T -> dXv^T            (M = 128)
@@ -369,12 +369,16 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
     __shared__ float GL[D];   // Gam_e per key channel
-    __shared__ uint64_t bar_in, bar_mma;
+    __shared__ uint64_t bar_s, bar_a, bar_b, bar_k, bar_q, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    if (threadIdx.x == 0) { mbar_init(&bar_in, 1); mbar_init(&bar_mma, 1); fence_mbar_init(); }
+    if (threadIdx.x == 0) {
+        mbar_init(&bar_s, 1); mbar_init(&bar_a, 1); mbar_init(&bar_b, 1); mbar_init(&bar_k, 1); mbar_init(&bar_q, 1);
+        mbar_init(&bar_mma, 1);
+        fence_mbar_init();
+    }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
@@ -383,36 +387,59 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     const int f = q4 * 32 + lane;             // feature row of the M = 128 accumulators
     const int tr = q4 * 16 + (lane & 15);     // token row of the M = 64 accumulators (lanes 0..15 of the quadrant)
     const bool ga = lane < 16;
-    bool ok = true, pending = false;
+    bool ok = true;
     uint32_t mma_phase = 0, in_phase = 0;
+    // The tiles of a trip arrive in five groups, each loaded during the previous trip as soon as the last product that
+    // reads its region is done (look-ahead without a second buffer):
+    //   s  h, dh'          after round 2      k  K-               after round 5
+    //   a  dO', P          after round 3      q  Q~, K+, T        after round 5 (needed from round 3 on)
+    //   b  W^T, U~^T       after round 4
+    bool pend_s = false, pend_a = false, pend_b = false, pend_k = false, pend_q = false;   // thread 0
+    auto load_s = [&](size_t c) {
+        mbar_expect_tx(&bar_s, 65536);
+        bulk_load(sm + HH, p.ws + p.L.hc + c * 32768, 32768, &bar_s);
+        bulk_load(sm + DH, p.ws + p.L.dhn + c * 32768, 32768, &bar_s);
+        pend_s = true;
+    };
+    auto load_a = [&](size_t c) {
+        mbar_expect_tx(&bar_a, 24576);
+        bulk_load(sm + DOT, p.ws + p.L.img_dO + c * 16384, 16384, &bar_a);
+        bulk_load(sm + PT, p.ws + p.L.Pm + c * 8192, 8192, &bar_a);
+        pend_a = true;
+    };
+    auto load_b = [&](size_t c) {
+        mbar_expect_tx(&bar_b, 32768);
+        bulk_load(sm + WT, p.ws + p.L.img_W + c * 16384, 16384, &bar_b);
+        bulk_load(sm + UTT, p.ws + p.L.img_U + c * 16384, 16384, &bar_b);
+        pend_b = true;
+    };
+    auto load_kq = [&](size_t c) {
+        const char* iQKp = p.ws + p.L.img_QKp + c * 32768;
+        const char* iKm = p.ws + p.L.img_Km + c * 16384;
+        mbar_expect_tx(&bar_k, 16384);
+        for (int cb = 0; cb < 2; ++cb) bulk_load(sm + QKM + cb * 16384 + 8192, iKm + cb * 8192, 8192, &bar_k);      // K-
+        pend_k = true;
+        mbar_expect_tx(&bar_q, 40960);
+        for (int cb = 0; cb < 2; ++cb) {
+            bulk_load(sm + QKM + cb * 16384, iQKp + cb * 16384, 8192, &bar_q);                                        // Q~
+            bulk_load(sm + KP + cb * 8192, iQKp + cb * 16384 + 8192, 8192, &bar_q);                                   // K+
+        }
+        bulk_load(sm + TT, p.ws + p.L.Tm + c * 8192, 8192, &bar_q);
+        pend_q = true;
+    };
+    if (threadIdx.x == 0) { load_s(blockIdx.x); load_kq(blockIdx.x); load_b(blockIdx.x); load_a(blockIdx.x); }
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
         const size_t ch = (size_t)item;
+        const bool has_next = item + (int)gridDim.x < n_items;
+        const size_t chn = ch + gridDim.x;
         float* scr = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * ch);
-        if (threadIdx.x == 0) {
-            mbar_expect_tx(&bar_in, 180224);
-            const char* iQKp = p.ws + p.L.img_QKp + ch * 32768;
-            const char* iKm = p.ws + p.L.img_Km + ch * 16384;
-            for (int cb = 0; cb < 2; ++cb) {
-                bulk_load(sm + QKM + cb * 16384, iQKp + cb * 16384, 8192, &bar_in);             // Q~
-                bulk_load(sm + QKM + cb * 16384 + 8192, iKm + cb * 8192, 8192, &bar_in);        // K-
-                bulk_load(sm + KP + cb * 8192, iQKp + cb * 16384 + 8192, 8192, &bar_in);        // K+
-            }
-            bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
-            bulk_load(sm + WT, p.ws + p.L.img_W + ch * 16384, 16384, &bar_in);
-            bulk_load(sm + UTT, p.ws + p.L.img_U + ch * 16384, 16384, &bar_in);
-            bulk_load(sm + TT, p.ws + p.L.Tm + ch * 8192, 8192, &bar_in);
-            bulk_load(sm + PT, p.ws + p.L.Pm + ch * 8192, 8192, &bar_in);
-            bulk_load(sm + HH, p.ws + p.L.hc + ch * 32768, 32768, &bar_in);
-            bulk_load(sm + DH, p.ws + p.L.dhn + ch * 32768, 32768, &bar_in);
-            pending = true;
-        }
         if (threadIdx.x < D)
             GL[threadIdx.x] = expf(reinterpret_cast<const float*>(p.ws + p.L.gamma)[(ch * kC + kC - 1) * D + threadIdx.x]);
         if (ok) {
-            ok = mbar_wait(&bar_in, in_phase);
+            ok = mbar_wait(&bar_s, in_phase);
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 44);
-            if (ok && threadIdx.x == 0) pending = false;
+            if (ok && threadIdx.x == 0) pend_s = false;
         }
         __syncthreads();
         {   // dh'' = Diag(Gam_e) dh' in place, and rowdot(dh'', h): two threads per state row, eight 16-byte pieces each
@@ -430,6 +457,11 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             }
             hh += __shfl_xor_sync(0xffffffffu, hh, 1);
             if (ok && half == 0) scr[S_HH / 4 + r] = hh;
+        }
+        if (ok) {   // the rest of what round 1 reads
+            ok = mbar_wait(&bar_k, in_phase) && mbar_wait(&bar_b, in_phase) && mbar_wait(&bar_a, in_phase);
+            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 50);
+            if (ok && threadIdx.x == 0) pend_k = pend_a = pend_b = false;
         }
         fence_async_smem();
         __syncthreads();
@@ -472,6 +504,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(46)
+        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time
         if (ok) {
             const int j0 = grp * 32, i0 = grp * 32, c0 = grp * 64;
 #pragma unroll 1
@@ -504,6 +537,11 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         fence_async_smem();
         __syncthreads();
         // ---- round 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
+        if (ok) {
+            ok = mbar_wait(&bar_q, in_phase);
+            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 51);
+            if (ok && threadIdx.x == 0) pend_q = false;
+        }
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 128, 64>(tmem + C_KP, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);
@@ -513,6 +551,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(47)
+        if (ok && has_next && threadIdx.x == 0) load_a(chn);   // dW^T (over dO') and dP (over P) have been read
         if (ok) {
             const int i0 = grp * 32, c0 = grp * 64;
 #pragma unroll 1
@@ -544,6 +583,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(48)
+        if (ok && has_next && threadIdx.x == 0) load_b(chn);   // W^T and U~^T have been read for the last time
         if (ok) {   // dA = -stril(.)
             const int j0 = grp * 32;
 #pragma unroll 1
@@ -570,6 +610,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(49)
+        if (ok && has_next && threadIdx.x == 0) load_kq(chn);   // every tile of this trip has been read for the last time
         if (ok) {
             const int c0 = grp * 64;
 #pragma unroll 1
@@ -594,7 +635,14 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         __syncthreads();   // every reader of this trip's tiles and accumulators is done
         if (!ok) break;
     }
-    if (threadIdx.x == 0 && pending) (void)mbar_wait(&bar_in, in_phase);   // after a timeout a load may still be in flight
+    if (threadIdx.x == 0 && !ok) {   // after a timeout a load may still be in flight: wait for it (bounded) before the CTA retires
+        // a group issued during the trip that gave up belongs to the next phase of its barrier; one pending since the top of
+        // that trip to the current one.  Both parities are tried; the wrong one returns at once or after the bound.
+        uint64_t* bars[5] = {&bar_s, &bar_a, &bar_b, &bar_k, &bar_q};
+        const bool pend[5] = {pend_s, pend_a, pend_b, pend_k, pend_q};
+        for (int i = 0; i < 5; ++i)
+            if (pend[i]) { (void)mbar_wait(bars[i], in_phase); (void)mbar_wait(bars[i], in_phase ^ 1); }
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, 512);
