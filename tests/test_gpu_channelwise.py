@@ -166,3 +166,19 @@ def test_decay_beyond_the_range_of_the_tensor_core_route_is_reported():
     buf.inputs["g"].copy_(torch.from_numpy(wl.gv))
     runner.run_bwd_channelwise(buf)
     check(wl, runner.fetch(buf))
+
+
+def test_tensor_core_route_with_several_trips_per_cta_and_equal_lengths():
+    """More chunk-heads than SMs (every persistent CTA makes at least two trips, some three) and a fixed-length batch
+    (no cu_seqlens): both the look-ahead loads and the arithmetic chunk geometry are exercised."""
+    wl = synth.make_channelwise("cw_trips", member="gdn", dtype="bf16", B=3, T=700, H=10, d_k=128, d_v=128, states=True, seed=70)
+    assert (wl.T_total // 64 + 3) * wl.H > 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    errs, _ = check(wl, runner.backward_channelwise(wl))
+    print(wl.name, errs)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_no_tokens_passes_the_state_gradient_through(dtype, d):
+    wl = synth.make_channelwise("cw_empty", dtype=dtype, lengths=[0, 0], H=2, d_k=d, d_v=d, states=True, seed=71)
+    got = runner.backward_channelwise(wl)
+    assert np.array_equal(got["dh0"], wl.dhT.astype(np.float64))
