@@ -76,8 +76,9 @@ def test_captured_forward_then_backward_on_its_workspace():
     assert np.isfinite(got["o"].float().cpu().numpy()).all()
 
 
-def test_captured_channelwise_backward_replays_bit_exact():
-    wl = synth.make_channelwise("graph_channelwise", member="kda", dtype="bf16", lengths=[100, 64, 30], H=2, d_k=64, d_v=128,
+@pytest.mark.parametrize("dk", [64, 128])   # FFMA kernels / tensor-core route
+def test_captured_channelwise_backward_replays_bit_exact(dk):
+    wl = synth.make_channelwise("graph_channelwise", member="kda", dtype="bf16", lengths=[100, 64, 30], H=2, d_k=dk, d_v=128,
                                 states=True, seed=36)
     buf = runner.to_device_channelwise(wl)
     runner.run_bwd_channelwise(buf)
