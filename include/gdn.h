@@ -56,8 +56,9 @@ typedef enum gdn_status {
     GDN_ERR_WORKSPACE_TOO_SMALL = 6,
     GDN_ERR_CUDA = 7,               /* a CUDA runtime call or launch failed                            */
     GDN_ERR_DEVICE_TIMEOUT = 8,     /* device-side: a bounded wait gave up                             */
-    GDN_ERR_DECAY_RANGE = 9         /* device-side, channel-wise calls on the tensor cores: the cumulative log  */
-                                    /* decay of a chunk leaves [-80, 80] (or is not a number)                   */
+    GDN_ERR_DECAY_RANGE = 9         /* device-side and transient: the tensor-core kernels of a channel-wise call  */
+                                    /* stood down (cumulative log decay of a chunk outside [-80, 80]); the same   */
+                                    /* call then runs on the FFMA kernels and clears it.  Never left behind.      */
 } gdn_status;
 
 typedef enum gdn_dtype { GDN_F32 = 0, GDN_BF16 = 1 } gdn_dtype;
@@ -120,8 +121,9 @@ gdn_status gdn_bwd(const gdn_desc* desc,
  * gate gradients are required outputs.  The workspace has its own size (gdn_workspace_bytes_channelwise) and
  * layout; its status word is read with gdn_last_device_status.  With bf16 I/O at d_k = d_v = 128 these calls run on
  * the tensor cores (tcgen05): keys and queries are scaled by the chunk-local cumulative decay element by element, which
- * requires |sum of g over any prefix of a 64-token chunk| <= 80 per channel; a call whose gates leave that range
- * reports GDN_ERR_DECAY_RANGE through the status word and writes no output (the fp32 dtype has no such limit).  Every
+ * requires |sum of g over any prefix of a 64-token chunk| <= 80 per channel; a call whose gates leave that range is
+ * computed by the FFMA kernels instead (which evaluate the decay inside the contractions and have no such limit): the
+ * decision is taken on the device, the call enqueues the same launches either way and needs no host round trip.  Every
  * other shape and dtype runs on fp32 FFMA kernels (bf16 I/O: inputs and dq, dk, dv are bf16, all arithmetic and the
  * gate tensors are fp32). */
 gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);

@@ -19,7 +19,7 @@ struct Rec { Stage s; cudaEvent_t a, b; };
 std::vector<Rec> g_recs;          // recorded since the last read
 std::vector<cudaEvent_t> g_pool;  // reusable events
 cudaEvent_t g_open = nullptr;
-const char* kStageNames[ST_COUNT] = {"table", "prep", "fscan", "out", "eprep", "rscan", "intra", "scans", "scale", "post"};
+const char* kStageNames[ST_COUNT] = {"table", "prep", "fscan", "out", "eprep", "rscan", "intra", "scans", "scale", "post", "fallback"};
 cudaEvent_t take_event() {
     if (!g_pool.empty()) { cudaEvent_t e = g_pool.back(); g_pool.pop_back(); return e; }
     cudaEvent_t e = nullptr;

@@ -107,12 +107,12 @@ inline WsLayout make_layout_vec(const gdn_desc& d, size_t scratch_per_ch) {
     L.img_QKp = take(L.tc_scans ? CH * 32768 : 0);
     L.img_Km = take(L.tc_scans ? CH * 16384 : 0);
     L.img_Vt = take(L.tc_scans ? CH * 16384 : 0);
-    L.hc = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
+    L.hc = take(4 * CH * d.d_k * d.d_v);   // (fp32, or a bf16 tile image in the first half of each slot)
     L.fwd_end = o;
     L.E = take(4 * CH * d.d_k * d.d_v);
     L.img_E = take(L.tc_scans ? CH * 32768 : 0);
     L.img_dO = take(L.tc_scans ? CH * 16384 : 0);
-    L.dhn = take((L.tc_scans ? 2 : 4) * CH * d.d_k * d.d_v);
+    L.dhn = take(4 * CH * d.d_k * d.d_v);
     L.scratch_per_ch = scratch_per_ch;
     L.scratch = take(scratch_per_ch * CH);
     L.total = o;
@@ -131,13 +131,14 @@ struct Problem {
     // channel-wise entry points only: gate vectors g, b [.., d_k], w [.., d_v] and their gradients (g, dg above unused)
     const float *gv, *bv, *wv;
     float *dgv, *dbv, *dwv;
+    int fallback;   // channel-wise FFMA kernels only: 1 = run only if the tensor-core route has refused the gates (status word)
     char* ws;
     WsLayout L;
 };
 
 // Launch bookkeeping: every kernel launch goes through stage_begin / stage_end so that launches can be
 // counted and, when enabled, timed per stage with CUDA events on the launching stream.
-enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_SCANS, ST_SCALE, ST_POST, ST_COUNT };
+enum Stage { ST_TABLE = 0, ST_PREP, ST_FSCAN, ST_OUT, ST_EPREP, ST_RSCAN, ST_INTRA, ST_SCANS, ST_SCALE, ST_POST, ST_FALLBACK, ST_COUNT };
 void stage_begin(Stage s, cudaStream_t st);
 void stage_end(Stage s, cudaStream_t st);
 struct StageScope {

@@ -43,6 +43,17 @@ __device__ __forceinline__ void mac_decay(float (&acc)[4][4], int i0, int j0, in
     }
 }
 
+// Whether this launch has work: normally when no earlier stage has reported an error; a launch of the fall-back sequence
+// only when the tensor-core route has refused the gates of this call (decided on the device, no host round trip).
+__device__ __forceinline__ bool vec_go(const Problem& p) {
+    const int st = reinterpret_cast<const WsHeader*>(p.ws)->status;
+    return p.fallback ? st == GDN_ERR_DECAY_RANGE : st == GDN_OK;
+}
+__global__ void vec_clear_refusal_kernel(Problem p) {
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(p.ws);
+    if (hdr->status == GDN_ERR_DECAY_RANGE) { hdr->status = GDN_OK; hdr->detail = 0; }
+}
+
 // Element (r, c) of a bf16 tile image with R rows (the operand format of the tensor-core kernels).
 __device__ __forceinline__ void img_put(char* img, int R, int r, int c, float x) {
     *reinterpret_cast<__nv_bfloat16*>(img + tc::tile_off(R, r, c)) = __float2bfloat16_rn(x);
@@ -74,7 +85,7 @@ __device__ __forceinline__ void load_gamma(const float* wsG, float* gam) {
 template <typename IO, int DK, int DV>
 __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
     ChunkCtx x;
-    if (!chunk_ctx(p, x)) return;
+    if (!vec_go(p) || !chunk_ctx(p, x)) return;
     extern __shared__ __align__(16) float smf[];
     float* gam = smf;                                   // [64][DK + 1]
     float (*A)[kC + 1] = reinterpret_cast<float (*)[kC + 1]>(smf + kC * (DK + 1));
@@ -156,7 +167,7 @@ __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 __global__ void __launch_bounds__(kThreads) veprep_kernel(Problem p) {
     ChunkCtx x;
-    if (!chunk_ctx(p, x)) return;
+    if (!vec_go(p) || !chunk_ctx(p, x)) return;
     const int H = p.d.H;
     const IO* qp = reinterpret_cast<const IO*>(p.q) + ((size_t)x.tok0 * H + x.hd) * DK;
     const IO* gp = reinterpret_cast<const IO*>(p.dO) + ((size_t)x.tok0 * H + x.hd) * DV;
@@ -199,8 +210,7 @@ __global__ void __launch_bounds__(kThreads) vscan_kernel(Problem p) {
     float* Y = nxt + DK * DV;         // [64][DV]: U = Ut - W h (forward) or Kb dh' (reverse)
     const int H = p.d.H, n = blockIdx.x / H, hd = blockIdx.x % H;
     const int32_t* seq_first = reinterpret_cast<const int32_t*>(p.ws + p.L.seq_first);
-    const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
-    if (hdr->status != GDN_OK) return;
+    if (!vec_go(p)) return;
     const int c0 = seq_first[n], c1 = seq_first[n + 1];
     const size_t soff = ((size_t)n * H + hd) * DK * DV;
     const float* init = REVERSE ? p.dhT : p.h0;
@@ -258,7 +268,7 @@ __global__ void __launch_bounds__(kThreads) vscan_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 __global__ void __launch_bounds__(kThreads) vout_kernel(Problem p) {
     ChunkCtx x;
-    if (!chunk_ctx(p, x)) return;
+    if (!vec_go(p) || !chunk_ctx(p, x)) return;
     const int H = p.d.H;
     const IO* qp = reinterpret_cast<const IO*>(p.q) + ((size_t)x.tok0 * H + x.hd) * DK;
     IO* op = reinterpret_cast<IO*>(p.o) + ((size_t)x.tok0 * H + x.hd) * DV;
@@ -306,7 +316,7 @@ __global__ void __launch_bounds__(kThreads) vout_kernel(Problem p) {
 template <typename IO, int DK, int DV>
 __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     ChunkCtx x;
-    if (!chunk_ctx(p, x)) return;
+    if (!vec_go(p) || !chunk_ctx(p, x)) return;
     extern __shared__ __align__(16) float smf[];
     float* gam = smf;                                                                       // [64][DK + 1]
     float (*dP)[kC + 1] = reinterpret_cast<float (*)[kC + 1]>(smf + kC * (DK + 1));         // scale tril(dO U^T)
@@ -465,58 +475,71 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     }
 }
 
+// The FFMA sequences.  `q` is the problem as these kernels see it (fp32 factors and states); with q.fallback set the chunk
+// table is not rebuilt (the tensor-core route has built it, and rebuilding would reset the status word the launches look at).
 template <typename IO, int DK, int DV>
-cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st, bool with_scan = true) {
-    const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
-    if (p.L.tc_scans) {   // bf16 I/O at d = 128: scaled operand images, tcgen05 preparation and carry
-        cudaError_t e = cw_tc_launch(p, /*bwd=*/false, false, st);
-        if (e != cudaSuccess) return e;
-        if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
-        return cudaGetLastError();
-    }
-    launch_table(p, st);
+cudaError_t ffma_fwd(const Problem& q, cudaStream_t st) {
+    const int CH = q.L.max_chunks * q.d.H, chains = q.d.N * q.d.H;
+    if (!q.fallback) launch_table(q, st);
     const size_t smp = sizeof(float) * (kC * (DK + 1) + 2 * kC * (kC + 1));
     cudaError_t e = cudaFuncSetAttribute(vprep_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smp);
     if (e != cudaSuccess) return e;
-    if (CH > 0) { StageScope t(ST_PREP, st); vprep_kernel<IO, DK, DV><<<CH, kThreads, smp, st>>>(p); }
-    if (with_scan) {
-        if (p.L.tc_scans) {
-            if (chains > 0 && (e = tc_launch_scan_channelwise(p, 0, st)) != cudaSuccess) return e;
-        } else {
-            const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
-            e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-            if (e != cudaSuccess) return e;
-            if (chains > 0) { StageScope t(ST_FSCAN, st); vscan_kernel<IO, DK, DV, false><<<chains, kThreads, sm, st>>>(p); }
-        }
-    }
-    if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
+    if (CH > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_PREP, st); vprep_kernel<IO, DK, DV><<<CH, kThreads, smp, st>>>(q); }
+    const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
+    e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    if (chains > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_FSCAN, st); vscan_kernel<IO, DK, DV, false><<<chains, kThreads, sm, st>>>(q); }
+    if (q.o && CH > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(q); }
     return cudaGetLastError();
 }
 
 template <typename IO, int DK, int DV>
-cudaError_t vlaunch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st) {
+cudaError_t ffma_bwd(const Problem& q, bool skip_recompute, cudaStream_t st) {
     cudaError_t e;
-    if (p.L.tc_scans) return cw_tc_launch(p, /*bwd=*/true, skip_recompute, st);   // bf16 I/O at d = 128: all on tcgen05
-    const bool tcs = false;
-    if (!skip_recompute) {
-        e = vlaunch_fwd_t<IO, DK, DV>(p, st, /*with_scan=*/!tcs);
-        if (e != cudaSuccess) return e;
-    }
-    const int CH = p.L.max_chunks * p.d.H, chains = p.d.N * p.d.H;
-    if (CH > 0) { StageScope t(ST_EPREP, st); veprep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
-    if (tcs) {
-        if (chains > 0 && (e = tc_launch_scan_channelwise(p, skip_recompute ? 1 : 2, st)) != cudaSuccess) return e;
-    } else {
-        const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
-        e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-        if (e != cudaSuccess) return e;
-        if (chains > 0) { StageScope t(ST_RSCAN, st); vscan_kernel<IO, DK, DV, true><<<chains, kThreads, sm, st>>>(p); }
-    }
+    if (!skip_recompute && (e = ffma_fwd<IO, DK, DV>(q, st)) != cudaSuccess) return e;
+    const int CH = q.L.max_chunks * q.d.H, chains = q.d.N * q.d.H;
+    if (CH > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_EPREP, st); veprep_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(q); }
+    const size_t sm = sizeof(float) * (2 * DK * DV + kC * DV);
+    e = cudaFuncSetAttribute(vscan_kernel<IO, DK, DV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    if (chains > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_RSCAN, st); vscan_kernel<IO, DK, DV, true><<<chains, kThreads, sm, st>>>(q); }
     const size_t smi = sizeof(float) * (kC * (DK + 1) + 2 * kC * (kC + 1));
     e = cudaFuncSetAttribute(vintra_kernel<IO, DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smi);
     if (e != cudaSuccess) return e;
-    if (CH > 0) { StageScope t(ST_INTRA, st); vintra_kernel<IO, DK, DV><<<CH, kThreads, smi, st>>>(p); }
+    if (CH > 0) { StageScope t(q.fallback ? ST_FALLBACK : ST_INTRA, st); vintra_kernel<IO, DK, DV><<<CH, kThreads, smi, st>>>(q); }
     return cudaGetLastError();
+}
+
+// bf16 I/O at d = 128 runs on the tensor cores (gdn_tc_cw.cu).  That route refuses gates whose chunk-cumulative log decay
+// leaves its range, through the status word; the FFMA sequence is therefore enqueued behind it in fall-back mode: its
+// launches return at once unless the status word says so, in which case they compute the call (with the decay inside the
+// contractions there is no range limit) and clear the refusal.  No host round trip, the same launches every call.
+template <typename IO, int DK, int DV>
+cudaError_t ffma_fallback(const Problem& p, bool bwd, bool skip_recompute, cudaStream_t st) {
+    Problem q = p;
+    q.fallback = 1;
+    q.L.tc_scans = 0;
+    cudaError_t e = bwd ? ffma_bwd<IO, DK, DV>(q, skip_recompute, st) : ffma_fwd<IO, DK, DV>(q, st);
+    if (e != cudaSuccess) return e;
+    { StageScope t(ST_FALLBACK, st); vec_clear_refusal_kernel<<<1, 1, 0, st>>>(q); }
+    return cudaGetLastError();
+}
+
+template <typename IO, int DK, int DV>
+cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st) {
+    if (!p.L.tc_scans) return ffma_fwd<IO, DK, DV>(p, st);
+    const int CH = p.L.max_chunks * p.d.H;
+    cudaError_t e = cw_tc_launch(p, /*bwd=*/false, false, st);
+    if (e != cudaSuccess) return e;
+    if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
+    return ffma_fallback<IO, DK, DV>(p, false, false, st);
+}
+
+template <typename IO, int DK, int DV>
+cudaError_t vlaunch_bwd_t(const Problem& p, bool skip_recompute, cudaStream_t st) {
+    if (!p.L.tc_scans) return ffma_bwd<IO, DK, DV>(p, skip_recompute, st);
+    const cudaError_t e = cw_tc_launch(p, /*bwd=*/true, skip_recompute, st);
+    return e != cudaSuccess ? e : ffma_fallback<IO, DK, DV>(p, true, skip_recompute, st);
 }
 
 }  // namespace

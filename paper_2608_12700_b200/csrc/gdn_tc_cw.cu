@@ -15,7 +15,8 @@
 // and the gradients of the caller's tensors follow element by element (cw_post).  Four kernels beside the carries
 // (tc_scan_cw in gdn_tc.cu):
 //   cw_scale  scaled operand tiles as bf16 tile images, gam; checks that |gam| stays below 80 (beyond that the split
-//             would need reference points inside the chunk; the call then reports GDN_ERR_DECAY_RANGE and writes nothing)
+//             would need reference points inside the chunk): otherwise it records GDN_ERR_DECAY_RANGE, the kernels below
+//             stand down, and the FFMA sequence enqueued behind them computes the call (gdn_simt_vec.cu)
 //   cw_prep   [Q~;K+] K-^T, fp32 blocked inversion, W^T, U~^T, (P^T dO')^T, E               (tcgen05)
 //   cw_intra  the sixteen products of the gradient stage in five dependent rounds (K#2 reuses T)   (tcgen05)
 //   cw_post   dq, dk, dv, db, dw, and dg by a reverse cumulative sum per channel

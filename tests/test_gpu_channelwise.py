@@ -144,28 +144,33 @@ def test_argument_errors():
     assert s == 6
 
 
-def test_decay_beyond_the_range_of_the_tensor_core_route_is_reported():
-    """bf16 I/O at d = 128 scales keys by exp(-gam): a chunk whose cumulative log decay leaves [-80, 80] is refused
-    through the status word (nothing is written); the same gates are fine at fp32, which never splits the decay."""
+def test_decay_beyond_the_range_of_the_tensor_core_route_falls_back_on_the_device():
+    """bf16 I/O at d = 128 scales keys by exp(-gam), which is only safe while the cumulative log decay of a chunk stays in
+    [-80, 80].  A call whose gates leave that range is computed by the FFMA kernels instead (the decision is taken on the
+    device: the tensor-core kernels stand down, the fall-back launches behind them do the work) and must be just as
+    right; the status word ends up clean, and the next call with tame gates is back on the tensor cores."""
     wl = synth.make_channelwise("cw_range", dtype="bf16", lengths=[100, 64], H=2, d_k=128, d_v=128, states=True, seed=69)
     wl.gv[70:100, 1, 5] = -3.0                       # channel 5 of head 1: 30 tokens of e^-3 inside the second chunk
-    buf = runner.to_device_channelwise(wl)
+    buf = runner.to_device_channelwise(wl, want_o=True)
     for v in buf.outputs.values():
         if v is not None:
-            v.fill_(7.0)
+            v.fill_(float("nan"))
     runner.run_bwd_channelwise(buf)
-    assert binding.gdn_last_device_status(buf.workspace) == 9   # GDN_ERR_DECAY_RANGE
-    assert "decay" in binding.status_string(9)
-    for n in ("dq", "dk", "dv", "dg", "db", "dw"):
-        assert torch.all(buf.outputs[n] == 7.0), n
-    wl32 = synth.make_channelwise("cw_range", dtype="f32", lengths=[100, 64], H=2, d_k=128, d_v=128, states=True, seed=69)
-    wl32.gv[70:100, 1, 5] = -3.0
-    check(wl32, runner.backward_channelwise(wl32))
-    # and the status word clears with the next well-formed call on the same workspace
+    assert binding.gdn_last_device_status(buf.workspace) == binding.GDN_OK
+    errs, ref = check(wl, runner.fetch(buf))
+    assert max(errs[n] for n in ("dg", "db", "dw", "dh0")) < 1e-5     # fp32 arithmetic on that route (dq, dk, dv are bf16)
+    # forward outputs and the save-forward arm take the same decision
+    runner.run_fwd_channelwise(buf)
+    f = runner.fetch(buf)
+    assert rel(f["o"], ref["o"]) < TOL["bf16"] and rel(f["hT"], ref["hT"]) < 1e-5
+    runner.run_bwd_channelwise(buf, fresh=1)
+    check(wl, runner.fetch(buf))
+    # tame gates again: tensor-core route, bf16-level errors in the gate gradients
     wl.gv[70:100, 1, 5] = -0.1
     buf.inputs["g"].copy_(torch.from_numpy(wl.gv))
     runner.run_bwd_channelwise(buf)
-    check(wl, runner.fetch(buf))
+    errs, _ = check(wl, runner.fetch(buf))
+    assert errs["dg"] > 1e-4
 
 
 def test_tensor_core_route_with_several_trips_per_cta_and_equal_lengths():
