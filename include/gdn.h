@@ -119,13 +119,14 @@ gdn_status gdn_bwd(const gdn_desc* desc,
  * gdn_fwd_recompute / gdn_bwd; desc->delta_rule is not read (the gates say which family member runs: KDA is
  * b = w = beta broadcast over the channels, GLA is b = 0, w = 1, the full GDN has independent vectors).  All three
  * gate gradients are required outputs.  The workspace has its own size (gdn_workspace_bytes_channelwise) and
- * layout; its status word is read with gdn_last_device_status.  With bf16 I/O at d_k = d_v = 128 these calls run on
- * the tensor cores (tcgen05): keys and queries are scaled by the chunk-local cumulative decay element by element, which
+ * layout; its status word is read with gdn_last_device_status.  With bf16 I/O these calls run on the tensor cores
+ * (tcgen05; kernels for d_k = d_v = 128, a head dimension of 64 is zero-padded to 128 inside the workspace, gate
+ * vectors included, which is exact): keys and queries are scaled by the chunk-local cumulative decay element by element, which
  * requires |sum of g over any prefix of a 64-token chunk| <= 80 per channel; a call whose gates leave that range is
  * computed by the FFMA kernels instead (which evaluate the decay inside the contractions and have no such limit): the
- * decision is taken on the device, the call enqueues the same launches either way and needs no host round trip.  Every
- * other shape and dtype runs on fp32 FFMA kernels (bf16 I/O: inputs and dq, dk, dv are bf16, all arithmetic and the
- * gate tensors are fp32). */
+ * decision is taken on the device, the call enqueues the same launches either way and needs no host round trip.  fp32
+ * I/O runs on fp32 FFMA kernels throughout (with bf16 I/O they take bf16 inputs and give bf16 dq, dk, dv; all their
+ * arithmetic and the gate tensors are fp32). */
 gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes);
 gdn_status gdn_fwd_recompute_channelwise(const gdn_desc* desc,
                                          const void* q, const void* k, const void* v,
@@ -156,6 +157,10 @@ const char* gdn_status_string(gdn_status s);
  * kernels of their own, zero-padded onto the d = 128 tensor-core kernels inside the workspace),
  * or NULL for an unsupported descriptor.  Diagnostic only. */
 const char* gdn_kernel_path(const gdn_desc* desc);
+/* The same for the channel-wise calls: "tcgen05_bf16_channelwise" (bf16, d_k = d_v = 128),
+ * "tcgen05_bf16_channelwise_padded" (bf16, a head dimension of 64: zero-padded onto the former inside the workspace),
+ * "simt_f32_channelwise", "simt_bf16_channelwise" (the latter only under gdn_debug_force_family(1)). */
+const char* gdn_kernel_path_channelwise(const gdn_desc* desc);
 
 /* ---- backward without a caller-provided workspace (the paper has no counterpart) ----------------
  * Some callers may not allocate device memory at the point where they need the gradients: code running

@@ -21,7 +21,7 @@ STATUS_NAMES = {0: "GDN_OK", 1: "GDN_ERR_NULL_ARG", 2: "GDN_ERR_BAD_SHAPE", 3: "
                 7: "GDN_ERR_CUDA", 8: "GDN_ERR_DEVICE_TIMEOUT", 9: "GDN_ERR_DECAY_RANGE"}
 
 EXPORTS = ["gdn_workspace_bytes", "gdn_fwd_recompute", "gdn_bwd", "gdn_last_device_status",
-           "gdn_status_string", "gdn_kernel_path", "gdn_launch_count", "gdn_stage_timing_enable",
+           "gdn_status_string", "gdn_kernel_path", "gdn_kernel_path_channelwise", "gdn_launch_count", "gdn_stage_timing_enable",
            "gdn_stage_timing_read", "gdn_debug_read", "gdn_debug_force_family", "gdn_bwd_noalloc",
            "gdn_noalloc_last_device_status", "gdn_workspace_bytes_channelwise", "gdn_fwd_recompute_channelwise",
            "gdn_bwd_channelwise", "gdn_debug_inject_timeout"]
@@ -65,6 +65,8 @@ def lib():
         L.gdn_status_string.argtypes = [I]
         L.gdn_kernel_path.restype = ctypes.c_char_p
         L.gdn_kernel_path.argtypes = [D]
+        L.gdn_kernel_path_channelwise.restype = ctypes.c_char_p
+        L.gdn_kernel_path_channelwise.argtypes = [D]
         L.gdn_launch_count.restype = ctypes.c_uint64
         L.gdn_launch_count.argtypes = []
         L.gdn_stage_timing_enable.restype = I
@@ -120,6 +122,11 @@ def status_string(status: int) -> str:
 
 def gdn_kernel_path(desc: gdn_desc) -> Optional[str]:
     r = lib().gdn_kernel_path(ctypes.byref(desc))
+    return None if r is None else r.decode()
+
+
+def gdn_kernel_path_channelwise(desc: gdn_desc) -> Optional[str]:
+    r = lib().gdn_kernel_path_channelwise(ctypes.byref(desc))
     return None if r is None else r.decode()
 
 

@@ -77,12 +77,30 @@ WsLayout layout_for(const gdn_desc& d) {
         const gdn_desc w = tc_padded_desc(d);
         WsLayout L = make_layout(w, 2, 2, 0, !tc_carries_lowrank(w));
         L.scratch = align_up(L.total, 256);
-        L.total = L.scratch + tc_padded_extra_bytes(d);
+        L.total = L.scratch + tc_padded_extra_bytes(d, false);
         L.fwd_end = L.total;
         return L;
     }
     // The SIMT kernels keep every factor in fp32, whatever the I/O dtype.
     return make_layout(d, sizeof(float), sizeof(float), simt_scratch_per_chunkhead(d));
+}
+
+// Channel-wise calls: the layout the kernels see (of the widened problem when a head dimension of 64 is zero-padded onto
+// the d = 128 tensor-core route) and the sizes the caller is told (padded: one size for both calls).
+struct VecPlan {
+    bool padded;
+    WsLayout inner;
+    size_t fwd_bytes, total;
+};
+VecPlan vec_plan(const gdn_desc& d) {
+    VecPlan v{};
+    v.padded = tc_padded_supported(d) && g_force_family != 1;
+    const gdn_desc w = v.padded ? tc_padded_desc(d) : d;
+    v.inner = make_layout_vec(w, vec_scratch_per_chunkhead(w));
+    if (g_force_family == 1) v.inner.tc_scans = 0;   // (debug override: the FFMA kernels; the image regions stay unused)
+    v.total = v.padded ? align_up(v.inner.total, 256) + tc_padded_extra_bytes(d, true) : v.inner.total;
+    v.fwd_bytes = v.padded ? v.total : v.inner.fwd_end;
+    return v;
 }
 
 }  // namespace
@@ -162,7 +180,7 @@ gdn_status gdn_fwd_recompute(const gdn_desc* desc, const void* q, const void* k,
     cudaError_t e;
     if (path == Path::TcBf16Padded) {
         const gdn_desc w = tc_padded_desc(*desc);
-        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), false, false, st);
+        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), false, false, false, st);
     } else {
         e = path == Path::TcBf16 ? tc_launch_fwd(p, st) : path == Path::Tc64Bf16 ? tc64_launch_fwd(p, st) : simt_launch_fwd(p, st);
     }
@@ -189,7 +207,7 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
     cudaError_t e;
     if (path == Path::TcBf16Padded) {
         const gdn_desc w = tc_padded_desc(*desc);
-        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), true, fresh, st);
+        e = tc_padded_launch(p, make_layout(w, 2, 2, 0, !tc_carries_lowrank(w)), true, fresh, false, st);
     } else {
         e = path == Path::TcBf16 ? tc_launch_bwd(p, fresh, st)
             : path == Path::Tc64Bf16 ? tc64_launch_bwd(p, fresh, st) : simt_launch_bwd(p, fresh, st);
@@ -201,9 +219,9 @@ gdn_status gdn_bwd(const gdn_desc* desc, const void* q, const void* k, const voi
 gdn_status gdn_workspace_bytes_channelwise(const gdn_desc* desc, size_t* fwd_bytes, size_t* bwd_bytes) {
     gdn_status s = check_desc(desc);
     if (s != GDN_OK) return s;
-    const WsLayout L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
-    if (fwd_bytes) *fwd_bytes = L.fwd_end;
-    if (bwd_bytes) *bwd_bytes = L.total;
+    const VecPlan v = vec_plan(*desc);
+    if (fwd_bytes) *fwd_bytes = v.fwd_bytes;
+    if (bwd_bytes) *bwd_bytes = v.total;
     return GDN_OK;
 }
 
@@ -222,11 +240,14 @@ gdn_status gdn_fwd_recompute_channelwise(const gdn_desc* desc, const void* q, co
     Problem p{};
     p.d = *desc;
     p.Ttot = desc->B * desc->T;
-    p.L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
-    if (workspace_bytes < p.L.fwd_end) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    const VecPlan plan = vec_plan(*desc);
+    p.L = plan.inner;
+    if (workspace_bytes < plan.fwd_bytes) return GDN_ERR_WORKSPACE_TOO_SMALL;
     p.q = q; p.k = k; p.v = v; p.gv = g; p.bv = b; p.wv = w; p.h0 = h0; p.cu = cu; p.o = o; p.hT = hT;
     p.ws = static_cast<char*>(workspace);
-    return vec_launch_fwd(p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t e = plan.padded ? tc_padded_launch(p, plan.inner, false, false, true, st) : vec_launch_fwd(p, st);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 gdn_status gdn_bwd_channelwise(const gdn_desc* desc, const void* q, const void* k, const void* v, const float* g,
@@ -245,13 +266,16 @@ gdn_status gdn_bwd_channelwise(const gdn_desc* desc, const void* q, const void* 
     Problem p{};
     p.d = *desc;
     p.Ttot = desc->B * desc->T;
-    p.L = make_layout_vec(*desc, vec_scratch_per_chunkhead(*desc));
-    if (workspace_bytes < p.L.total) return GDN_ERR_WORKSPACE_TOO_SMALL;
+    const VecPlan plan = vec_plan(*desc);
+    p.L = plan.inner;
+    if (workspace_bytes < plan.total) return GDN_ERR_WORKSPACE_TOO_SMALL;
     p.q = q; p.k = k; p.v = v; p.gv = g; p.bv = b; p.wv = w; p.h0 = h0; p.dO = dO; p.dhT = dhT; p.cu = cu;
     p.dq = dq; p.dk = dk; p.dv = dv; p.dgv = dg; p.dbv = db; p.dwv = dw; p.dh0 = dh0;
     p.ws = static_cast<char*>(workspace);
-    return vec_launch_bwd(p, workspace_is_fresh_from_fwd != 0, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
-               ? GDN_OK : GDN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const bool fresh = workspace_is_fresh_from_fwd != 0;
+    const cudaError_t e = plan.padded ? tc_padded_launch(p, plan.inner, true, fresh, true, st) : vec_launch_bwd(p, fresh, st);
+    return e == cudaSuccess ? GDN_OK : GDN_ERR_CUDA;
 }
 
 gdn_status gdn_last_device_status(const void* workspace, void* cuda_stream) {
@@ -364,6 +388,13 @@ gdn_status gdn_stage_timing_read(int32_t max_stages, float* total_ms, int32_t* l
     for (int i = 0; i < n; ++i) { total_ms[i] = ms[i]; launches[i] = cnt[i]; names[i] = kStageNames[i]; }
     *n_stages = n;
     return rc;
+}
+
+const char* gdn_kernel_path_channelwise(const gdn_desc* desc) {
+    if (check_desc(desc) != GDN_OK) return nullptr;
+    if (g_force_family != 1 && tc_padded_supported(*desc)) return "tcgen05_bf16_channelwise_padded";
+    if (g_force_family != 1 && vec_tc_scans(*desc)) return "tcgen05_bf16_channelwise";
+    return desc->dtype == GDN_BF16 ? "simt_bf16_channelwise" : "simt_f32_channelwise";
 }
 
 const char* gdn_kernel_path(const gdn_desc* desc) {

@@ -200,11 +200,12 @@ cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 
 
-// bf16 delta-rule shapes with a head dimension of 64, zero-padded onto the d = 128 kernels (gdn_pad.cu).
+// bf16 shapes with a head dimension of 64, zero-padded onto the d = 128 kernels (gdn_pad.cu); `channelwise`: the call has
+// gate vectors, which are padded too, and the widened problem runs through vec_launch_fwd / vec_launch_bwd.
 bool tc_padded_supported(const gdn_desc& d);
 gdn_desc tc_padded_desc(const gdn_desc& d);          // the widened descriptor (d_k = d_v = 128)
-size_t tc_padded_extra_bytes(const gdn_desc& d);     // bytes of padded copies behind the widened problem's own workspace
-cudaError_t tc_padded_launch(const Problem& p, const WsLayout& inner, bool bwd, bool skip_recompute, cudaStream_t st);
+size_t tc_padded_extra_bytes(const gdn_desc& d, bool channelwise);   // bytes of padded copies behind the widened problem's own workspace
+cudaError_t tc_padded_launch(const Problem& p, const WsLayout& inner, bool bwd, bool skip_recompute, bool channelwise, cudaStream_t st);
 
 // tcgen05 family for the scalar-gate recurrence (bf16 I/O, d_k = d_v = 64, delta rule off).
 bool tc64_supported(const gdn_desc& d);

@@ -187,3 +187,43 @@ def test_no_tokens_passes_the_state_gradient_through(dtype, d):
     wl = synth.make_channelwise("cw_empty", dtype=dtype, lengths=[0, 0], H=2, d_k=d, d_v=d, states=True, seed=71)
     got = runner.backward_channelwise(wl)
     assert np.array_equal(got["dh0"], wl.dhT.astype(np.float64))
+
+
+@pytest.mark.parametrize("member", ["gdn", "kda"])
+@pytest.mark.parametrize("dk,dv", [(128, 64), (64, 128), (64, 64)])
+def test_head_dimension_64_is_padded_onto_the_tensor_core_route(dk, dv, member):
+    """bf16 I/O with a head dimension of 64: inputs, gate vectors and states are zero-padded to d = 128 inside the
+    workspace and the tcgen05 kernels run (a padded key channel has decay 1 and erase gate 0, a padded value channel
+    write gate 0: every product is what it was).  Against the oracle, with the forward outputs and the save-forward
+    arm; the FFMA family on the same inputs must agree with the oracle too."""
+    wl = synth.make_channelwise(f"cw_pad_{dk}_{dv}_{member}", member=member, dtype="bf16", lengths=[65, 128, 0, 37, 300], H=3,
+                                d_k=dk, d_v=dv, states=True, seed=71, scale=0.5)
+    buf = runner.to_device_channelwise(wl, want_o=True)
+    assert binding.gdn_kernel_path_channelwise(buf.desc) == "tcgen05_bf16_channelwise_padded"
+    runner.run_bwd_channelwise(buf)
+    got = runner.fetch(buf)
+    errs, ref = check(wl, got)
+    print(wl.name, errs)
+    assert np.array_equal(got["dh0"][2], wl.dhT[2].astype(np.float64))
+    runner.run_fwd_channelwise(buf)
+    f = runner.fetch(buf)
+    assert rel(f["o"], ref["o"]) < TOL["bf16"] and rel(f["hT"], ref["hT"]) < TOL["bf16"]
+    runner.run_bwd_channelwise(buf, fresh=1)
+    fresh = runner.fetch(buf)
+    for n in GRADS:
+        assert np.array_equal(fresh[n], got[n]), n
+    binding.gdn_debug_force_family(1)
+    try:
+        fbuf = runner.to_device_channelwise(wl)
+        assert binding.gdn_kernel_path_channelwise(fbuf.desc) == "simt_bf16_channelwise"
+        runner.run_bwd_channelwise(fbuf)
+        check(wl, runner.fetch(fbuf))
+    finally:
+        binding.gdn_debug_force_family(0)
+
+
+def test_kernel_path_names():
+    mk = lambda dt, dk, dv: binding.make_desc(B=1, T=64, H=1, d_k=dk, d_v=dv, N=1, dtype=dt)
+    assert binding.gdn_kernel_path_channelwise(mk("bf16", 128, 128)) == "tcgen05_bf16_channelwise"
+    assert binding.gdn_kernel_path_channelwise(mk("bf16", 64, 64)) == "tcgen05_bf16_channelwise_padded"
+    assert binding.gdn_kernel_path_channelwise(mk("f32", 128, 128)) == "simt_f32_channelwise"
