@@ -217,3 +217,39 @@ def config(i: int, *, heads: Optional[int] = None) -> Workload:
         return make_workload(CONFIG_NAMES[4], dtype="bf16", H=heads or 32, d_k=128, d_v=128, seed=4,
                              lengths=draw_packed_lengths(4), states=True)
     raise ValueError("config index must be 0..4")
+
+
+def device_inputs(*, B: int, T: int, H: int, d_k: int, d_v: int, dtype: str, seed: int, device="cuda:0",
+                  g_scale: float = 0.1, delta_rule: int = 1, states: bool = False, state_std: float = 0.1):
+    """The same value distributions as `make_workload`, drawn on the device with torch's generator, one batch row at a
+    time: for inputs too large to be drawn on the host and uploaded (tensors beyond 4 GiB).  Returns a dict of torch
+    tensors q, k [B*T, H, d_k], v, dO [B*T, H, d_v] (I/O dtype), g, beta [B*T, H] (fp32; beta None without the delta
+    rule), h0, dhT [B, H, d_k, d_v] (fp32, or None).  Whoever wants a CPU result copies the rows it needs to the host."""
+    import torch
+
+    dev = torch.device(device)
+    io = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    q = torch.empty((B * T, H, d_k), dtype=io, device=dev)
+    k = torch.empty_like(q)
+    v = torch.empty((B * T, H, d_v), dtype=io, device=dev)
+    dO = torch.empty_like(v)
+    g = torch.empty((B * T, H), dtype=torch.float32, device=dev)
+    beta = torch.empty_like(g) if delta_rule else None
+    normal = lambda *shape: torch.randn(shape, generator=gen, device=dev, dtype=torch.float32)
+    for n in range(B):
+        rows = slice(n * T, (n + 1) * T)
+        for dst, d in ((q, d_k), (k, d_k)):
+            x = normal(T, H, d)
+            dst[rows] = (x / x.norm(dim=-1, keepdim=True).clamp_min(1e-30)).to(io)
+        v[rows] = normal(T, H, d_v).to(io)
+        dO[rows] = normal(T, H, d_v).to(io)
+        g[rows] = -g_scale * torch.nn.functional.softplus(normal(T, H))
+        if delta_rule:
+            beta[rows] = torch.sigmoid(normal(T, H))
+    h0 = dhT = None
+    if states:
+        h0 = state_std * normal(B, H, d_k, d_v)
+        dhT = state_std * normal(B, H, d_k, d_v)
+    return dict(q=q, k=k, v=v, dO=dO, g=g, beta=beta, h0=h0, dhT=dhT)
