@@ -29,7 +29,9 @@
  * frees nothing.  Inputs are never written.  Outputs are overwritten for every valid token.  All work
  * is enqueued on the caller's stream (a cudaStream_t passed as void*, NULL = default stream) and the
  * calls return without synchronising; cu_seqlens is never read on the host.  The workspace is scratch
- * owned by the caller; two calls may not share one workspace concurrently.
+ * owned by the caller; two calls may not share one workspace concurrently.  The entry points may be called
+ * from several host threads at once (each call with its own workspace, on any stream): the library keeps
+ * no per-call state outside the workspace, and results do not depend on what else runs on the device.
  *
  * Errors.  Argument errors are detected on the host before anything is launched and returned as a
  * status; nothing is thrown, aborted or trapped.  Conditions only visible on the device (malformed
