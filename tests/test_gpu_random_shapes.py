@@ -71,3 +71,18 @@ def test_channelwise_gates(seed):
         assert rel(got[n], ref[n]) <= TOL[wl.dtype], (wl.name, member, n, rel(got[n], ref[n]))
         e, _ = block_errors(wl, n, got[n], ref[n])
         assert e.size == 0 or e.max() <= BLOCK_TOL[wl.dtype], (wl.name, member, n, float(e.max()))
+
+
+@pytest.mark.parametrize("dtype,d,delta", [("bf16", 128, 1), ("bf16", 64, 0), ("f32", 64, 1)])
+def test_thousands_of_short_sequences(dtype, d, delta):
+    """A packed batch of 3000 sequences of 0..150 tokens (many of them empty or shorter than a chunk): the chunk table,
+    the chain-per-CTA carries and the persistent chunk kernels with far more chains than SMs."""
+    rng = np.random.default_rng(4242)
+    lengths = rng.integers(0, 151, size=3000)
+    lengths[rng.random(3000) < 0.1] = 0
+    wl = synth.make_workload(f"many_short_{dtype}_{d}", dtype=dtype, lengths=lengths.tolist(), H=2, d_k=d, d_v=d, states=True,
+                             delta_rule=delta, seed=4243)
+    got = runner.backward(wl)
+    check_against_oracle(wl, got)
+    empty = np.flatnonzero(lengths == 0)
+    assert np.array_equal(got["dh0"][empty], wl.dhT[empty].astype(np.float64))   # empty sequences pass dhT through
