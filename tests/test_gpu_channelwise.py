@@ -227,3 +227,13 @@ def test_kernel_path_names():
     assert binding.gdn_kernel_path_channelwise(mk("bf16", 128, 128)) == "tcgen05_bf16_channelwise"
     assert binding.gdn_kernel_path_channelwise(mk("bf16", 64, 64)) == "tcgen05_bf16_channelwise_padded"
     assert binding.gdn_kernel_path_channelwise(mk("f32", 128, 128)) == "simt_f32_channelwise"
+
+
+def test_full_size_shape_of_the_bench_every_chain():
+    """The workload `bench.py` times for the channel-wise calls (KDA gates, bf16, B = 4, T = 2048, H = 16, d = 128; 2048
+    chunk-heads, 14 trips per persistent CTA), every chain against the per-channel oracle, whole tensors and 64-token
+    blocks."""
+    wl = synth.make_channelwise("channelwise_kda_bf16_B4_T2048_H16_d128", member="kda", dtype="bf16", B=4, T=2048, H=16,
+                                d_k=128, d_v=128, seed=7, states=True)
+    errs, _ = check(wl, runner.backward_channelwise(wl))
+    print(wl.name, errs)
