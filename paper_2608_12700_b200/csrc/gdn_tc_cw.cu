@@ -18,10 +18,10 @@
 //             would need reference points inside the chunk): otherwise it records GDN_ERR_DECAY_RANGE, the kernels below
 //             stand down, and the FFMA sequence enqueued behind them computes the call (gdn_simt_vec.cu)
 //   cw_prep   [Q~;K+] K-^T, fp32 blocked inversion, W^T, U~^T, (P^T dO')^T, E               (tcgen05)
-//   cw_intra  the sixteen products of the gradient stage in five dependent rounds (K#2 reuses T)   (tcgen05)
+//   cw_intra  the sixteen products of the gradient stage in five dependent steps (K#2 reuses T)   (tcgen05)
 //   cw_post   dq, dk, dv, db, dw, and dg by a reverse cumulative sum per channel
 // The tensor-core kernels are written straight-line (one CTA per SM walks over chunk-heads; one thread issues every
-// product and copy; CTA-wide barriers between the rounds): the plain statement of the channel-wise path on tcgen05,
+// product and copy; CTA-wide barriers between the steps): the plain statement of the channel-wise path on tcgen05,
 // not a tuned one.  Accumulators live in one TMEM reservation at fixed column offsets; every wait is bounded.
 #include "tc_common.cuh"
 #include "tc_inverse.cuh"
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
             if (ok && threadIdx.x == 0) pending = false;
         }
         __syncthreads();
-        // ---- round 1: S1 = [Q~; K+] K-^T  (rows 0..63: P before masking, rows 64..127: A)
+        // ---- step 1: S1 = [Q~; K+] K-^T  (rows 0..63: P before masking, rows 64..127: A)
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<128, 64, 128>(tmem + C_S1, op_k_major(sm + QKP, 128, 0), op_k_major(sm + KM, 64), false);
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
         }
         fence_async_smem();
         __syncthreads();
-        // ---- round 2: W^T = K+^T T^T ; U~^T = V~^T T^T
+        // ---- step 2: W^T = K+^T T^T ; U~^T = V~^T T^T
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<128, 64, 64>(tmem + C_W, op_mn_major(sm + QKP, 128, 64), op_k_major(sm + TT, 64), false);
@@ -290,7 +290,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- round 3: E = Q~^T dO' - W^T (P^T dO')
+        // ---- step 3: E = Q~^T dO' - W^T (P^T dO')
         if (bwd) {
             if (ok && threadIdx.x == 0) {
                 tc_fence_after();
@@ -348,7 +348,7 @@ constexpr uint32_t DH = HH + 32768;         // dh'' = Diag(Gam_e) dh' [128][128]
 constexpr uint32_t UT = DH + 32768;         // U^T  [128][64]; later dXk [64][128]              16 KB
 constexpr uint32_t DUT = UT + 16384;        // dU^T [128][64]; later dXv^T [128][64]            16 KB
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = UT, DXVT = DUT;   // (dXk over U^T, dXv^T over dU^T: the state tiles are free after round 2)
+constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = UT, DXVT = DUT;   // (dXk over U^T, dXv^T over dU^T: the state tiles are free after step 2)
 // TMEM columns (512 allocated, fixed offsets).  Accumulators with features on the lanes use all 128 lanes (M = 128);
 // token-major ones (M = 64) occupy lanes 0..15 of each lane quadrant.
 //   0..63     (W h)^T  -> dW^T -> dXv^T            (M = 128)
@@ -392,9 +392,9 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     uint32_t mma_phase = 0, in_phase = 0;
     // The tiles of a trip arrive in five groups, each loaded during the previous trip as soon as the last product that
     // reads its region is done (look-ahead without a second buffer):
-    //   s  h, dh'          after round 2      k  K-               after round 5
-    //   a  dO', P          after round 3      q  Q~, K+, T        after round 5 (needed from round 3 on)
-    //   b  W^T, U~^T       after round 4
+    //   s  h, dh'          after step 2      k  K-               after step 5
+    //   a  dO', P          after step 3      q  Q~, K+, T        after step 5 (needed from step 3 on)
+    //   b  W^T, U~^T       after step 4
     bool pend_s = false, pend_a = false, pend_b = false, pend_k = false, pend_q = false;   // thread 0
     auto load_s = [&](size_t c) {
         mbar_expect_tx(&bar_s, 65536);
@@ -459,14 +459,14 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             hh += __shfl_xor_sync(0xffffffffu, hh, 1);
             if (ok && half == 0) scr[S_HH / 4 + r] = hh;
         }
-        if (ok) {   // the rest of what round 1 reads
+        if (ok) {   // the rest of what step 1 reads
             ok = mbar_wait(&bar_k, in_phase) && mbar_wait(&bar_b, in_phase) && mbar_wait(&bar_a, in_phase);
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 50);
             if (ok && threadIdx.x == 0) pend_k = pend_a = pend_b = false;
         }
         fence_async_smem();
         __syncthreads();
-        // ---- round 1: (W h)^T ; (K- dh'')^T ; (P^T dO')^T
+        // ---- step 1: (W h)^T ; (K- dh'')^T ; (P^T dO')^T
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<128, 64, 128>(tmem + C_A, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
@@ -495,7 +495,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- round 2: dO' U^T ; dW^T = -(dU h^T)^T ; dO' h^T ; U dh''^T
+        // ---- step 2: dO' U^T ; dW^T = -(dU h^T)^T ; dO' h^T ; U dh''^T
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 64, 128>(tmem + C_PP, op_k_major(sm + DOT, 64), op_mn_major(sm + UT, 128), false);
@@ -537,7 +537,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- round 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
+        // ---- step 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
         if (ok) {
             ok = mbar_wait(&bar_q, in_phase);
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 51);
@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- round 4 (K#2, the sandwich): dXk W^T + dXv U~^T
+        // ---- step 4 (K#2, the sandwich): dXk W^T + dXv U~^T
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 64, 128>(tmem + C_PP, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
@@ -603,7 +603,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- round 5: dK+ += dA K- ; dK- += dA^T K+
+        // ---- step 5: dK+ += dA K- ; dK- += dA^T K+
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 128, 64>(tmem + C_KP, op_k_major(sm + DA, 64), op_mn_major(sm + QKM, 128, 64), true);
