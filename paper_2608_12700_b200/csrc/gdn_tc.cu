@@ -40,6 +40,7 @@ struct TcParams {
     Problem p;
     CUtensorMap tm_q, tm_k, tm_v, tm_do;   // [T_total, H * 128] bf16, boxes of 64 rows x 64 columns
     CUtensorMap tm_dq, tm_dk, tm_dv;       // same geometry, for the gradient stores of full chunks
+    CUtensorMap tm_o;                      // same geometry, for the forward output (forward calls that want it)
     int with_bwd;                          // prep: also produce E
     int scan_dirs;                         // scan: 0 = forward carry only, 1 = reverse only, 2 = both
     int lowrank;                           // carries in low-rank form (tc_scan_lr): tc_prep makes no Nm, Bf
@@ -1473,19 +1474,32 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 }
 
 // ------------------------------------------------------------------------------------------------
-// tc_out (optional forward output): o = scale (Diag(Gam) Q h + P (U~ - W h))
+// tc_out (optional forward output): o = scale (Diag(Gam) Q h + P (U~ - W h)),  P = tril(Q K^T . D)
+//
+// Persistent, two CTAs per SM (96 KB of shared memory, 256 TMEM columns each): a CTA walks through the dependent
+// steps of one chunk-head while its neighbour is in another step of another one.  The tiles of the next trip are
+// loaded as soon as the last product (or store) that reads their region is done.  Q h and P U are formed token-major
+// (M = 64: a thread owns a token row), so the output tile is staged with 16-byte stores and leaves by TMA.
 // ------------------------------------------------------------------------------------------------
 namespace outk {
-constexpr uint32_t QK = 0, WT = 32768, UTT = WT + 16384, HH = UTT + 16384, PT = HH + 32768, UT = PT + 8192, STG = UT + 16384;
-constexpr uint32_t SMEM_BYTES = STG + 16384 + 1024;
+constexpr uint32_t QK = 0;                  // [Q rows 0..63 ; K rows 64..127] x 128              32 KB
+constexpr uint32_t WT = 32768;              // W^T [128][64]; after the first products: P [64][64]  16 KB
+constexpr uint32_t UTT = WT + 16384;        // U~^T [128][64]; U^T in place                         16 KB
+constexpr uint32_t HH = UTT + 16384;        // h [128][128]; after the first products: staged o     32 KB
+constexpr uint32_t PT = WT, STG = HH;
+constexpr uint32_t SMEM_BYTES = HH + 32768 + 1024 /* alignment slack */;
+constexpr uint32_t C_P = 0, C_WH = 64, C_QH = 128, C_PU = 0;   // TMEM columns (256 allocated)
+constexpr uint32_t IN_BYTES = 32768 + 16384 + 16384 + 32768;
+static_assert(2 * (SMEM_BYTES + 4096) <= 228 * 1024, "two CTAs per SM");
 }  // namespace outk
 
-__global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_constant__ TcParams P) {
+__global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_constant__ TcParams P) {
     using namespace outk;
     const Problem& p = P.p;
-    ChunkInfo x;
-    if (!chunk_info(p, x)) return;
     const int H = p.d.H;
+    if (reinterpret_cast<const WsHeader*>(p.ws)->status != GDN_OK) return;
+    const int n_items = n_chunks_of(p) * H;
+    if ((int)blockIdx.x >= n_items) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
     __shared__ __align__(16) float gl[kC], Gam[kC];
@@ -1500,85 +1514,143 @@ __global__ void __launch_bounds__(kThreads, 1) tc_out_kernel(const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    if (threadIdx.x == 0) {
-        mbar_expect_tx(&bar_in, 32768 + 16384 + 16384 + 32768);
+    bool ok = true, pending = false;
+    uint32_t mma_phase = 0, in_phase = 0, pending_phase = 0;   // (pending_phase: the phase of bar_in the loads in flight belong to)
+    // One mbarrier phase per trip collects all five tiles; they are issued in three pieces, each when its region is free.
+    auto load_qk = [&](const ChunkInfo& c, uint32_t phase) {   // thread 0; first piece of a trip: announces the whole trip's bytes
+        pending_phase = phase;
+        mbar_expect_tx(&bar_in, IN_BYTES);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, x.hd * D + cb * 64, x.tok0, &bar_in);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, x.hd * D + cb * 64, x.tok0, &bar_in);
+            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, c.hd * D + cb * 64, c.tok0, &bar_in);
+            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, c.hd * D + cb * 64, c.tok0, &bar_in);
         }
-        bulk_load(sm + WT, p.ws + p.L.W + (size_t)x.ch * 16384, 16384, &bar_in);
-        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)x.ch * 16384, 16384, &bar_in);
-        bulk_load(sm + HH, p.ws + p.L.hc + (size_t)x.ch * 32768, 32768, &bar_in);
-    }
-    if (threadIdx.x < kC) {
-        const float g = reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)x.ch * kC + threadIdx.x];
-        gl[threadIdx.x] = g * kLog2e;
-        Gam[threadIdx.x] = expf(g);
-    }
-    bool ok = mbar_wait(&bar_in, 0);
-    uint32_t mma_phase = 0;
-    if (!ok && threadIdx.x == 0) report_timeout(p.ws, 30);
-    if (ok && x.len < kC) {
-        zero_tail_rows(sm + QK, 128, 0, x.len);
-        zero_tail_rows(sm + QK, 128, 64, x.len);
-        fence_async_smem();
-    }
-    __syncthreads();
-    if (ok && threadIdx.x == 0) {
-        tc_fence_after();
-        mma_tile<64, 64, 128>(tmem + 0, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
-        mma_tile<128, 64, 128>(tmem + 64, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
-        mma_tile<128, 64, 128>(tmem + 128, op_mn_major(sm + HH, 128), op_k_major(sm + QK, 128, 0), false);
-        mma_commit(&bar_mma);
-    }
-    GDN_WAIT_MMA(31)
-    const int f = q4 * 32 + lane, i0 = half * 32, mi = q4 * 16 + lane, j0 = half * 32;
-    if (ok) {
+        pending = true;
+    };
+    auto load_wu = [&](const ChunkInfo& c) {
+        bulk_load(sm + WT, p.ws + p.L.W + (size_t)c.ch * 16384, 16384, &bar_in);
+        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)c.ch * 16384, 16384, &bar_in);
+    };
+    auto load_h = [&](const ChunkInfo& c) { bulk_load(sm + HH, p.ws + p.L.hc + (size_t)c.ch * 32768, 32768, &bar_in); };
+    auto fetch_gamma = [&](const ChunkInfo& c) {   // threads 0..63: cumulative log decay of their token
+        return reinterpret_cast<const float*>(p.ws + p.L.gamma)[(size_t)c.ch * kC + threadIdx.x];
+    };
+    ChunkInfo x;
+    chunk_entry(p, x, blockIdx.x);
+    if (threadIdx.x == 0) { load_qk(x, 0); load_wu(x); load_h(x); }
+    float gnext = threadIdx.x < kC ? fetch_gamma(x) : 0.f;
+    const int f = q4 * 32 + lane;            // feature row of the transposed accumulator (W h)^T
+    const int tr = q4 * 16 + (lane & 15);    // token row of the M = 64 accumulators (lanes 0..15 of a quadrant hold them)
+    const bool ga = lane < 16;
+    const float sc = p.d.scale;
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
-            float v[8], u[8], t[8];
-            const int jb = j0 + part * 8, ib = i0 + part * 8;
-            tmem_ld8(tmem + lane_base + 0 + jb, v);
-            tmem_ld8(tmem + lane_base + 64 + ib, t);
-            chunk_load(sm + UTT, 128, f, ib >> 3, u);
-            tmem_wait_ld();
-            if (lane < 16) {
-                float g8[8];
-                ld8s(gl + jb, g8);
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
+        const bool has_next = item + (int)gridDim.x < n_items;
+        ChunkInfo xn = x;
+        if (has_next) chunk_entry(p, xn, item + gridDim.x);
+        if (threadIdx.x < kC) {
+            gl[threadIdx.x] = gnext * kLog2e;
+            Gam[threadIdx.x] = expf(gnext);
+        }
+        if (ok) {
+            ok = mbar_wait(&bar_in, in_phase);
+            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 30);
+            if (ok && threadIdx.x == 0) pending = false;
+        }
+        if (ok && x.len < kC) {   // ragged tail: rows beyond the sequence belong to somebody else
+            zero_tail_rows(sm + QK, 128, 0, x.len);
+            zero_tail_rows(sm + QK, 128, 64, x.len);
+            fence_async_smem();
+        }
+        __syncthreads();
+        // ---- step 1: Q K^T ; (W h)^T ; Q h
+        if (ok && threadIdx.x == 0) {
+            tc_fence_after();
+            mma_tile<64, 64, 128>(tmem + C_P, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
+            mma_tile<128, 64, 128>(tmem + C_WH, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
+            mma_tile<64, 128, 128>(tmem + C_QH, op_k_major(sm + QK, 128, 0), op_mn_major(sm + HH, 128), false);
+            mma_commit(&bar_mma);
+        }
+        GDN_WAIT_MMA(31)
+        if (ok && has_next) {   // Q and K have been read for the last time
+            if (threadIdx.x == 0) load_qk(xn, in_phase ^ 1);
+            if (threadIdx.x < kC) gnext = fetch_gamma(xn);
+        }
+        if (ok) {   // P = tril(Q K^T . D) over W^T (dead), U = U~ - W h in place
+            const int i0 = half * 32, j0 = half * 32;
+#pragma unroll 1
+            for (int part = 0; part < 4; ++part) {
+                float v[8], u[8], t[8];
+                const int jb = j0 + part * 8, ib = i0 + part * 8;
+                tmem_ld8(tmem + lane_base + C_P + jb, v);
+                tmem_ld8(tmem + lane_base + C_WH + ib, t);
+                chunk_load(sm + UTT, 128, f, ib >> 3, u);
+                tmem_wait_ld();
+                if (ga) {
+                    float g8[8];
+                    ld8s(gl + jb, g8);
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = (jb + j <= mi) ? v[j] * ex2(gl[mi] - g8[j]) : 0.f;
-                chunk_store(sm + PT, 64, mi, jb >> 3, v);
+                    for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? v[j] * ex2(gl[tr] - g8[j]) : 0.f;
+                    chunk_store(sm + PT, 64, tr, jb >> 3, v);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) u[i] -= t[i];
+                chunk_store(sm + UTT, 128, f, ib >> 3, u);
             }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) u[i] -= t[i];
-            chunk_store(sm + UT, 128, f, ib >> 3, u);
         }
-    }
-    tc_fence_before();
-    fence_async_smem();
-    __syncthreads();
-    if (ok && threadIdx.x == 0) {
-        tc_fence_after();
-        mma_tile<128, 64, 64>(tmem + 192, op_k_major(sm + UT, 128), op_k_major(sm + PT, 64), false);
-        mma_commit(&bar_mma);
-    }
-    GDN_WAIT_MMA(32)
-    if (ok) {
-        const float sc = p.d.scale;
+        tc_fence_before();
+        fence_async_smem();
+        __syncthreads();
+        // ---- step 2: P U (token-major, over the columns of the first two accumulators)
+        if (ok && threadIdx.x == 0) {
+            tc_fence_after();
+            mma_tile<64, 128, 64>(tmem + C_PU, op_k_major(sm + PT, 64), op_k_major(sm + UTT, 128), false);
+            mma_commit(&bar_mma);
+        }
+        GDN_WAIT_MMA(32)
+        if (ok && has_next && threadIdx.x == 0) load_wu(xn);   // P (over W^T) and U^T have been read for the last time
+        if (ok) {   // o = scale (Gam . (Q h) + P U): the sixteen low lanes of a warp own a token row and 64 columns each
+            const float coef = sc * Gam[tr];
 #pragma unroll 1
-        for (int part = 0; part < 4; ++part) {
-            const int ib = i0 + part * 8;
-            float a[8], b[8];
-            tmem_ld8(tmem + lane_base + 128 + ib, a);
-            tmem_ld8(tmem + lane_base + 192 + ib, b);
-            tmem_wait_ld();
+            for (int part = 0; part < 8; ++part) {
+                const int cb = half * 64 + part * 8;
+                float a[8], b[8];
+                tmem_ld8(tmem + lane_base + C_QH + cb, a);
+                tmem_ld8(tmem + lane_base + C_PU + cb, b);
+                tmem_wait_ld();
+                if (ga) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) tile_put(sm + STG, 64, ib + i, f, sc * fmaf(Gam[ib + i], a[i], b[i]));
+                    for (int j = 0; j < 8; ++j) b[j] = fmaf(coef, a[j], sc * b[j]);
+                    chunk_store(sm + STG, 64, tr, cb >> 3, b);
+                }
+            }
         }
+        tc_fence_before();
+        fence_async_smem();
+        __syncthreads();
+        if (ok) {
+            if (x.len == kC) {
+                if (threadIdx.x == 0) {
+                    for (int cb = 0; cb < 2; ++cb) tma_store_2d(&P.tm_o, x.hd * D + cb * 64, x.tok0, sm + STG + cb * 8192);
+                    bulk_commit();
+                }
+            } else {
+                flush_rows(sm + STG, reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)x.tok0 * H + x.hd) * D, (size_t)H * D, x.len);
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) {
+                bulk_wait_read<0>();            // the store has read the staged tile: h of the next trip may land on it
+                if (has_next) load_h(xn);
+            }
+        }
+        if (!ok) break;
+        x = xn;
+    }
+    if (threadIdx.x == 0) {
+        bulk_wait_read<0>();
+        if (pending) (void)mbar_wait(&bar_in, pending_phase);   // after a timeout a load may still be in flight
     }
     tc_fence_before();
     __syncthreads();
-    if (ok) flush_rows(sm + STG, reinterpret_cast<__nv_bfloat16*>(p.o) + ((size_t)x.tok0 * H + x.hd) * D, (size_t)H * D, x.len);
     if (warp == 0) tmem_dealloc(tmem, 256);
 }
 
@@ -1615,6 +1687,7 @@ static bool fill_params(TcParams& P, const Problem& p, bool with_bwd, int scan_d
     if (!tc::make_tmap_bf16_2d(&P.tm_k, p.k, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_v, p.v, rows, cols, pitch, 64)) return false;
     if (!tc::make_tmap_bf16_2d(&P.tm_do, with_bwd ? p.dO : p.v, rows, cols, pitch, 64)) return false;
+    if (!with_bwd && p.o && !tc::make_tmap_bf16_2d(&P.tm_o, p.o, rows, cols, pitch, 64)) return false;
     if (with_bwd) {
         if (!tc::make_tmap_bf16_2d(&P.tm_dq, p.dq, rows, cols, pitch, 64)) return false;
         if (!tc::make_tmap_bf16_2d(&P.tm_dk, p.dk, rows, cols, pitch, 64)) return false;
@@ -1685,7 +1758,8 @@ static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
 }
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done;
-    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, P.p.L.max_chunks * P.p.d.H, kThreads, P, st);
+    const int items = P.p.L.max_chunks * P.p.d.H, ctas = 2 * sm_count();
+    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, items < ctas ? items : ctas, kThreads, P, st);
 }
 
 // Carries of the channel-wise path: dirs = 0 forward, 1 reverse, 2 both in one launch.  Needs the tile images the
