@@ -196,6 +196,7 @@ bool tc_supported(const gdn_desc& d);
 // fresh from the forward, so that the layout of a workspace does not depend on which call sized it.
 bool tc_carries_lowrank(const gdn_desc& d);
 cudaError_t tc_launch_scan_channelwise(const Problem& p, int dirs, cudaStream_t st);   // carries of the channel-wise path
+cudaError_t tc_launch_out_channelwise(const Problem& p, cudaStream_t st);              // its forward output (p.o non-null)
 cudaError_t tc_launch_fwd(const Problem& p, cudaStream_t st);
 cudaError_t tc_launch_bwd(const Problem& p, bool skip_recompute, cudaStream_t st);
 

@@ -54,14 +54,6 @@ __global__ void vec_clear_refusal_kernel(Problem p) {
     if (hdr->status == GDN_ERR_DECAY_RANGE) { hdr->status = GDN_OK; hdr->detail = 0; }
 }
 
-// Element (r, c) of a bf16 tile image with R rows (the operand format of the tensor-core kernels).
-__device__ __forceinline__ void img_put(char* img, int R, int r, int c, float x) {
-    *reinterpret_cast<__nv_bfloat16*>(img + tc::tile_off(R, r, c)) = __float2bfloat16_rn(x);
-}
-__device__ __forceinline__ float img_get(const char* img, int R, int r, int c) {
-    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(img + tc::tile_off(R, r, c)));
-}
-
 // Chunk-local cumulative log decay per channel into shared memory (pitch DK + 1); rows beyond the sequence repeat the
 // last valid row (identity padding: g = 0 there).
 template <int DK>
@@ -107,7 +99,6 @@ __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
     float* wsW = reinterpret_cast<float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
     float* wsU = reinterpret_cast<float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
 
-    const bool imgs = p.L.tc_scans != 0;
     cumulate_gates<DK>(p, x, gam);
     __syncthreads();
     for (int t = threadIdx.x; t < kC * DK; t += blockDim.x) wsG[t] = gam[(t / DK) * (DK + 1) + t % DK];
@@ -140,25 +131,14 @@ __global__ void __launch_bounds__(kThreads) vprep_kernel(Problem p) {
         mac(acc, i0, j0, kC, [&](int i, int m) { return Ti[i][m]; },
             [&](int m, int j) { return expf(gam[m * (DK + 1) + j]) * Bf(m, j) * Kf(m, j); });
         for (int a = 0; a < 4; ++a)
-            for (int b = 0; b < 4; ++b) {
-                wsW[(i0 + a) * DK + j0 + b] = acc[a][b];
-                if (imgs) img_put(p.ws + p.L.img_W + (size_t)x.ch * 16384, 128, j0 + b, i0 + a, acc[a][b]);   // W^T [d_k][tokens]
-            }
+            for (int b = 0; b < 4; ++b) wsW[(i0 + a) * DK + j0 + b] = acc[a][b];
     });
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
         mac(acc, i0, j0, kC, [&](int i, int m) { return Ti[i][m]; }, [&](int m, int j) { return Wf(m, j) * Vf(m, j); });
         for (int a = 0; a < 4; ++a)
-            for (int b = 0; b < 4; ++b) {
-                wsU[(i0 + a) * DV + j0 + b] = acc[a][b];
-                if (imgs) img_put(p.ws + p.L.img_U + (size_t)x.ch * 16384, 128, j0 + b, i0 + a, acc[a][b]);   // U~^T [d_v][tokens]
-            }
+            for (int b = 0; b < 4; ++b) wsU[(i0 + a) * DV + j0 + b] = acc[a][b];
     });
-    if (imgs)   // Kb_j = exp(gam_e - gam_j) . k_j, [tokens][d_k]; rows beyond the sequence are zero
-        for (int t = threadIdx.x; t < kC * DK; t += blockDim.x) {
-            const int i = t / DK, r = t % DK;
-            img_put(p.ws + p.L.img_K + (size_t)x.ch * 16384, 64, i, r, expf(gam[(kC - 1) * (DK + 1) + r] - gam[i * (DK + 1) + r]) * Kf(i, r));
-        }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -192,10 +172,7 @@ __global__ void __launch_bounds__(kThreads) veprep_kernel(Problem p) {
         float acc[4][4] = {};
         mac(acc, i0, j0, kC, [&](int i, int m) { return X[m * DK + i]; }, Of);
         for (int a = 0; a < 4; ++a)
-            for (int b = 0; b < 4; ++b) {
-                wsE[(i0 + a) * DV + j0 + b] = sc * acc[a][b];
-                if (p.L.tc_scans) img_put(p.ws + p.L.img_E + (size_t)x.ch * 32768, 128, i0 + a, j0 + b, sc * acc[a][b]);
-            }
+            for (int b = 0; b < 4; ++b) wsE[(i0 + a) * DV + j0 + b] = sc * acc[a][b];
     });
 }
 
@@ -275,23 +252,14 @@ __global__ void __launch_bounds__(kThreads) vout_kernel(Problem p) {
     const size_t rk = (size_t)H * DK, rv = (size_t)H * DV;
     auto Qf = [&](int i, int m) -> float { return i < x.len ? ldf(qp + i * rk + m) : 0.f; };
     const float* wsG = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC * DK;
-    const bool img = p.L.tc_scans != 0;   // tensor-core route: the factors and states are bf16 tile images
-    auto Pf = [&](int i, int m) -> float {
-        return img ? img_get(p.ws + p.L.Pm + (size_t)x.ch * 8192, 64, i, m)
-                   : reinterpret_cast<const float*>(p.ws + p.L.Pm)[(size_t)x.ch * kC * kC + i * kC + m];
-    };
-    auto Wm = [&](int i, int m) -> float {   // W[i][m]
-        return img ? img_get(p.ws + p.L.img_W + (size_t)x.ch * 16384, 128, m, i)
-                   : reinterpret_cast<const float*>(p.ws + p.L.W)[(size_t)x.ch * kC * DK + i * DK + m];
-    };
-    auto Um = [&](int i, int j) -> float {   // U~[i][j]
-        return img ? img_get(p.ws + p.L.img_U + (size_t)x.ch * 16384, 128, j, i)
-                   : reinterpret_cast<const float*>(p.ws + p.L.Ut)[(size_t)x.ch * kC * DV + i * DV + j];
-    };
-    const char* hraw = p.ws + p.L.hc;
-    auto Hf = [&](int m, int j) -> float {
-        return img ? img_get(hraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(hraw)[(size_t)x.ch * DK * DV + m * DV + j];
-    };
+    const float* wsP = reinterpret_cast<const float*>(p.ws + p.L.Pm) + (size_t)x.ch * kC * kC;
+    const float* wsW = reinterpret_cast<const float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
+    const float* wsU = reinterpret_cast<const float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
+    const float* wsH = reinterpret_cast<const float*>(p.ws + p.L.hc) + (size_t)x.ch * DK * DV;
+    auto Pf = [&](int i, int m) -> float { return wsP[i * kC + m]; };
+    auto Wm = [&](int i, int m) -> float { return wsW[i * DK + m]; };
+    auto Um = [&](int i, int j) -> float { return wsU[i * DV + j]; };
+    auto Hf = [&](int m, int j) -> float { return wsH[m * DV + j]; };
     float* U = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);  // [64, DV]
     tiles(kC, DV, [&](int i0, int j0) {
         float acc[4][4] = {};
@@ -342,16 +310,10 @@ __global__ void __launch_bounds__(kThreads) vintra_kernel(Problem p) {
     const float* Pm = reinterpret_cast<const float*>(p.ws + p.L.Pm) + (size_t)x.ch * kC * kC;
     const float* W = reinterpret_cast<const float*>(p.ws + p.L.W) + (size_t)x.ch * kC * DK;
     const float* Ut = reinterpret_cast<const float*>(p.ws + p.L.Ut) + (size_t)x.ch * kC * DV;
-    // per-chunk states: fp32 row-major, or the bf16 tile images the tensor-core carries leave
-    const bool img = p.L.tc_scans != 0;
-    const char* hraw = p.ws + p.L.hc;
-    const char* dhraw = p.ws + p.L.dhn;
-    auto Hs = [&](int m, int j) -> float {   // h[m][j]
-        return img ? img_get(hraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(hraw)[(size_t)x.ch * DK * DV + m * DV + j];
-    };
-    auto DHs = [&](int m, int j) -> float {  // dh'[m][j]
-        return img ? img_get(dhraw + (size_t)x.ch * 32768, 128, m, j) : reinterpret_cast<const float*>(dhraw)[(size_t)x.ch * DK * DV + m * DV + j];
-    };
+    const float* hs = reinterpret_cast<const float*>(p.ws + p.L.hc) + (size_t)x.ch * DK * DV;     // per-chunk states, fp32
+    const float* dhs = reinterpret_cast<const float*>(p.ws + p.L.dhn) + (size_t)x.ch * DK * DV;
+    auto Hs = [&](int m, int j) -> float { return hs[m * DV + j]; };     // h[m][j]
+    auto DHs = [&](int m, int j) -> float { return dhs[m * DV + j]; };   // dh'[m][j]
     float* scr = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);
     float* U = scr;                    // [64, DV]
     float* dU = U + kC * DV;           // [64, DV]
@@ -531,7 +493,7 @@ cudaError_t vlaunch_fwd_t(const Problem& p, cudaStream_t st) {
     const int CH = p.L.max_chunks * p.d.H;
     cudaError_t e = cw_tc_launch(p, /*bwd=*/false, false, st);
     if (e != cudaSuccess) return e;
-    if (p.o && CH > 0) { StageScope t(ST_OUT, st); vout_kernel<IO, DK, DV><<<CH, kThreads, 0, st>>>(p); }
+    if (p.o && CH > 0 && (e = tc_launch_out_channelwise(p, st)) != cudaSuccess) return e;
     return ffma_fallback<IO, DK, DV>(p, false, false, st);
 }
 

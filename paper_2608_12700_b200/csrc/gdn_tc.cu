@@ -1480,6 +1480,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 // steps of one chunk-head while its neighbour is in another step of another one.  The tiles of the next trip are
 // loaded as soon as the last product (or store) that reads their region is done.  Q h and P U are formed token-major
 // (M = 64: a thread owns a token row), so the output tile is staged with 16-byte stores and leaves by TMA.
+// CW: the channel-wise path.  Its preparation kernels leave Q~ = Gam.q, P = tril(Q~ K-^T), W^T, U~^T and the per-chunk
+// states in the workspace as tile images, the decay is inside Q~ and P, so o = scale (Q~ h + P (U~ - W h)): no product
+// Q K^T, no gates, and P U accumulates onto Q~ h.  P arrives in the half of the [Q ; K] tile that K would occupy.
 // ------------------------------------------------------------------------------------------------
 namespace outk {
 constexpr uint32_t QK = 0;                  // [Q rows 0..63 ; K rows 64..127] x 128              32 KB
@@ -1489,10 +1492,12 @@ constexpr uint32_t HH = UTT + 16384;        // h [128][128]; after the first pro
 constexpr uint32_t PT = WT, STG = HH;
 constexpr uint32_t SMEM_BYTES = HH + 32768 + 1024 /* alignment slack */;
 constexpr uint32_t C_P = 0, C_WH = 64, C_QH = 128, C_PU = 0;   // TMEM columns (256 allocated)
-constexpr uint32_t IN_BYTES = 32768 + 16384 + 16384 + 32768;
+constexpr uint32_t PT_CW = QK + 8192;        // channel-wise: P, loaded, in rows 64..127 of the first column block of [Q ; K]
+constexpr uint32_t IN_BYTES = 32768 + 16384 + 16384 + 32768, IN_BYTES_CW = 16384 + 8192 + 16384 + 16384 + 32768;
 static_assert(2 * (SMEM_BYTES + 4096) <= 228 * 1024, "two CTAs per SM");
 }  // namespace outk
 
+template <bool CW>
 __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_constant__ TcParams P) {
     using namespace outk;
     const Problem& p = P.p;
@@ -1519,16 +1524,21 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
     // One mbarrier phase per trip collects all five tiles; they are issued in three pieces, each when its region is free.
     auto load_qk = [&](const ChunkInfo& c, uint32_t phase) {   // thread 0; first piece of a trip: announces the whole trip's bytes
         pending_phase = phase;
-        mbar_expect_tx(&bar_in, IN_BYTES);
+        mbar_expect_tx(&bar_in, CW ? IN_BYTES_CW : IN_BYTES);
         for (int cb = 0; cb < 2; ++cb) {
-            tma_load_2d(sm + QK + cb * 16384, &P.tm_q, c.hd * D + cb * 64, c.tok0, &bar_in);
-            tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, c.hd * D + cb * 64, c.tok0, &bar_in);
+            if (CW) {
+                bulk_load(sm + QK + cb * 16384, p.ws + p.L.img_QKp + (size_t)c.ch * 32768 + cb * 16384, 8192, &bar_in);
+            } else {
+                tma_load_2d(sm + QK + cb * 16384, &P.tm_q, c.hd * D + cb * 64, c.tok0, &bar_in);
+                tma_load_2d(sm + QK + cb * 16384 + 8192, &P.tm_k, c.hd * D + cb * 64, c.tok0, &bar_in);
+            }
         }
         pending = true;
     };
-    auto load_wu = [&](const ChunkInfo& c) {
-        bulk_load(sm + WT, p.ws + p.L.W + (size_t)c.ch * 16384, 16384, &bar_in);
-        bulk_load(sm + UTT, p.ws + p.L.Ut + (size_t)c.ch * 16384, 16384, &bar_in);
+    auto load_wu = [&](const ChunkInfo& c) {   // (channel-wise: and P, whose place the second product reads)
+        bulk_load(sm + WT, p.ws + (CW ? p.L.img_W : p.L.W) + (size_t)c.ch * 16384, 16384, &bar_in);
+        bulk_load(sm + UTT, p.ws + (CW ? p.L.img_U : p.L.Ut) + (size_t)c.ch * 16384, 16384, &bar_in);
+        if (CW) bulk_load(sm + PT_CW, p.ws + p.L.Pm + (size_t)c.ch * 8192, 8192, &bar_in);
     };
     auto load_h = [&](const ChunkInfo& c) { bulk_load(sm + HH, p.ws + p.L.hc + (size_t)c.ch * 32768, 32768, &bar_in); };
     auto fetch_gamma = [&](const ChunkInfo& c) {   // threads 0..63: cumulative log decay of their token
@@ -1537,7 +1547,7 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
     ChunkInfo x;
     chunk_entry(p, x, blockIdx.x);
     if (threadIdx.x == 0) { load_qk(x, 0); load_wu(x); load_h(x); }
-    float gnext = threadIdx.x < kC ? fetch_gamma(x) : 0.f;
+    float gnext = (!CW && threadIdx.x < kC) ? fetch_gamma(x) : 0.f;
     const int f = q4 * 32 + lane;            // feature row of the transposed accumulator (W h)^T
     const int tr = q4 * 16 + (lane & 15);    // token row of the M = 64 accumulators (lanes 0..15 of a quadrant hold them)
     const bool ga = lane < 16;
@@ -1547,7 +1557,7 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
         const bool has_next = item + (int)gridDim.x < n_items;
         ChunkInfo xn = x;
         if (has_next) chunk_entry(p, xn, item + gridDim.x);
-        if (threadIdx.x < kC) {
+        if (!CW && threadIdx.x < kC) {
             gl[threadIdx.x] = gnext * kLog2e;
             Gam[threadIdx.x] = expf(gnext);
         }
@@ -1556,7 +1566,7 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 30);
             if (ok && threadIdx.x == 0) pending = false;
         }
-        if (ok && x.len < kC) {   // ragged tail: rows beyond the sequence belong to somebody else
+        if (!CW && ok && x.len < kC) {   // ragged tail: rows beyond the sequence belong to somebody else (the images are padded)
             zero_tail_rows(sm + QK, 128, 0, x.len);
             zero_tail_rows(sm + QK, 128, 64, x.len);
             fence_async_smem();
@@ -1565,7 +1575,7 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
         // ---- step 1: Q K^T ; (W h)^T ; Q h
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
-            mma_tile<64, 64, 128>(tmem + C_P, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
+            if (!CW) mma_tile<64, 64, 128>(tmem + C_P, op_k_major(sm + QK, 128, 0), op_k_major(sm + QK, 128, 64), false);
             mma_tile<128, 64, 128>(tmem + C_WH, op_mn_major(sm + HH, 128), op_mn_major(sm + WT, 128), false);
             mma_tile<64, 128, 128>(tmem + C_QH, op_k_major(sm + QK, 128, 0), op_mn_major(sm + HH, 128), false);
             mma_commit(&bar_mma);
@@ -1573,7 +1583,7 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
         GDN_WAIT_MMA(31)
         if (ok && has_next) {   // Q and K have been read for the last time
             if (threadIdx.x == 0) load_qk(xn, in_phase ^ 1);
-            if (threadIdx.x < kC) gnext = fetch_gamma(xn);
+            if (!CW && threadIdx.x < kC) gnext = fetch_gamma(xn);
         }
         if (ok) {   // P = tril(Q K^T . D) over W^T (dead), U = U~ - W h in place
             const int i0 = half * 32, j0 = half * 32;
@@ -1581,11 +1591,11 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
             for (int part = 0; part < 4; ++part) {
                 float v[8], u[8], t[8];
                 const int jb = j0 + part * 8, ib = i0 + part * 8;
-                tmem_ld8(tmem + lane_base + C_P + jb, v);
+                if (!CW) tmem_ld8(tmem + lane_base + C_P + jb, v);
                 tmem_ld8(tmem + lane_base + C_WH + ib, t);
                 chunk_load(sm + UTT, 128, f, ib >> 3, u);
                 tmem_wait_ld();
-                if (ga) {
+                if (!CW && ga) {
                     float g8[8];
                     ld8s(gl + jb, g8);
 #pragma unroll
@@ -1603,23 +1613,24 @@ __global__ void __launch_bounds__(kThreads, 2) tc_out_kernel(const __grid_consta
         // ---- step 2: P U (token-major, over the columns of the first two accumulators)
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
-            mma_tile<64, 128, 64>(tmem + C_PU, op_k_major(sm + PT, 64), op_k_major(sm + UTT, 128), false);
+            if (CW) mma_tile<64, 128, 64>(tmem + C_QH, op_k_major(sm + PT_CW, 64), op_k_major(sm + UTT, 128), true);
+            else mma_tile<64, 128, 64>(tmem + C_PU, op_k_major(sm + PT, 64), op_k_major(sm + UTT, 128), false);
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(32)
         if (ok && has_next && threadIdx.x == 0) load_wu(xn);   // P (over W^T) and U^T have been read for the last time
         if (ok) {   // o = scale (Gam . (Q h) + P U): the sixteen low lanes of a warp own a token row and 64 columns each
-            const float coef = sc * Gam[tr];
+            const float coef = CW ? sc : sc * Gam[tr];
 #pragma unroll 1
             for (int part = 0; part < 8; ++part) {
                 const int cb = half * 64 + part * 8;
                 float a[8], b[8];
                 tmem_ld8(tmem + lane_base + C_QH + cb, a);
-                tmem_ld8(tmem + lane_base + C_PU + cb, b);
+                if (!CW) tmem_ld8(tmem + lane_base + C_PU + cb, b);
                 tmem_wait_ld();
                 if (ga) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) b[j] = fmaf(coef, a[j], sc * b[j]);
+                    for (int j = 0; j < 8; ++j) b[j] = CW ? coef * a[j] : fmaf(coef, a[j], sc * b[j]);
                     chunk_store(sm + STG, 64, tr, cb >> 3, b);
                 }
             }
@@ -1759,7 +1770,18 @@ static cudaError_t launch_intra(const TcParams& P, cudaStream_t st) {
 static cudaError_t launch_out(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done;
     const int items = P.p.L.max_chunks * P.p.d.H, ctas = 2 * sm_count();
-    return launch_chunk_kernel(tc_out_kernel, done, outk::SMEM_BYTES, ST_OUT, items < ctas ? items : ctas, kThreads, P, st);
+    return launch_chunk_kernel(tc_out_kernel<false>, done, outk::SMEM_BYTES, ST_OUT, items < ctas ? items : ctas, kThreads, P, st);
+}
+
+// Forward output of the channel-wise path from the tile images its preparation kernels and carries left in the workspace.
+cudaError_t tc_launch_out_channelwise(const Problem& p, cudaStream_t st) {
+    static SmemLimitOnce done;
+    TcParams P{};
+    P.p = p;
+    const uint64_t rows = (uint64_t)p.Ttot, cols = (uint64_t)p.d.H * D;
+    if (!tc::make_tmap_bf16_2d(&P.tm_o, p.o, rows, cols, cols * 2, 64)) return cudaErrorUnknown;
+    const int items = p.L.max_chunks * p.d.H, ctas = 2 * sm_count();
+    return launch_chunk_kernel(tc_out_kernel<true>, done, outk::SMEM_BYTES, ST_OUT, items < ctas ? items : ctas, kThreads, P, st);
 }
 
 // Carries of the channel-wise path: dirs = 0 forward, 1 reverse, 2 both in one launch.  Needs the tile images the
