@@ -16,7 +16,9 @@ struct WsHeader {
     int32_t status;    // device-side gdn_status (0 = ok)
     int32_t n_chunks;  // chunks actually present (<= max_chunks)
     int32_t detail;    // where a bounded wait gave up / offending sequence index
-    int32_t pad[61];
+    int32_t cw_fallback;   // channel-wise calls: 1 if the last call on this workspace was computed by the fall-back kernels
+                           // (then the workspace holds their fp32 data, not tile images); kept across calls
+    int32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == 256, "header size");
 

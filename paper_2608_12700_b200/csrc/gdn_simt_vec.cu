@@ -51,7 +51,9 @@ __device__ __forceinline__ bool vec_go(const Problem& p) {
 }
 __global__ void vec_clear_refusal_kernel(Problem p) {
     WsHeader* hdr = reinterpret_cast<WsHeader*>(p.ws);
-    if (hdr->status == GDN_ERR_DECAY_RANGE) { hdr->status = GDN_OK; hdr->detail = 0; }
+    const bool refused = hdr->status == GDN_ERR_DECAY_RANGE;
+    hdr->cw_fallback = refused ? 1 : 0;   // a backward on this workspace "fresh from the forward" must know whose data it holds
+    if (refused) { hdr->status = GDN_OK; hdr->detail = 0; }
 }
 
 // Chunk-local cumulative log decay per channel into shared memory (pitch DK + 1); rows beyond the sequence repeat the

@@ -55,17 +55,42 @@ constexpr size_t S_DQ = 0, S_DKP = 32768, S_DKM = 65536, S_UDH = 98304, S_DXV = 
 // ------------------------------------------------------------------------------------------------
 // cw_scale
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kT) cw_scale_kernel(Problem p, int with_bwd) {
+// mode 0: the forward's images; 1: those and dO' (closed backward); 2: dO' alone, for a backward on a workspace fresh
+// from the forward (every other image, gam and the factors are still there).  If that forward was computed by the
+// fall-back kernels (its gates were refused; the header remembers), the workspace holds their fp32 data instead: the
+// refusal is raised again and the fall-back sequence computes this call too.
+__global__ void __launch_bounds__(kT) cw_scale_kernel(Problem p, int mode) {
     ChunkCtx x;
     if (!chunk_ctx(p, x)) return;
     extern __shared__ __align__(16) float gam[];   // [64][D + 1]
     __shared__ int bad;
     const int H = p.d.H;
     const size_t base = ((size_t)x.tok0 * H + x.hd) * D, rs = (size_t)H * D;
+    const bool with_bwd = mode != 0;
+    const __nv_bfloat16* op = with_bwd ? reinterpret_cast<const __nv_bfloat16*>(p.dO) + base : nullptr;
+    if (mode == 2) {
+        WsHeader* hdr = reinterpret_cast<WsHeader*>(p.ws);
+        if (hdr->cw_fallback) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) { hdr->status = GDN_ERR_DECAY_RANGE; hdr->detail = -1; }
+            return;
+        }
+        char* iDO = p.ws + p.L.img_dO + (size_t)x.ch * 16384;
+        const float sc = p.d.scale;
+        for (int t = threadIdx.x; t < kC * 16; t += kT) {
+            const int i = t >> 4, ch = t & 15;
+            float o8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o8[j] = 0.f;
+            if (i < x.len) unpack8(*reinterpret_cast<const uint4*>(op + i * rs + ch * 8), o8);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o8[j] *= sc;
+            *reinterpret_cast<uint4*>(iDO + tile_chunk_off(64, i, ch)) = pack8(o8);
+        }
+        return;
+    }
     const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(p.q) + base;
     const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(p.k) + base;
     const __nv_bfloat16* vp = reinterpret_cast<const __nv_bfloat16*>(p.v) + base;
-    const __nv_bfloat16* op = with_bwd ? reinterpret_cast<const __nv_bfloat16*>(p.dO) + base : nullptr;
     if (threadIdx.x == 0) bad = 0;
     __syncthreads();
     if (threadIdx.x < D) {
@@ -150,7 +175,9 @@ constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_E = 256;   // T
 static_assert(TT % 1024 == 0 && SMEM_BYTES <= 225 * 1024, "tile alignment and shared memory budget");
 }  // namespace prepcw
 
-__global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd) {
+// mode 0: the forward's share (P, A, T, W, U~); 1: that and E (closed backward); 2: E alone from the stored P and W^T
+// (backward on a workspace fresh from the forward: no product, inversion or store of the forward is repeated).
+__global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
     using namespace prepcw;
     const int H = p.d.H;
     const WsHeader* hdr = reinterpret_cast<const WsHeader*>(p.ws);
@@ -173,7 +200,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
     float* Af = reinterpret_cast<float*>(sm + XA);
     float* Tf = reinterpret_cast<float*>(sm + XT);
     float* Sf = reinterpret_cast<float*>(sm + SF);
-    const bool bwd = with_bwd != 0;
+    const bool bwd = mode != 0, fresh = mode == 2;
     bool ok = true, pending = false;
     uint32_t mma_phase = 0, in_phase = 0;
 #pragma unroll 1
@@ -181,11 +208,19 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
         const size_t ch = (size_t)item;
         if (threadIdx.x == 0) {
             bulk_wait_read<0>();   // the previous trip's stores have read their tiles
-            mbar_expect_tx(&bar_in, 65536 + (bwd ? 16384 : 0));
-            bulk_load(sm + QKP, p.ws + p.L.img_QKp + ch * 32768, 32768, &bar_in);
-            bulk_load(sm + KM, p.ws + p.L.img_Km + ch * 16384, 16384, &bar_in);
-            bulk_load(sm + VT, p.ws + p.L.img_Vt + ch * 16384, 16384, &bar_in);
-            if (bwd) bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
+            if (fresh) {   // Q~ (the upper halves of the [Q~; K+] image), dO', and the stored P and W^T
+                mbar_expect_tx(&bar_in, 16384 + 16384 + 8192 + 16384);
+                for (int cb = 0; cb < 2; ++cb) bulk_load(sm + QKP + cb * 16384, p.ws + p.L.img_QKp + ch * 32768 + cb * 16384, 8192, &bar_in);
+                bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
+                bulk_load(sm + PT, p.ws + p.L.Pm + ch * 8192, 8192, &bar_in);
+                bulk_load(sm + WT, p.ws + p.L.img_W + ch * 16384, 16384, &bar_in);
+            } else {
+                mbar_expect_tx(&bar_in, 65536 + (bwd ? 16384 : 0));
+                bulk_load(sm + QKP, p.ws + p.L.img_QKp + ch * 32768, 32768, &bar_in);
+                bulk_load(sm + KM, p.ws + p.L.img_Km + ch * 16384, 16384, &bar_in);
+                bulk_load(sm + VT, p.ws + p.L.img_Vt + ch * 16384, 16384, &bar_in);
+                if (bwd) bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
+            }
             pending = true;
         }
         if (ok) {
@@ -194,6 +229,30 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
             if (ok && threadIdx.x == 0) pending = false;
         }
         __syncthreads();
+        if (fresh) {
+            // (P^T dO')^T and Q~^T dO' from the loaded tiles; then E = Q~^T dO' - W^T (P^T dO') as in the closed arm
+            if (ok && threadIdx.x == 0) {
+                tc_fence_after();
+                mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + DOT, 64), op_mn_major(sm + PT, 64), false);
+                mma_tile<128, 128, 64>(tmem + C_E, op_mn_major(sm + QKP, 128, 0), op_mn_major(sm + DOT, 64), false);
+                mma_commit(&bar_mma);
+            }
+            GDN_WAIT_MMA(45)
+            if (ok) {
+                const int f = q4 * 32 + lane, i0 = grp * 32;
+#pragma unroll 1
+                for (int part = 0; part < 4; ++part) {
+                    const int ib = i0 + part * 8;
+                    float v[8];
+                    tmem_ld8(tmem + lane_base + C_PDO + ib, v);
+                    tmem_wait_ld();
+                    chunk_store(sm + PDOT, 128, f, ib >> 3, v);
+                }
+            }
+            tc_fence_before();
+            fence_async_smem();
+            __syncthreads();
+        } else {
         // ---- step 1: S1 = [Q~; K+] K-^T  (rows 0..63: P before masking, rows 64..127: A)
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
@@ -290,6 +349,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
+        }   // (!fresh)
         // ---- step 3: E = Q~^T dO' - W^T (P^T dO')
         if (bwd) {
             if (ok && threadIdx.x == 0) {
@@ -314,10 +374,12 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int with_bwd)
             __syncthreads();
         }
         if (ok && threadIdx.x == 0) {
-            bulk_store(p.ws + p.L.Tm + ch * 8192, sm + TT, 8192);
-            bulk_store(p.ws + p.L.Pm + ch * 8192, sm + PT, 8192);
-            bulk_store(p.ws + p.L.img_W + ch * 16384, sm + WT, 16384);
-            bulk_store(p.ws + p.L.img_U + ch * 16384, sm + UTT, 16384);
+            if (!fresh) {
+                bulk_store(p.ws + p.L.Tm + ch * 8192, sm + TT, 8192);
+                bulk_store(p.ws + p.L.Pm + ch * 8192, sm + PT, 8192);
+                bulk_store(p.ws + p.L.img_W + ch * 16384, sm + WT, 16384);
+                bulk_store(p.ws + p.L.img_U + ch * 16384, sm + UTT, 16384);
+            }
             if (bwd) bulk_store(p.ws + p.L.img_E + ch * 32768, sm + QKP, 32768);
             bulk_commit();
         }
@@ -753,8 +815,9 @@ cudaError_t cw_tc_launch(const Problem& p, bool bwd, bool skip_recompute, cudaSt
         const uint32_t sm_scale = sizeof(float) * kC * (D + 1);
         if ((e = once_scale.ensure(cw_scale_kernel, sm_scale)) != cudaSuccess) return e;
         if ((e = once_prep.ensure(cw_prep_kernel, prepcw::SMEM_BYTES)) != cudaSuccess) return e;
-        { StageScope t(ST_SCALE, st); cw_scale_kernel<<<CH, kT, sm_scale, st>>>(p, bwd ? 1 : 0); }
-        { StageScope t(ST_PREP, st); cw_prep_kernel<<<grid, kT, prepcw::SMEM_BYTES, st>>>(p, bwd ? 1 : 0); }
+        const int mode = bwd ? (skip_recompute ? 2 : 1) : 0;
+        { StageScope t(ST_SCALE, st); cw_scale_kernel<<<CH, kT, sm_scale, st>>>(p, mode); }
+        { StageScope t(ST_PREP, st); cw_prep_kernel<<<grid, kT, prepcw::SMEM_BYTES, st>>>(p, mode); }
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     if (chains > 0 && (e = tc_launch_scan_channelwise(p, bwd ? (skip_recompute ? 1 : 2) : 0, st)) != cudaSuccess) return e;
