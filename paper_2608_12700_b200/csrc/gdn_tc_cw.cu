@@ -96,10 +96,17 @@ __global__ void __launch_bounds__(kT) cw_scale_kernel(Problem p, int mode) {
     if (threadIdx.x < D) {
         const int r = threadIdx.x;
         float s = 0.f, worst = 0.f;
-        for (int i = 0; i < kC; ++i) {
-            if (i < x.len) s += p.gv[base + i * rs + r];
-            gam[i * (D + 1) + r] = s;
-            worst = fmaxf(worst, fabsf(s));
+#pragma unroll 1
+        for (int i0 = 0; i0 < kC; i0 += 16) {   // sixteen loads in flight, then their running sum in token order
+            float g16[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) g16[k] = (i0 + k < x.len) ? p.gv[base + (size_t)(i0 + k) * rs + r] : 0.f;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                s += g16[k];
+                gam[(i0 + k) * (D + 1) + r] = s;
+                worst = fmaxf(worst, fabsf(s));
+            }
         }
         if (!(worst <= kMaxDecay)) bad = 1;   // (also catches a NaN gate: it cannot be scaled apart either)
     }
@@ -122,22 +129,27 @@ __global__ void __launch_bounds__(kT) cw_scale_kernel(Problem p, int mode) {
     const float sc = p.d.scale;
     for (int t = threadIdx.x; t < kC * 16; t += kT) {   // one 16-byte piece (8 features) of one token row
         const int i = t >> 4, ch = t & 15;
-        float q8[8], k8[8], v8[8], o8[8], a[8], b[8], c[8], d8[8];
+        float q8[8], k8[8], v8[8], o8[8], a[8], b[8], c[8], d8[8], b8[8], w8[8];
         const bool live = i < x.len;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { q8[j] = k8[j] = v8[j] = o8[j] = 0.f; }
+        for (int j = 0; j < 8; ++j) { q8[j] = k8[j] = v8[j] = o8[j] = b8[j] = w8[j] = 0.f; }
         if (live) {
             unpack8(*reinterpret_cast<const uint4*>(qp + i * rs + ch * 8), q8);
             unpack8(*reinterpret_cast<const uint4*>(kp + i * rs + ch * 8), k8);
             unpack8(*reinterpret_cast<const uint4*>(vp + i * rs + ch * 8), v8);
             if (with_bwd) unpack8(*reinterpret_cast<const uint4*>(op + i * rs + ch * 8), o8);
+            const float4* bp = reinterpret_cast<const float4*>(p.bv + base + i * rs + ch * 8);
+            const float4* wp = reinterpret_cast<const float4*>(p.wv + base + i * rs + ch * 8);
+            const float4 b0 = bp[0], b1 = bp[1], w0 = wp[0], w1 = wp[1];
+            b8[0] = b0.x; b8[1] = b0.y; b8[2] = b0.z; b8[3] = b0.w; b8[4] = b1.x; b8[5] = b1.y; b8[6] = b1.z; b8[7] = b1.w;
+            w8[0] = w0.x; w8[1] = w0.y; w8[2] = w0.z; w8[3] = w0.w; w8[4] = w1.x; w8[5] = w1.y; w8[6] = w1.z; w8[7] = w1.w;
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int r = ch * 8 + j;
             const float g = gam[i * (D + 1) + r], ge = gam[(kC - 1) * (D + 1) + r];
             const float G = expf(g);
-            const float bb = live ? p.bv[base + i * rs + r] : 0.f, ww = live ? p.wv[base + i * rs + r] : 0.f;
+            const float bb = b8[j], ww = w8[j];
             a[j] = G * q8[j];                 // q~
             b[j] = G * bb * k8[j];            // k+
             c[j] = expf(-g) * k8[j];          // k-
