@@ -748,7 +748,8 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         mbar_expect_tx(&bar_full[stage], 32768 + x_chunk);
         bulk_load(slot + WT, w_base + ch * 16384, 16384, &bar_full[stage]);
         if constexpr (CW) {
-            bulk_load(slot + KT, p.ws + p.L.img_K + ch * 16384, 16384, &bar_full[stage]);
+            // forward: Kb = Gam_e . k- (second product); reverse: k- itself, against the state scaled by Gam_e (below)
+            bulk_load(slot + KT, p.ws + (reverse ? p.L.img_Km : p.L.img_K) + ch * 16384, 16384, &bar_full[stage]);
         } else {
             tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
             tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
@@ -781,6 +782,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
     __syncthreads();
     bool ok = true;
     uint32_t mma_phase = 0;
+    float cw_gam = (CW && nsteps > 0) ? gamma[(((size_t)chunk_of(0) * H + hd) * kC + kC - 1) * D + r] : 0.f;
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
         unsigned char* Ht = sm + HT + (s & 1) * 32768;
@@ -788,11 +790,23 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         const size_t ch = (size_t)c * H + hd;
         unsigned char* ring = sm + stage * STAGE_BYTES;
         const float* ee = ee2[s & 1];
-        // decay of the state over the chunk: a scalar, or (channel-wise) the factor of this thread's state row
-        const float Ge = CW ? expf(gamma[(ch * kC + kC - 1) * D + r]) : (s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]));
-        // state -> bf16: operand of the first product, and the per-chunk state the gradient stage reads
+        // decay of the state over the chunk: a scalar, or (channel-wise) the factor of this thread's state row, whose log
+        // was fetched during the step before (the reverse chain needs it at the top of the step)
+        const float Ge = CW ? expf(cw_gam) : (s < GE_CAP ? ge[s] : expf(gamma[ch * kC + kC - 1]));
+        if (CW && s + 1 < nsteps) cw_gam = gamma[(((size_t)chunk_of(s + 1) * H + hd) * kC + kC - 1) * D + r];
+        // state -> bf16: operand of the first product, and the per-chunk state the gradient stage reads.  Channel-wise,
+        // reverse: stored as dh'' = Diag(Gam_e) dh', the form the gradient stage works with ((Kb dh') = k- dh'').
 #pragma unroll
-        for (int k = 0; k < 8; ++k) *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
+        for (int k = 0; k < 8; ++k) {
+            if constexpr (CW && reverse) {
+                float sc8[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sc8[j] = Ge * st[8 * k + j];
+                *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(sc8);
+            } else {
+                *reinterpret_cast<uint4*>(Ht + tile_chunk_off(128, r, (lc0 >> 3) + k)) = pack8(st + 8 * k);
+            }
+        }
         if (!CW && len < kC) {   // ragged tail: the K rows beyond the sequence belong to somebody else
             ok = mbar_wait_inline(&bar_full[stage], (s / STAGES) & 1);
             if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 12); break; }

@@ -443,7 +443,6 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     if ((int)blockIdx.x >= n_items) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = align1024(smem_raw);
-    __shared__ float GL[D];   // Gam_e per key channel
     __shared__ uint64_t bar_s, bar_a, bar_b, bar_k, bar_q, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -509,36 +508,11 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         const bool has_next = item + (int)gridDim.x < n_items;
         const size_t chn = ch + gridDim.x;
         float* scr = reinterpret_cast<float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * ch);
-        if (threadIdx.x < D)
-            GL[threadIdx.x] = expf(reinterpret_cast<const float*>(p.ws + p.L.gamma)[(ch * kC + kC - 1) * D + threadIdx.x]);
-        if (ok) {
-            ok = mbar_wait(&bar_s, in_phase);
+        if (ok) {   // everything step 1 reads (the reverse carry left dh'' = Diag(Gam_e) dh', the form used here)
+            ok = mbar_wait(&bar_s, in_phase) && mbar_wait(&bar_k, in_phase) && mbar_wait(&bar_b, in_phase) && mbar_wait(&bar_a, in_phase);
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 44);
-            if (ok && threadIdx.x == 0) pend_s = false;
+            if (ok && threadIdx.x == 0) pend_s = pend_k = pend_a = pend_b = false;
         }
-        __syncthreads();
-        {   // dh'' = Diag(Gam_e) dh' in place, and rowdot(dh'', h): two threads per state row, eight 16-byte pieces each
-            const int r = threadIdx.x >> 1, half = threadIdx.x & 1;
-            const float G = GL[r];
-            float hh = 0.f;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                float a[8], b[8];
-                chunk_load(sm + DH, 128, r, half * 8 + k, a);
-                chunk_load(sm + HH, 128, r, half * 8 + k, b);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { a[j] *= G; hh = fmaf(a[j], b[j], hh); }
-                chunk_store(sm + DH, 128, r, half * 8 + k, a);
-            }
-            hh += __shfl_xor_sync(0xffffffffu, hh, 1);
-            if (ok && half == 0) scr[S_HH / 4 + r] = hh;
-        }
-        if (ok) {   // the rest of what step 1 reads
-            ok = mbar_wait(&bar_k, in_phase) && mbar_wait(&bar_b, in_phase) && mbar_wait(&bar_a, in_phase);
-            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 50);
-            if (ok && threadIdx.x == 0) pend_k = pend_a = pend_b = false;
-        }
-        fence_async_smem();
         __syncthreads();
         // ---- step 1: (W h)^T ; (K- dh'')^T ; (P^T dO')^T
         if (ok && threadIdx.x == 0) {
@@ -547,6 +521,20 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_tile<128, 64, 128>(tmem + C_B, op_mn_major(sm + DH, 128), op_k_major(sm + QKM, 128, 64), false);
             mma_tile<128, 64, 64>(tmem + C_PDO, op_mn_major(sm + DOT, 64), op_mn_major(sm + PT, 64), false);
             mma_commit(&bar_mma);
+        }
+        {   // rowdot(dh'', h) for the decay gradient of the chunk end, while the products run: two threads per state row
+            const int r = threadIdx.x >> 1, half = threadIdx.x & 1;
+            float hh = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                float a[8], b[8];
+                chunk_load(sm + DH, 128, r, half * 8 + k, a);
+                chunk_load(sm + HH, 128, r, half * 8 + k, b);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) hh = fmaf(a[j], b[j], hh);
+            }
+            hh += __shfl_xor_sync(0xffffffffu, hh, 1);
+            if (ok && half == 0) scr[S_HH / 4 + r] = hh;
         }
         GDN_WAIT_MMA(45)
         if (ok) {   // U^T = U~^T - (W h)^T ; dU^T = (P^T dO')^T + (K- dh'')^T
