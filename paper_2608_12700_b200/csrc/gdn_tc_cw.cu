@@ -48,9 +48,9 @@ __device__ __forceinline__ bool chunk_ctx(const Problem& p, ChunkCtx& x) {
     return true;
 }
 
-// Per chunk-head scratch between cw_intra and cw_post (fp32): dQ~, dK+, dK-, U dh''^T, dXv [64][128] each,
-// rowdot(dh'', h) [128].
-constexpr size_t S_DQ = 0, S_DKP = 32768, S_DKM = 65536, S_UDH = 98304, S_DXV = 131072, S_HH = 163840, S_BYTES = 164352;
+// Per chunk-head scratch between cw_intra and cw_post (fp32): dQ~, dK+, dK-, dXv [64][128] each, and per key channel
+// rowdot(dh'', h + K-^T U) [128], the chunk-end part of the decay gradient.
+constexpr size_t S_DQ = 0, S_DKP = 32768, S_DKM = 65536, S_DXV = 98304, S_HH = 131072, S_BYTES = 131584;
 
 // ------------------------------------------------------------------------------------------------
 // cw_scale
@@ -431,6 +431,7 @@ constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = UT, DXVT = DUT;   // (dXk 
 //   256..383  dQ~ = dO' h^T + dP K-                 (M = 64)
 //   384..511  dK- = U dh''^T + dP^T Q~ + dA^T K+    (M = 64)
 constexpr uint32_t C_A = 0, C_B = 64, C_PDO = 128, C_KP = 64, C_PP = 192, C_DQ = 256, C_KM = 384;
+constexpr uint32_t C_X = 64;   // K-^T U [128][128] over C_B | C_PDO (read by then), gone before dXk lands on C_KP
 static_assert(SMEM_BYTES <= 220 * 1024, "shared memory budget");
 }  // namespace intracw
 
@@ -445,6 +446,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     unsigned char* sm = align1024(smem_raw);
     __shared__ uint64_t bar_s, bar_a, bar_b, bar_k, bar_q, bar_mma;
     __shared__ uint32_t tmem_slot;
+    __shared__ float end_sum[3][D];   // per key channel: rowdot(dh'', h) and the two halves of rowdot(dh'', K-^T U)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
@@ -534,7 +536,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
                 for (int j = 0; j < 8; ++j) hh = fmaf(a[j], b[j], hh);
             }
             hh += __shfl_xor_sync(0xffffffffu, hh, 1);
-            if (ok && half == 0) scr[S_HH / 4 + r] = hh;
+            if (half == 0) end_sum[0][r] = hh;
         }
         GDN_WAIT_MMA(45)
         if (ok) {   // U^T = U~^T - (W h)^T ; dU^T = (P^T dO')^T + (K- dh'')^T
@@ -564,10 +566,11 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_tile<128, 64, 128>(tmem + C_A, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
             mma_tile<64, 128, 128>(tmem + C_DQ, op_k_major(sm + DOT, 64), op_k_major(sm + HH, 128), false);
             mma_tile<64, 128, 128>(tmem + C_KM, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);
+            // K-^T U: its row dots with dh'' are the part sum_j k-_j . (U dh''^T)_j of the decay gradient of the chunk end
+            mma_tile<128, 128, 64>(tmem + C_X, op_mn_major(sm + QKM, 128, 64), op_k_major(sm + UT, 128), false);
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(46)
-        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time
         if (ok) {
             const int j0 = grp * 32, i0 = grp * 32, c0 = grp * 64;
 #pragma unroll 1
@@ -584,21 +587,23 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
                 }
                 chunk_store(sm + DWT, 128, f, (i0 >> 3) + part, w8);   // (every product that reads dO' is done)
             }
+            float xs = 0.f;   // rowdot(dh'', K-^T U): this thread's state row f, its half of the columns
 #pragma unroll 1
-            for (int part = 0; part < 8; ++part) {   // U dh''^T alone is needed for the decay gradient of the chunk end
-                float v[8];
-                tmem_ld8(tmem + lane_base + C_KM + c0 + part * 8, v);
+            for (int part = 0; part < 8; ++part) {
+                float v[8], d8[8];
+                tmem_ld8(tmem + lane_base + C_X + c0 + part * 8, v);
+                chunk_load(sm + DH, 128, f, (c0 >> 3) + part, d8);
                 tmem_wait_ld();
-                if (ga) {
-                    float* dst = scr + S_UDH / 4 + tr * D + c0 + part * 8;
-                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-                    *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
-                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) xs = fmaf(v[j], d8[j], xs);
             }
+            end_sum[1 + grp][f] = xs;
         }
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
+        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time
+        if (ok && threadIdx.x < D) scr[S_HH / 4 + threadIdx.x] = end_sum[0][threadIdx.x] + end_sum[1][threadIdx.x] + end_sum[2][threadIdx.x];
         // ---- step 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
         if (ok) {
             ok = mbar_wait(&bar_q, in_phase);
@@ -729,12 +734,9 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
     __nv_bfloat16* dvp = reinterpret_cast<__nv_bfloat16*>(p.dv) + base;
     const float* wsG = reinterpret_cast<const float*>(p.ws + p.L.gamma) + (size_t)x.ch * kC * D;
     const float* scr = reinterpret_cast<const float*>(p.ws + p.L.scratch + p.L.scratch_per_ch * x.ch);
-    const float *dQ = scr + S_DQ / 4, *dKp = scr + S_DKP / 4, *dKm = scr + S_DKM / 4, *udh = scr + S_UDH / 4;
+    const float *dQ = scr + S_DQ / 4, *dKp = scr + S_DKP / 4, *dKm = scr + S_DKM / 4;
     const float *dXv = scr + S_DXV / 4, *hh = scr + S_HH / 4;
-    __shared__ __align__(16) float part[8][D];   // per channel: the chunk-end sum, from the eight threads that share the channel
-    // a thread owns four adjacent channels and every eighth token: 16-byte accesses, coalesced rows, and the chunk-end sum
-    // of its tokens on the way
-    float extra[4] = {0.f, 0.f, 0.f, 0.f};
+    // a thread owns four adjacent channels and every eighth token: 16-byte accesses, coalesced rows
     const int r4 = (threadIdx.x & 31) * 4;
 #pragma unroll 2
     for (int i = threadIdx.x >> 5; i < kC; i += kT / 32) {
@@ -742,7 +744,7 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
         const bool live = i < x.len;
         const float4 g4 = *reinterpret_cast<const float4*>(wsG + t), a4 = *reinterpret_cast<const float4*>(dQ + t);
         const float4 p4 = *reinterpret_cast<const float4*>(dKp + t), m4 = *reinterpret_cast<const float4*>(dKm + t);
-        const float4 u4 = *reinterpret_cast<const float4*>(udh + t), x4 = *reinterpret_cast<const float4*>(dXv + t);
+        const float4 x4 = *reinterpret_cast<const float4*>(dXv + t);
         float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f), w4 = b4;
         uint2 qr = make_uint2(0, 0), kr = qr, vr = qr;
         if (live) {
@@ -753,7 +755,7 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
             vr = *reinterpret_cast<const uint2*>(vp + i * rs + r4);
         }
         const float g[4] = {g4.x, g4.y, g4.z, g4.w}, dqt[4] = {a4.x, a4.y, a4.z, a4.w}, dkp4[4] = {p4.x, p4.y, p4.z, p4.w};
-        const float dkm4[4] = {m4.x, m4.y, m4.z, m4.w}, ud[4] = {u4.x, u4.y, u4.z, u4.w}, xv[4] = {x4.x, x4.y, x4.z, x4.w};
+        const float dkm4[4] = {m4.x, m4.y, m4.z, m4.w}, xv[4] = {x4.x, x4.y, x4.z, x4.w};
         const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, ww[4] = {w4.x, w4.y, w4.z, w4.w};
         const float q[4] = {bf16_lo(qr.x), bf16_hi(qr.x), bf16_lo(qr.y), bf16_hi(qr.y)};
         const float k[4] = {bf16_lo(kr.x), bf16_hi(kr.x), bf16_lo(kr.y), bf16_hi(kr.y)};
@@ -768,7 +770,6 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
             dk[j] = fmaf(bb[j], row, col);
             db[j] = k[j] * row;
             dgm[j] = q[j] * dq[j] + k[j] * bb[j] * row - k[j] * col;
-            extra[j] = fmaf(k[j] * iG, ud[j], extra[j]);   // k-_j . (U dh''^T)_j
             dv[j] = ww[j] * xv[j];                    // dv = w . dXv
             dw[j] = v[j] * xv[j];                     // dw = v . dXv
         }
@@ -781,14 +782,11 @@ __global__ void __launch_bounds__(kT) cw_post_kernel(Problem p) {
             *reinterpret_cast<float4*>(p.dwv + base + i * rs + r4) = make_float4(dw[0], dw[1], dw[2], dw[3]);
         }
     }
-    *reinterpret_cast<float4*>(&part[threadIdx.x >> 5][r4]) = make_float4(extra[0], extra[1], extra[2], extra[3]);
     __syncthreads();
-    // the chunk end collects sum_j k-_j . (U dh''^T)_j and rowdot(dh'', h); then dg_j = sum_{i >= j} dgam_i per channel
+    // the chunk end collects rowdot(dh'', h + K-^T U) (from cw_intra); then dg_j = sum_{i >= j} dgam_i per channel
     if (threadIdx.x < D) {
         const int r = threadIdx.x;
         float run = hh[r];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) run += part[w][r];
         for (int i = kC - 1; i >= 0; --i) {
             run += dgam[i * D + r];
             if (i < x.len) p.dgv[base + i * rs + r] = run;
