@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(kT) cw_scale_kernel(Problem p, int mode) {
 // cw_prep
 // ------------------------------------------------------------------------------------------------
 namespace prepcw {
-constexpr uint32_t QKP = 0;                 // [Q~ rows 0..63 ; K+ rows 64..127] x 128; finally the staged E image   32 KB
+constexpr uint32_t QKP = 0;                 // [Q~ rows 0..63 ; K+ rows 64..127] x 128                               32 KB
 constexpr uint32_t KM = 32768;              // K- [64][128]                                     16 KB
 constexpr uint32_t VT = KM + 16384;         // V~ [64][128]                                     16 KB
 constexpr uint32_t DOT = VT + 16384;        // dO' [64][128]                                    16 KB
@@ -182,8 +182,10 @@ constexpr uint32_t PT = TT + 8192;          // P  bf16 [64][64]                 
 constexpr uint32_t WT = PT + 8192;          // W^T  [128][64]                                   16 KB
 constexpr uint32_t UTT = WT + 16384;        // U~^T [128][64]                                   16 KB
 constexpr uint32_t PDOT = UTT + 16384;      // (P^T dO')^T [128][64]                            16 KB
+constexpr uint32_t EST = XA;                // staged E image [128][128] over the fp32 A and T blocks                       32 KB
 constexpr uint32_t SMEM_BYTES = PDOT + 16384 + 1024;
 constexpr uint32_t C_S1 = 0, C_W = 64, C_U = 128, C_PDO = 192, C_E = 256;   // TMEM columns (512 allocated)
+static_assert(EST % 1024 == 0 && EST + 32768 <= SF + 17408, "the E image fits over the inversion's scratch");
 static_assert(TT % 1024 == 0 && SMEM_BYTES <= 225 * 1024, "tile alignment and shared memory budget");
 }  // namespace prepcw
 
@@ -214,27 +216,39 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
     float* Sf = reinterpret_cast<float*>(sm + SF);
     const bool bwd = mode != 0, fresh = mode == 2;
     bool ok = true, pending = false;
-    uint32_t mma_phase = 0, in_phase = 0;
+    uint32_t mma_phase = 0, in_phase = 0, pending_phase = 0;   // (pending_phase: the phase of bar_in the loads in flight belong to)
+    // The tiles of a trip arrive in two pieces on one mbarrier phase, each issued during the trip before as soon as the
+    // last product that reads its region is done (E is staged over the inversion's scratch, never over an input tile):
+    //   closed / forward:  a = K-                     after step 1      b = [Q~; K+], V~, dO'     after step 2
+    //   fresh workspace:   a = Q~, dO', stored P      after its first products      b = stored W^T   after step 3
+    auto load_a = [&](size_t c, uint32_t phase) {   // thread 0; the first piece announces the whole trip's bytes
+        pending_phase = phase;
+        pending = true;
+        if (fresh) {
+            mbar_expect_tx(&bar_in, 16384 + 16384 + 8192 + 16384);
+            for (int cb = 0; cb < 2; ++cb) bulk_load(sm + QKP + cb * 16384, p.ws + p.L.img_QKp + c * 32768 + cb * 16384, 8192, &bar_in);
+            bulk_load(sm + DOT, p.ws + p.L.img_dO + c * 16384, 16384, &bar_in);
+            bulk_load(sm + PT, p.ws + p.L.Pm + c * 8192, 8192, &bar_in);
+        } else {
+            mbar_expect_tx(&bar_in, 65536 + (bwd ? 16384 : 0));
+            bulk_load(sm + KM, p.ws + p.L.img_Km + c * 16384, 16384, &bar_in);
+        }
+    };
+    auto load_b = [&](size_t c) {
+        if (fresh) {
+            bulk_load(sm + WT, p.ws + p.L.img_W + c * 16384, 16384, &bar_in);
+        } else {
+            bulk_load(sm + QKP, p.ws + p.L.img_QKp + c * 32768, 32768, &bar_in);
+            bulk_load(sm + VT, p.ws + p.L.img_Vt + c * 16384, 16384, &bar_in);
+            if (bwd) bulk_load(sm + DOT, p.ws + p.L.img_dO + c * 16384, 16384, &bar_in);
+        }
+    };
+    if (threadIdx.x == 0) { load_a(blockIdx.x, 0); load_b(blockIdx.x); }
 #pragma unroll 1
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, in_phase ^= 1) {
-        const size_t ch = (size_t)item;
-        if (threadIdx.x == 0) {
-            bulk_wait_read<0>();   // the previous trip's stores have read their tiles
-            if (fresh) {   // Q~ (the upper halves of the [Q~; K+] image), dO', and the stored P and W^T
-                mbar_expect_tx(&bar_in, 16384 + 16384 + 8192 + 16384);
-                for (int cb = 0; cb < 2; ++cb) bulk_load(sm + QKP + cb * 16384, p.ws + p.L.img_QKp + ch * 32768 + cb * 16384, 8192, &bar_in);
-                bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
-                bulk_load(sm + PT, p.ws + p.L.Pm + ch * 8192, 8192, &bar_in);
-                bulk_load(sm + WT, p.ws + p.L.img_W + ch * 16384, 16384, &bar_in);
-            } else {
-                mbar_expect_tx(&bar_in, 65536 + (bwd ? 16384 : 0));
-                bulk_load(sm + QKP, p.ws + p.L.img_QKp + ch * 32768, 32768, &bar_in);
-                bulk_load(sm + KM, p.ws + p.L.img_Km + ch * 16384, 16384, &bar_in);
-                bulk_load(sm + VT, p.ws + p.L.img_Vt + ch * 16384, 16384, &bar_in);
-                if (bwd) bulk_load(sm + DOT, p.ws + p.L.img_dO + ch * 16384, 16384, &bar_in);
-            }
-            pending = true;
-        }
+        const size_t ch = (size_t)item, chn = ch + gridDim.x;
+        const bool has_next = item + (int)gridDim.x < n_items;
+        if (threadIdx.x == 0) bulk_wait_read<0>();   // the previous trip's stores have read their tiles (rewritten from here on)
         if (ok) {
             ok = mbar_wait(&bar_in, in_phase);
             if (!ok && threadIdx.x == 0) report_timeout(p.ws, 40);
@@ -250,6 +264,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
                 mma_commit(&bar_mma);
             }
             GDN_WAIT_MMA(45)
+            if (ok && has_next && threadIdx.x == 0) load_a(chn, in_phase ^ 1);   // Q~, dO' and P have been read for the last time
             if (ok) {
                 const int f = q4 * 32 + lane, i0 = grp * 32;
 #pragma unroll 1
@@ -272,6 +287,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(41)
+        if (ok && has_next && threadIdx.x == 0) load_a(chn, in_phase ^ 1);   // K- has been read for the last time
         if (ok) {
             const int i = (q4 & 1) * 32 + lane, j0 = grp * 32;
 #pragma unroll 1
@@ -339,6 +355,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(42)
+        if (ok && has_next && threadIdx.x == 0) load_b(chn);   // [Q~; K+], V~ and dO' have been read for the last time
         if (ok) {
             const int f = q4 * 32 + lane, i0 = grp * 32;
 #pragma unroll 1
@@ -370,7 +387,8 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
                 mma_commit(&bar_mma);
             }
             GDN_WAIT_MMA(43)
-            if (ok) {   // E -> bf16 tile image over [Q~; K+], which no product reads any more
+            if (ok && fresh && has_next && threadIdx.x == 0) load_b(chn);   // W^T has been read for the last time
+            if (ok) {   // E -> bf16 tile image, staged over the scratch of the inversion (dead since T was converted)
                 const int r = q4 * 32 + lane, c0 = grp * 64;
 #pragma unroll 1
                 for (int part = 0; part < 8; ++part) {
@@ -378,7 +396,7 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
                     float v[8];
                     tmem_ld8(tmem + lane_base + C_E + cb, v);
                     tmem_wait_ld();
-                    chunk_store(sm + QKP, 128, r, cb >> 3, v);
+                    chunk_store(sm + EST, 128, r, cb >> 3, v);
                 }
             }
             tc_fence_before();
@@ -392,14 +410,14 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
                 bulk_store(p.ws + p.L.img_W + ch * 16384, sm + WT, 16384);
                 bulk_store(p.ws + p.L.img_U + ch * 16384, sm + UTT, 16384);
             }
-            if (bwd) bulk_store(p.ws + p.L.img_E + ch * 32768, sm + QKP, 32768);
+            if (bwd) bulk_store(p.ws + p.L.img_E + ch * 32768, sm + EST, 32768);
             bulk_commit();
         }
         if (!ok) break;
     }
     if (threadIdx.x == 0) {
         bulk_wait_read<0>();
-        if (pending) (void)mbar_wait(&bar_in, in_phase);   // after a timeout a load may still be in flight
+        if (pending) (void)mbar_wait(&bar_in, pending_phase);   // after a timeout a load may still be in flight
     }
     tc_fence_before();
     __syncthreads();
