@@ -583,10 +583,12 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_tile<64, 64, 128>(tmem + C_PP, op_k_major(sm + DOT, 64), op_mn_major(sm + UT, 128), false);
             mma_tile<128, 64, 128>(tmem + C_A, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
             mma_tile<64, 128, 128>(tmem + C_DQ, op_k_major(sm + DOT, 64), op_k_major(sm + HH, 128), false);
-            mma_tile<64, 128, 128>(tmem + C_KM, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);
             // K-^T U: its row dots with dh'' are the part sum_j k-_j . (U dh''^T)_j of the decay gradient of the chunk end
             mma_tile<128, 128, 64>(tmem + C_X, op_mn_major(sm + QKM, 128, 64), op_k_major(sm + UT, 128), false);
             mma_commit(&bar_mma);
+            // U dh''^T is only accumulated upon: it runs under the readout (its operands stay untouched until step 3's
+            // products, whose commit covers it, are done)
+            mma_tile<64, 128, 128>(tmem + C_KM, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);
         }
         GDN_WAIT_MMA(46)
         if (ok) {
@@ -620,7 +622,6 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time
         if (ok && threadIdx.x < D) scr[S_HH / 4 + threadIdx.x] = end_sum[0][threadIdx.x] + end_sum[1][threadIdx.x] + end_sum[2][threadIdx.x];
         // ---- step 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
         if (ok) {
@@ -632,12 +633,13 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             tc_fence_after();
             mma_tile<64, 128, 64>(tmem + C_KP, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);
             mma_tile<128, 64, 64>(tmem + C_A, op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), false);
+            mma_commit(&bar_mma);
+            // the two accumulations onto dQ~ and dK- run under the readout (covered by step 4's commit)
             mma_tile<64, 128, 64>(tmem + C_DQ, op_k_major(sm + DP, 64), op_mn_major(sm + QKM, 128, 64), true);
             mma_tile<64, 128, 64>(tmem + C_KM, op_mn_major(sm + DP, 64), op_mn_major(sm + QKM, 128, 0), true);
-            mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(47)
-        if (ok && has_next && threadIdx.x == 0) load_a(chn);   // dW^T (over dO') and dP (over P) have been read
+        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time (U dh''^T is done)
         if (ok) {
             const int i0 = grp * 32, c0 = grp * 64;
 #pragma unroll 1
@@ -669,7 +671,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_commit(&bar_mma);
         }
         GDN_WAIT_MMA(48)
-        if (ok && has_next && threadIdx.x == 0) load_b(chn);   // W^T and U~^T have been read for the last time
+        if (ok && has_next && threadIdx.x == 0) { load_a(chn); load_b(chn); }   // dW^T (over dO'), dP (over P), W^T, U~^T: all read
         if (ok) {   // dA = -stril(.)
             const int j0 = grp * 32;
 #pragma unroll 1
