@@ -379,8 +379,14 @@ def time_other_configs(args, peaks, barrier, stream, dev):
     torch.cuda.synchronize()
     stg = {k: round(v[0] / v[1], 5) for k, v in binding.gdn_stage_timing_read().items() if v[1] > 0}
     binding.gdn_stage_timing_enable(False)
+    # the same backward on a workspace filled by the forward call, and that forward alone
+    fwd_ms = time_steps(lambda: runner.run_fwd_channelwise(buf), 10, barrier, stream) / 10
+    runner.run_fwd_channelwise(buf)
+    fresh_ms = time_steps(lambda: runner.run_bwd_channelwise(buf, fresh=1), 10, barrier, stream) / 10
     out[wl.name] = {"ms_per_step": ms, "tokens_per_s": wl.tokens / (ms * 1e-3), "steps": 10, "tokens": wl.tokens,
-                    "kernel_path": "tcgen05_bf16_channelwise", "entry_point": "gdn_bwd_channelwise", "stage_ms_per_launch": stg}
+                    "kernel_path": binding.gdn_kernel_path_channelwise(buf.desc), "entry_point": "gdn_bwd_channelwise",
+                    "stage_ms_per_launch": stg,
+                    "save_forward_arm": {"ms_per_step": fresh_ms, "gdn_fwd_recompute_channelwise_ms": fwd_ms}}
     del buf, wl
     torch.cuda.empty_cache()
     return out
