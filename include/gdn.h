@@ -157,11 +157,12 @@ const char* gdn_status_string(gdn_status s);
 /* Name of the kernel family a descriptor dispatches to ("simt_f32", "simt_bf16", "tcgen05_bf16",
  * "tcgen05_bf16_scalar_gate", "tcgen05_bf16_padded": bf16 shapes with one or both head dimensions at 64 that have no
  * kernels of their own, zero-padded onto the d = 128 tensor-core kernels inside the workspace),
- * or NULL for an unsupported descriptor.  Diagnostic only. */
+ * or NULL for an unsupported descriptor.  Diagnostic only (the paper has no counterpart). */
 const char* gdn_kernel_path(const gdn_desc* desc);
 /* The same for the channel-wise calls: "tcgen05_bf16_channelwise" (bf16, d_k = d_v = 128),
  * "tcgen05_bf16_channelwise_padded" (bf16, a head dimension of 64: zero-padded onto the former inside the workspace),
- * "simt_f32_channelwise", "simt_bf16_channelwise" (the latter only under gdn_debug_force_family(1)). */
+ * "simt_f32_channelwise", "simt_bf16_channelwise" (the latter only under gdn_debug_force_family(1)).  Diagnostic only
+ * (the paper has no counterpart); gdn_debug_force_family(1) also pins the channel-wise calls to their FFMA kernels. */
 const char* gdn_kernel_path_channelwise(const gdn_desc* desc);
 
 /* ---- backward without a caller-provided workspace (the paper has no counterpart) ----------------
