@@ -691,13 +691,24 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_kernel(const __grid_const
 // ------------------------------------------------------------------------------------------------
 namespace scanlr {
 constexpr int GE_CAP = 2048;
-constexpr int STAGES = 2;
-constexpr uint32_t WT = 0, KT = 16384, XT = 32768, STAGE_BYTES = 65536;   // ring slot: W^T | K | U~^T (16 KB) or E (32 KB)
-constexpr uint32_t HT = STAGES * STAGE_BYTES;      // two bf16 state tiles [128][128]
-constexpr uint32_t GT = HT + 2 * 32768;            // operand of the second product, [128 features][64 tokens]
-constexpr uint32_t SMEM_BYTES = GT + 16384 + 1024;
-constexpr uint32_t C_D1 = 0, C_D2 = 64;            // TMEM columns: first product (64), second product (128)
-static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budget");
+constexpr uint32_t WT = 0, KT = 16384, XT = 32768;   // ring slot: W^T | K | this CTA's part of U~^T (16 KB / S) or E (32 KB / S)
+constexpr uint32_t C_D1 = 0, C_D2 = 64;              // TMEM columns: first product (64), second product (128 / S)
+// S = number of CTAs that share a chain, each carrying 128 / S state columns (the columns of the state evolve
+// independently; W and K are needed whole by every one of them).  S = 2 serves calls that run one direction only with so
+// few chains that half of the SMs would idle (the forward, the backward on a fresh workspace): a step of a half is
+// shorter, and a step's latency is what bounds those launches.
+template <int S> struct Cfg {
+    static constexpr int NS = D / S;                          // state columns of this CTA = rows of the first product
+    static constexpr int NSH = NS / 2;                        // ... of one thread
+    static constexpr int STAGES = S == 1 ? 2 : 3;
+    static constexpr uint32_t STAGE_BYTES = 32768 + 32768 / S;
+    static constexpr uint32_t HT = STAGES * STAGE_BYTES;      // two bf16 state tiles [128][NS]
+    static constexpr uint32_t HT_BYTES = 32768 / S;
+    static constexpr uint32_t GT = HT + 2 * HT_BYTES;         // operand of the second product, [NS features][64 tokens]
+    static constexpr uint32_t SMEM_BYTES = GT + 16384 / S + 1024;
+    static constexpr uint32_t TMEM_COLS = S == 1 ? 256 : 128;
+    static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budget");
+};
 }  // namespace scanlr
 
 // One direction of one chain (the direction is a compile-time constant: the two differ in operands and readouts).
@@ -705,10 +716,13 @@ static_assert(SMEM_BYTES + GE_CAP * 4 + 2048 <= 227 * 1024, "shared memory budge
 // row, i.e. per thread), and the key tile arrives already scaled, Kb_j = exp(gam_e - gam_j) . k_j, as a tile image from the
 // workspace together with images of W^T, U~^T and E (written by the channel-wise preparation kernels), so the readout of the
 // first product applies no per-token factor.
-template <bool reverse, bool CW>
-__device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, float* ge, float (*ee2)[kC], uint64_t* bar_full,
+template <bool reverse, bool CW, int S>
+__device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, int part, float* ge, float (*ee2)[kC], uint64_t* bar_full,
                                               uint64_t& bar_mma, uint32_t& tmem_slot) {
     using namespace scanlr;
+    using C = Cfg<S>;
+    constexpr int NS = C::NS, NSH = C::NSH, STAGES = C::STAGES;
+    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES, HT = C::HT, HT_BYTES = C::HT_BYTES, GT = C::GT;
     const Problem& p = P.p;
     const int H = p.d.H, n = chain / H, hd = chain % H;
     const SeqGeom sg = seq_geom(p, n);
@@ -719,8 +733,12 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, hf = warp >> 2;
     const int r = q4 * 32 + lane;              // TMEM lane of this thread: state row (d_k) or feature of the first product (d_v)
-    const int lc0 = hf * 64;                   // first of its 64 state columns
+    const int lc0 = hf * NSH;                  // first of its NSH state columns inside the CTA's block
     const int tk0 = hf * 32;                   // first of its 32 tokens in the first product
+    // The first product has NS rows.  With 128 of them a thread's TMEM lane is its feature; with 64 (M = 64) the rows sit
+    // on lanes 0..15 of each quadrant and the other lanes of a warp have nothing to read out.
+    const int r1 = S == 1 ? r : q4 * 16 + (lane & 15);
+    const bool act1 = S == 1 || lane < 16;
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
 
     if (threadIdx.x == 0) {
@@ -728,7 +746,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, C::TMEM_COLS); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -736,16 +754,17 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
 
     auto chunk_of = [&](int s) { return reverse ? (c1 - 1 - s) : (c0 + s); };
     const char* w_base = p.ws + (CW ? p.L.img_W : p.L.W);
-    const char* x_base = p.ws + (reverse ? (CW ? p.L.img_E : p.L.E) : (CW ? p.L.img_U : p.L.Ut));
-    const uint32_t x_chunk = reverse ? 32768u : 16384u;
-    char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc);
+    // this CTA's part of the additive image: rows part * NS.. of U~^T [d_v][tokens], column block `part` of E [d_k][d_v]
+    const uint32_t x_chunk = reverse ? 32768u : 16384u, x_bytes = x_chunk / S;
+    const char* x_base = p.ws + (reverse ? (CW ? p.L.img_E : p.L.E) : (CW ? p.L.img_U : p.L.Ut)) + part * x_bytes;
+    char* keep_base = p.ws + (reverse ? p.L.dhn : p.L.hc) + part * HT_BYTES;
     const float* gamma = reinterpret_cast<const float*>(p.ws + p.L.gamma);
     // (L2 prefetches running ahead of the ring, as in tc_scan, made this kernel slower: 79.7 -> 78.5 us without)
     auto fill = [&](int s) {   // thread 32: bring chunk step s into ring slot s % STAGES
         const int stage = s % STAGES, c = chunk_of(s);
         const size_t ch = (size_t)c * H + hd;
         unsigned char* slot = sm + stage * STAGE_BYTES;
-        mbar_expect_tx(&bar_full[stage], 32768 + x_chunk);
+        mbar_expect_tx(&bar_full[stage], 32768 + x_bytes);
         bulk_load(slot + WT, w_base + ch * 16384, 16384, &bar_full[stage]);
         if constexpr (CW) {
             // forward: Kb = Gam_e . k- (second product); reverse: k- itself, against the state scaled by Gam_e (below)
@@ -754,7 +773,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
             tma_load_2d(slot + KT, &P.tm_k, hd * D, sg.chunk_tok0(c), &bar_full[stage]);
             tma_load_2d(slot + KT + 8192, &P.tm_k, hd * D + 64, sg.chunk_tok0(c), &bar_full[stage]);
         }
-        bulk_load(slot + XT, x_base + ch * x_chunk, x_chunk, &bar_full[stage]);
+        bulk_load(slot + XT, x_base + ch * x_chunk, x_bytes, &bar_full[stage]);
     };
     if (threadIdx.x == 32) {
         for (int s = 0; s < STAGES && s < nsteps; ++s) fill(s);
@@ -769,12 +788,12 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         ee2[0][threadIdx.x] = expf(gate_row(0)[kC - 1] - gate_row(0)[threadIdx.x]);
         if (nsteps > 1) { gnext = gate_row(1)[threadIdx.x]; gend_next = gate_row(1)[kC - 1]; }
     }
-    float st[64];
+    float st[NSH];
     {
         const float* init = reverse ? p.dhT : p.h0;
-        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + lc0;
+        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + part * NS + lc0;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
+        for (int k = 0; k < NSH / 4; ++k) {
             float4 v = init ? *reinterpret_cast<const float4*>(init + soff + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
             st[4 * k] = v.x; st[4 * k + 1] = v.y; st[4 * k + 2] = v.z; st[4 * k + 3] = v.w;
         }
@@ -785,7 +804,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
     float cw_gam = (CW && nsteps > 0) ? gamma[(((size_t)chunk_of(0) * H + hd) * kC + kC - 1) * D + r] : 0.f;
 #pragma unroll 1
     for (int s = 0; s < nsteps; ++s) {
-        unsigned char* Ht = sm + HT + (s & 1) * 32768;
+        unsigned char* Ht = sm + HT + (s & 1) * HT_BYTES;
         const int c = chunk_of(s), stage = s % STAGES, len = sg.chunk_len(c);
         const size_t ch = (size_t)c * H + hd;
         unsigned char* ring = sm + stage * STAGE_BYTES;
@@ -797,7 +816,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         // state -> bf16: operand of the first product, and the per-chunk state the gradient stage reads.  Channel-wise,
         // reverse: stored as dh'' = Diag(Gam_e) dh', the form the gradient stage works with ((Kb dh') = k- dh'').
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < NSH / 8; ++k) {
             if constexpr (CW && reverse) {
                 float sc8[8];
 #pragma unroll
@@ -820,11 +839,11 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
                 tc_fence_after();
                 // forward (W h)^T = h^T W^T ; reverse (K dh')^T = dh'^T K^T : [d_v][tokens]
                 const Operand b = reverse ? op_k_major(ring + KT, 64) : op_mn_major(ring + WT, 128);
-                mma_tile<128, 64, 128>(tmem + C_D1, op_mn_major(Ht, 128), b, false);
+                mma_tile<NS, 64, 128>(tmem + C_D1, op_mn_major(Ht, 128), b, false);
             } else {
                 report_timeout(p.ws, 10);
             }
-            bulk_store(keep_base + ch * 32768, Ht, 32768);
+            bulk_store(keep_base + ch * 32768, Ht, HT_BYTES);
             bulk_commit();
             bulk_wait_read<1>();   // (the store of the step before has read its tile: it is rewritten in the next step)
             mma_commit(&bar_mma);
@@ -840,21 +859,25 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             float d1[8], u[8], e8[8];
+            if constexpr (S == 2) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) u[j] = 0.f;
+            }
             tmem_ld8(tmem + lane_base + C_D1 + tk0 + 8 * k, d1);
-            if (!reverse) chunk_load(ring + XT, 128, r, (tk0 >> 3) + k, u);
+            if (!reverse && act1) chunk_load(ring + XT, NS, r1, (tk0 >> 3) + k, u);
             ld8s(ee + tk0 + 8 * k, e8);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 8; ++j) d1[j] = (CW ? 1.f : e8[j]) * (reverse ? d1[j] : (u[j] - d1[j]));
-            chunk_store(sm + GT, 128, r, (tk0 >> 3) + k, d1);
+            if (act1) chunk_store(sm + GT, NS, r1, (tk0 >> 3) + k, d1);
         }
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
         if (threadIdx.x == 0) {
             tc_fence_after();
-            if (reverse) mma_tile<128, 128, 64>(tmem + C_D2, op_k_major(ring + WT, 128), op_k_major(sm + GT, 128), false, /*neg_a=*/true);
-            else mma_tile<128, 128, 64>(tmem + C_D2, op_mn_major(ring + KT, 64), op_k_major(sm + GT, 128), false);
+            if (reverse) mma_tile<128, NS, 64>(tmem + C_D2, op_k_major(ring + WT, 128), op_k_major(sm + GT, NS), false, /*neg_a=*/true);
+            else mma_tile<128, NS, 64>(tmem + C_D2, op_mn_major(ring + KT, 64), op_k_major(sm + GT, NS), false);
             mma_commit(&bar_mma);
         }
         if (!CW && threadIdx.x < kC && s + 1 < nsteps) {   // e_j of the next step, while the product runs
@@ -866,7 +889,7 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
         if (!ok) { if (threadIdx.x == 0) report_timeout(p.ws, 13); break; }
         tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int k = 0; k < NSH / 8; ++k) {
             float d2[8], ad[8];
             tmem_ld8(tmem + lane_base + C_D2 + lc0 + 8 * k, d2);
             if (reverse) chunk_load(ring + XT, 128, r, (lc0 >> 3) + k, ad);
@@ -878,42 +901,48 @@ __device__ __forceinline__ void scan_lr_chain(const TcParams& P, int chain, floa
     }
     float* fin = reverse ? p.dh0 : p.hT;
     if (fin && ok) {
-        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + lc0;
+        const size_t soff = ((size_t)n * H + hd) * D * D + (size_t)r * D + part * NS + lc0;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
+        for (int k = 0; k < NSH / 4; ++k) *reinterpret_cast<float4*>(fin + soff + 4 * k) = make_float4(st[4 * k], st[4 * k + 1], st[4 * k + 2], st[4 * k + 3]);
     }
     if (threadIdx.x == 0) bulk_wait_read<0>();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, 256);
+    if (warp == 0) tmem_dealloc(tmem, C::TMEM_COLS);
 }
 
+// Block index -> (chain, direction, column block): with both directions in one launch the direction is the low bit
+// (S = 1 only); with S = 2 (one direction per launch) the low bit is the column block.
+template <int S>
 __global__ void __launch_bounds__(kThreads, 1) tc_scan_lr_kernel(const __grid_constant__ TcParams P) {
     using namespace scanlr;
     __shared__ float ge[GE_CAP];
     __shared__ __align__(16) float ee2[2][kC];   // e_j of a step, made during the step before it
-    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ uint64_t bar_full[Cfg<S>::STAGES], bar_mma;
     __shared__ uint32_t tmem_slot;
     const int bid = (int)blockIdx.x;
     if (reinterpret_cast<const WsHeader*>(P.p.ws)->status != GDN_OK) return;
-    const int rev = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
-    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
-    if (rev) scan_lr_chain<true, false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
-    else scan_lr_chain<false, false>(P, chain, ge, ee2, bar_full, bar_mma, tmem_slot);
+    const int rev = (S == 1 && P.scan_dirs == 2) ? (bid & 1) : P.scan_dirs;
+    const int chain = (S == 2 || P.scan_dirs == 2) ? (bid >> 1) : bid;
+    const int part = S == 2 ? (bid & 1) : 0;
+    if (rev) scan_lr_chain<true, false, S>(P, chain, part, ge, ee2, bar_full, bar_mma, tmem_slot);
+    else scan_lr_chain<false, false, S>(P, chain, part, ge, ee2, bar_full, bar_mma, tmem_slot);
 }
 
 // The carries of the channel-wise path (per-channel gates, d_k = d_v = 128, bf16 I/O) on the same machinery.
+template <int S>
 __global__ void __launch_bounds__(kThreads, 1) tc_scan_cw_kernel(const __grid_constant__ TcParams P) {
     using namespace scanlr;
     __shared__ __align__(16) float ee2[2][kC];   // (unused: the key tile arrives scaled)
-    __shared__ uint64_t bar_full[STAGES], bar_mma;
+    __shared__ uint64_t bar_full[Cfg<S>::STAGES], bar_mma;
     __shared__ uint32_t tmem_slot;
     const int bid = (int)blockIdx.x;
     if (reinterpret_cast<const WsHeader*>(P.p.ws)->status != GDN_OK) return;
-    const int rev = P.scan_dirs == 2 ? (bid & 1) : P.scan_dirs;
-    const int chain = P.scan_dirs == 2 ? (bid >> 1) : bid;
-    if (rev) scan_lr_chain<true, true>(P, chain, nullptr, ee2, bar_full, bar_mma, tmem_slot);
-    else scan_lr_chain<false, true>(P, chain, nullptr, ee2, bar_full, bar_mma, tmem_slot);
+    const int rev = (S == 1 && P.scan_dirs == 2) ? (bid & 1) : P.scan_dirs;
+    const int chain = (S == 2 || P.scan_dirs == 2) ? (bid >> 1) : bid;
+    const int part = S == 2 ? (bid & 1) : 0;
+    if (rev) scan_lr_chain<true, true, S>(P, chain, part, nullptr, ee2, bar_full, bar_mma, tmem_slot);
+    else scan_lr_chain<false, true, S>(P, chain, part, nullptr, ee2, bar_full, bar_mma, tmem_slot);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1768,8 +1797,13 @@ static cudaError_t launch_scan(const TcParams& P, cudaStream_t st) {
     static SmemLimitOnce done2;
     const int ctas = P.p.d.N * P.p.d.H * (P.scan_dirs == 2 ? 2 : 1);
     if (P.lowrank) {
-        static SmemLimitOnce done_lr;
-        return launch_chunk_kernel(tc_scan_lr_kernel, done_lr, scanlr::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
+        static SmemLimitOnce done_lr, done_lr2;
+        // the reverse carry alone (backward on a fresh workspace) with few chains: two CTAs per chain, each carrying half of
+        // the state columns (measured on 64 chains of 32 chunks: reverse 64 -> 58 us; the forward carry alone became
+        // slower that way, 62 -> 66 us, and keeps one CTA per chain)
+        if (P.scan_dirs == 1 && 2 * ctas <= sm_count())
+            return launch_chunk_kernel(tc_scan_lr_kernel<2>, done_lr2, scanlr::Cfg<2>::SMEM_BYTES, ST_SCANS, 2 * ctas, kThreads, P, st);
+        return launch_chunk_kernel(tc_scan_lr_kernel<1>, done_lr, scanlr::Cfg<1>::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
     }
     // few chains: two CTAs per (chain, direction), each carrying half of the state columns
     if (2 * ctas <= sm_count())
@@ -1807,7 +1841,10 @@ cudaError_t tc_launch_scan_channelwise(const Problem& p, int dirs, cudaStream_t 
     P.scan_dirs = dirs;
     P.lowrank = 1;
     const int ctas = p.d.N * p.d.H * (dirs == 2 ? 2 : 1);
-    return launch_chunk_kernel(tc_scan_cw_kernel, done, scanlr::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
+    static SmemLimitOnce done2;
+    if (dirs != 2 && 2 * ctas <= sm_count())
+        return launch_chunk_kernel(tc_scan_cw_kernel<2>, done2, scanlr::Cfg<2>::SMEM_BYTES, ST_SCANS, 2 * ctas, kThreads, P, st);
+    return launch_chunk_kernel(tc_scan_cw_kernel<1>, done, scanlr::Cfg<1>::SMEM_BYTES, ST_SCANS, ctas, kThreads, P, st);
 }
 
 // A call with no tokens still owes the pass-through of the states.
