@@ -967,17 +967,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_cw_kernel(const __grid_co
 namespace intra {
 constexpr uint32_t QK = 0;                 // [Q ; K] x 128                     32 KB
 constexpr uint32_t VT = 32768;             // V  [64][128]                      16 KB   later staged dv
-constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dW^T [128][64]
+constexpr uint32_t DO = VT + 16384;        // dO [64][128]                      16 KB   later dXv [64][128], then G and Diag(b) G [64][64] each
 constexpr uint32_t WT = DO + 16384;        // W^T  [128][64]                    16 KB
 constexpr uint32_t UTT = WT + 16384;       // U~^T [128][64]                    16 KB
 constexpr uint32_t TT = UTT + 16384;       // T [64][64]                         8 KB
-constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB   later dXk, dXv [64][128] each
+constexpr uint32_t HH = TT + 8192;         // h [128][128]                      32 KB
 constexpr uint32_t DH = HH + 32768;        // dh' [128][128]                    32 KB
 constexpr uint32_t PT = DH + 32768;        // P [64][64]                         8 KB   later dPD
-constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later G and Diag(b) G [64][64] each, then staged dk
+constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     16 KB   later staged dk
 constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dq
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DO, DXK = HH, DXV = HH + 16384, DPD = PT, GT = UT, BGT = UT + 8192;
+constexpr uint32_t DXV = DO, DPD = PT, GT = DO, BGT = DO + 8192;
 // token-major staging of dq (over dU^T, last read by the early products of phase 4), of dv (in place over V: a thread
 // overwrites exactly the chunk it has just read) and of dk (over G, last read by phase 6).  None of these is read by
 // the late products of phase 4 or rewritten within the trip, and of the loads that run ahead only V targets one of
@@ -1003,7 +1003,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     __shared__ __align__(16) float gate_sets[2][5][kC];   // two sets: a trip's gate arrays are written during the trip before
     __shared__ float red[4][kGroups][kC];       // four token-wise partial sums: [which][column group][token]
     __shared__ float dgam[kC], scal[2][kIntraThreads / 32];
-    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_do, bar_ld0, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma, bar_mma2;
+    __shared__ uint64_t bar_k, bar_g1, bar_g2, bar_do, bar_ld0, bar_ldw, bar_ldh, bar_ld1, bar_ld2, bar_st1, bar_st2, bar_kfree, bar_free, bar_mma;
     __shared__ uint32_t tmem_slot;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q4 = warp & 3, grp = warp >> 2;
@@ -1021,9 +1021,9 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
 
     if (threadIdx.x == 0) {
         mbar_init(&bar_k, 1); mbar_init(&bar_g1, 1); mbar_init(&bar_g2, 1); mbar_init(&bar_do, 1);
-        mbar_init(&bar_ld0, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_ld2, 1);
+        mbar_init(&bar_ld0, 1); mbar_init(&bar_ldw, 1); mbar_init(&bar_ldh, 1); mbar_init(&bar_ld1, 1); mbar_init(&bar_ld2, 1);
         mbar_init(&bar_st1, 1); mbar_init(&bar_st2, 1); mbar_init(&bar_kfree, 16); mbar_init(&bar_free, 1);
-        mbar_init(&bar_mma, 1); mbar_init(&bar_mma2, 1);
+        mbar_init(&bar_mma, 1);
         fence_mbar_init();
     }
     if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
@@ -1033,9 +1033,12 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const uint32_t tmem = tmem_slot;
     bool ok = true;
 
-    // The tiles of a trip arrive in three groups, one mbarrier each, loaded during the previous trip:
-    //   g1  Q, U~^T, dh', h, W   once the products of phase 5 are done       needed by phase 1
-    //   g2  dO, T, V             once the products of phase 6 are done       needed from phase 2 on
+    // The tiles of a trip arrive in groups, one mbarrier each, loaded during the previous trip as their regions fall free:
+    //   g1  W, U~^T              once the second readout is done             needed by phase 1
+    //       h, dh', P            once the products of phase 4 are done
+    //       Q                    once the readout of phase 4 is done
+    //   do  dO;  g2  T, V        once the products of phase 5 are done       needed from phase 2 / 3 on
+    //                            (V goes where dv is staged: its store, or the flush of a ragged tail, must have read it)
     //   k   K                    once the last readout holds its K values    needed by phase 1
     constexpr uint32_t K_BYTES = 16384, G1_BYTES = 16384 + 16384 + 32768 + 32768 + 16384 + 8192, G2_BYTES = 8192 + 16384, DO_BYTES = 16384;
     auto load_piece = [&](int piece, const ChunkInfo& c) {
@@ -1073,6 +1076,25 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     prefetch_l2_tma_2d(&P.tm_k, nx.hd * D, nx.tok0);
                     prefetch_l2_tma_2d(&P.tm_k, nx.hd * D + 64, nx.tok0);
                 }
+                // (Early loads not in a CTA's first trip: there every CTA of the grid reaches these points at the same moment,
+                // the loads come as one burst of 25 MB, and the instruction fetches of the last phases, which run for the
+                // first time, queue behind it for microseconds.  The first trip loads at its end instead.)
+                const bool early = item != (int)blockIdx.x;
+                // the second readout is done: W^T and U~^T have been read for the last time
+                if (!(lok = mbar_wait(&bar_ldw, ph))) break;
+                if (has_next && early) {
+                    mbar_expect_tx(&bar_g1, G1_BYTES);   // the first piece of the group announces all of it
+                    pend1 = true;
+                    load_piece(7, nx);
+                    load_piece(4, nx);
+                }
+                // the products of phase 4 are done: h, dh' and dPD (over P) have been read for the last time
+                if (!(lok = mbar_wait(&bar_ldh, ph))) break;
+                if (has_next && early) {
+                    load_piece(6, nx);
+                    load_piece(5, nx);
+                    load_piece(13, nx);
+                }
                 // dq, dv are staged
                 if (!(lok = mbar_wait(&bar_st1, ph))) break;
                 if (full) {
@@ -1082,18 +1104,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     }
                     bulk_commit();
                 }
-                // phase 5 is done
+                // the readout of phase 4 is done too: Q has been read for the last time
                 if (!(lok = mbar_wait(&bar_ld1, ph))) break;
-                // (Not in a CTA's first trip: there every CTA of the grid reaches this point at the same moment, the
-                // loads come as one burst of 25 MB, and the instruction fetches of the last phases, which run for the
-                // first time, queue behind it for microseconds.  The first trip loads at its end instead.)
-                const bool early = item != (int)blockIdx.x;
                 if (has_next && early) {
-                    mbar_expect_tx(&bar_g1, G1_BYTES);
-                    pend1 = true;
-#pragma unroll 1
-                    for (int piece = 2; piece <= 7; ++piece) load_piece(piece, nx);
-                    load_piece(13, nx);
+                    load_piece(2, nx);
+                    load_piece(3, nx);
                 }
                 // phase 6 is done and the last readout holds its K values in registers: K first, the next trip starts with
                 // it; dO, T, V are not needed before its second phase (V goes where dv is staged, so that store must have
@@ -1272,9 +1287,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             chunk_store(sm + DUT, 128, f, ib >> 3, pd);
         }
     }
+    if (ok) {   // T and V, the last tiles of this trip, are needed from phase 3 on
+        ok = mbar_wait(&bar_g2, in_phase);
+        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 31);
+    }
+    if (ok && x.len < kC) zero_tail_rows(sm + VT, 64, 0, x.len, kIntraThreads);
     tc_fence_before();
     fence_async_smem();
     cta_sync();
+    if (threadIdx.x == 32) mbar_arrive(&bar_ldw);   // W^T (read by phase 1) and U~^T (read by the readout) are free
 
     // From here on the accumulators that become gradients are produced token-major (64 token rows x 128 features,
     // M = 64): a thread owns a token row, so row dots are thread-local and rows leave with 16-byte stores.  A 64-row
@@ -1291,17 +1312,14 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     const int cb0 = grp * 32;               // first of this thread's 32 feature columns
     const int j0b = grp * kTG;              // first of its 16 columns in 64-column accumulators
 
-    // ---- phase 3
+    // ---- phase 3: dO U^T and dXv = T^T dU
     if (ok && issuer) {
         tc_fence_after();
         mma_tile<64, 64, 128>(tmem + 0 + LB, op_k_major(sm + DO, 64), op_mn_major(sm + UT, 128), false);           // dO U^T
-        mma_commit(&bar_mma);   // dPD is formed while dW^T is still being multiplied
-        mma_tile<128, 64, 128>(tmem + 256, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
-        // (a barrier of its own: two commits in a row on one mbarrier could complete two of its phases before a waiter
-        // has looked, and a parity wait cannot tell a phase from the one two later)
-        mma_commit(&bar_mma2);
+        mma_tile<64, 128, 64>(tmem + 128 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DUT, 128), false);         // T^T dU
+        mma_commit(&bar_mma);
     }
-    if (has_next && threadIdx.x < kC) make_gates(in_phase ^ 1);   // the next trip's gate arrays, while the product runs
+    if (has_next && threadIdx.x < kC) make_gates(in_phase ^ 1);   // the next trip's gate arrays, while the products run
     // <dh', h> over the whole state, while the products run (both tiles share one format, so offsets pair up)
     float hh = 0.f;
 #pragma unroll 1
@@ -1313,12 +1331,15 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
         for (int k = 0; k < 8; ++k) hh = fmaf(a[k], b[k], hh);
     }
     GDN_WAIT_MMA(23)
-    if (ok && worker) {   // dPD = scale tril(dO U^T) . D  (group B; the accumulator loads are warp-wide instructions)
+    const bool full = x.len == kC;
+    // (addresses of the ragged-tail flushes are formed where they are used: nothing of them lives across the phases)
+    auto grad_rows = [&](void* base) { return reinterpret_cast<__nv_bfloat16*>(base) + ((size_t)x.tok0 * H + x.hd) * D; };
+    if (ok && worker) {   // group B holds both accumulators (the loads are warp-wide instructions)
         float v2[2][8];
         tmem_ld8(tmem + lane_base + 0 + j0b, v2[0]);
         tmem_ld8(tmem + lane_base + 0 + j0b + 8, v2[1]);
         tmem_wait_ld();
-        if (!ga) {
+        if (!ga) {   // dPD = scale tril(dO U^T) . D
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 const int jb = j0b + part * 8;
@@ -1330,110 +1351,78 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                 chunk_store(sm + DPD, 64, tr, jb >> 3, v);
             }
         }
-    }
-    if (ok) {   // dW^T is complete (and with it dO h^T of phase 2, which reads the dO tile that dW^T now overwrites)
-        ok = mbar_wait(&bar_mma2, in_phase);
-        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 29);
-    }
-    tc_fence_after();
-    if (ok && worker) {
-        float w2[2][8];
-        tmem_ld8(tmem + lane_base + 256 + i0, w2[0]);
-        tmem_ld8(tmem + lane_base + 256 + i0 + 8, w2[1]);
-        tmem_wait_ld();
-        chunk_store(sm + DWT, 128, f, i0 >> 3, w2[0]);              // dW^T = -(dU h^T)^T
-        chunk_store(sm + DWT, 128, f, (i0 >> 3) + 1, w2[1]);
-    }
-    if (ok) {   // V and T, the last tiles of this trip, are needed from phase 4 on
-        ok = mbar_wait(&bar_g2, in_phase);
-        if (!ok && threadIdx.x == 0) report_timeout(p.ws, 31);
-    }
-    if (ok && x.len < kC) zero_tail_rows(sm + VT, 64, 0, x.len, kIntraThreads);
-    tc_fence_before();
-    fence_async_smem();
-    cta_sync();
-
-    // ---- phase 4
-    if (ok && issuer) {
-        tc_fence_after();
-        mma_tile<64, 128, 64>(tmem + 128, op_k_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 64), false);           // (dP.D) K
-        mma_tile<64, 128, 64>(tmem + 0 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);            // T^T dW
-        mma_tile<64, 128, 64>(tmem + 128 + LB, op_mn_major(sm + TT, 64), op_k_major(sm + DUT, 128), false);          // T^T dU
-        mma_commit(&bar_mma);   // the two dk^col products are first read after phase 6
-        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
-        mma_tile<64, 128, 128>(tmem + 0, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);                // U dh'^T
-    }
-    GDN_WAIT_MMA(24)
-    const bool full = x.len == kC;
-    // (addresses of the ragged-tail flushes are formed where they are used: nothing of them lives across the phases)
-    auto grad_rows = [&](void* base) { return reinterpret_cast<__nv_bfloat16*>(base) + ((size_t)x.tok0 * H + x.hd) * D; };
-    if (ok && worker) {
-        // The two lane groups hold different quantities but share one instruction stream where they can (a warp runs
-        // both sides of a branch one after the other):
-        //   group A: dq = scale Gam (dO h^T) + (dP.D) K, staged ; acc = <q, dq>
-        //   group B: dXk, dXv -> operand tiles ; acc = <v, dXv> (dw partial) ; dv = w dXv, staged
+        // dXv -> operand tile (over dO, which every product has read) ; <v, dXv> (dw partial) ; dv = w dXv, staged over V
         float acc = 0.f;
-        const float coef = sc * Gam[tr], outscale = ga ? 1.f : gate_sets[in_phase][4][tr];
-        const unsigned char* dot_tile = sm + (ga ? QK : VT);   // q rows (128-row tile) or v rows (64-row tile)
-        unsigned char* stage = sm + (ga ? STG_A : STG_B);
+        const float wg = gate_sets[in_phase][4][tr];
 #pragma unroll
         for (int part = 0; part < 4; ++part) {
             const int cb = cb0 + part * 8;
-            float a[8], b[8], t8[8], xk[8];
-            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: dO h^T
-            tmem_ld8(tmem + lane_base + 0 + cb, xk);      //                B: dXk
-            tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: (dP.D) K    B: dXv
+            float b[8], t8[8];
+            tmem_ld8(tmem + lane_base + 128 + cb, b);
             tmem_wait_ld();
-            unpack8(*reinterpret_cast<const uint4*>(dot_tile + tile_chunk_off(ga ? 128 : 64, tr, cb >> 3)), t8);
             if (!ga) {
-                chunk_store(sm + DXK, 64, tr, cb >> 3, xk);
+                unpack8(*reinterpret_cast<const uint4*>(sm + VT + tile_chunk_off(64, tr, cb >> 3)), t8);
                 chunk_store(sm + DXV, 64, tr, cb >> 3, b);
-            }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float val = ga ? fmaf(coef, a[j], b[j]) : b[j];   // (a select, not a zero coefficient: group B's
-                acc = fmaf(t8[j], val, acc);                            // lanes of `a` hold an unrelated accumulator)
-                b[j] = val * outscale;
+                for (int j = 0; j < 8; ++j) {
+                    acc = fmaf(t8[j], b[j], acc);
+                    b[j] *= wg;
+                }
+                chunk_store(sm + STG_B, 64, tr, cb >> 3, b);
             }
-            chunk_store(stage, 64, tr, cb >> 3, b);
         }
-        red[ga ? 0 : 1][grp][tr] = acc;
+        if (!ga) red[1][grp][tr] = acc;
     }
     tc_fence_before();
     fence_async_smem();
     cta_sync();
 
-    // ---- phase 5
+    // ---- phase 4: dA = -stril(dXv U^T) (= -stril(dXk W^T + dXv U~^T), since dXk = T^T dW = -dXv h^T and U = U~ - W h),
+    // (dP.D) K, dXk = -dXv h^T; under the readout (dP.D)^T Q and U dh'^T
     if (ok && issuer) {
         tc_fence_after();
-        mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
-        mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UTT, 128), true);
-        mma_commit(&bar_mma);
-        mma_commit(&bar_ld1);   // Q, U~^T, dh', h (by now dXk, dXv) have been read for the last time
-        // dXk once more, on the lanes of group A where dk is assembled; first read after phase 6
-        mma_tile<64, 128, 64>(tmem + 128, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);
-    } else if (threadIdx.x == 32) {
-        // staged dq, dv leave through the async proxy (generic global stores would stall the next proxy fence); the
-        // loader issues the stores
-        mbar_arrive(&bar_st1);
+        mma_tile<64, 64, 128>(tmem + 384 + LB, op_k_major(sm + DXV, 64), op_mn_major(sm + UT, 128), false);         // dXv U^T
+        mma_tile<64, 128, 64>(tmem + 128, op_k_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 64), false);          // (dP.D) K
+        mma_tile<64, 128, 128>(tmem + 256 + LB, op_k_major(sm + DXV, 64), op_k_major(sm + HH, 128), false, /*neg_a=*/true);   // dXk
+        mma_commit(&bar_mma);   // the two dk^col products are first read after the last phase
+        mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + DPD, 64), op_mn_major(sm + QK, 128, 0), false);           // (dP.D)^T Q
+        mma_tile<64, 128, 128>(tmem + 0, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);                // U dh'^T
+        mma_commit(&bar_ldh);   // h, dh' and dPD (over P) have been read for the last time
     }
-    if (ok && !full) {   // ragged tail: rows beyond the sequence must not be written
-        flush_rows(sm + STG_A, grad_rows(p.dq), (size_t)H * D, x.len, kIntraThreads);
-        flush_rows(sm + STG_B, grad_rows(p.dv), (size_t)H * D, x.len, kIntraThreads);
-    }
-    GDN_WAIT_MMA(25)
+    GDN_WAIT_MMA(24)
     if (ok && worker) {
+        // group A: dq = scale Gam (dO h^T) + (dP.D) K, staged ; acc = <q, dq>
+        float acc = 0.f;
+        const float coef = sc * Gam[tr];
+#pragma unroll
+        for (int part = 0; part < 4; ++part) {
+            const int cb = cb0 + part * 8;
+            float a[8], b[8], t8[8];
+            tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: dO h^T
+            tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: (dP.D) K
+            tmem_wait_ld();
+            if (ga) {
+                unpack8(*reinterpret_cast<const uint4*>(sm + QK + tile_chunk_off(128, tr, cb >> 3)), t8);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    b[j] = fmaf(coef, a[j], b[j]);
+                    acc = fmaf(t8[j], b[j], acc);
+                }
+                chunk_store(sm + STG_A, 64, tr, cb >> 3, b);
+            }
+        }
+        if (ga) red[0][grp][tr] = acc;
+        // group B: G = dA . D and Diag(b) G (over dXv, which the products above have read)
         float v2[2][8];
         tmem_ld8(tmem + lane_base + 384 + j0b, v2[0]);
         tmem_ld8(tmem + lane_base + 384 + j0b + 8, v2[1]);
         tmem_wait_ld();
+        if (!ga) {
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float (&v)[8] = v2[part];
-            float w[8];
-            const int jb = j0b + part * 8;
-            if (!ga) {   // G = dA . D,  dA = -stril(dXk W^T + dXv U~^T)
-                float g8[8];
+            for (int part = 0; part < 2; ++part) {
+                float (&v)[8] = v2[part];
+                float w[8], g8[8];
+                const int jb = j0b + part * 8;
                 ld8s(gl + jb, g8);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -1448,14 +1437,20 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     tc_fence_before();
     fence_async_smem();
     cta_sync();
+    if (threadIdx.x == 32) mbar_arrive(&bar_st1);   // dq, dv are staged: the loader stores them (async proxy)
+    if (ok && !full) {   // ragged tail: rows beyond the sequence must not be written
+        flush_rows(sm + STG_A, grad_rows(p.dq), (size_t)H * D, x.len, kIntraThreads);
+        flush_rows(sm + STG_B, grad_rows(p.dv), (size_t)H * D, x.len, kIntraThreads);
+    }
 
-    // ---- phase 6
+    // ---- phase 5: G K ; += (Diag(b) G)^T K
     if (ok && issuer) {
         tc_fence_after();
+        mma_commit(&bar_ld1);   // Q has been read for the last time (by (dP.D)^T Q and by the readout before this phase)
         mma_tile<64, 128, 64>(tmem + 384, op_k_major(sm + GT, 64), op_mn_major(sm + QK, 128, 64), false);            // G K
         mma_tile<64, 128, 64>(tmem + 256, op_mn_major(sm + BGT, 64), op_mn_major(sm + QK, 128, 64), true);           // += (bG)^T K
         mma_commit(&bar_mma);
-        mma_commit(&bar_ld2);   // dW^T (over dO) and T have been read for the last time
+        mma_commit(&bar_ld2);   // G (over dXv, over dO) and T have been read for the last time
     }
     GDN_WAIT_MMA(26)
     if (worker) {   // this thread's K values leave shared memory now, so that the next trip's K can be loaded over them
@@ -1475,10 +1470,11 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
             const int cb = cb0 + part * 8;
             float a[8], b[8], c8[8], d8[8], kk[8];
             tmem_ld8(tmem + lane_base + 384 + cb, a);     // A: G K
-            tmem_ld8(tmem + lane_base + 128 + cb, b);     // A: dXk
-            tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: (dP.D)^T Q + (bG)^T K
+            tmem_ld8(tmem + lane_base + 256 + cb, c8);    // A: (dP.D)^T Q + (bG)^T K      B: dXk
             tmem_ld8(tmem + lane_base + 0 + cb, d8);      // A: U dh'^T
             tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) b[j] = __shfl_down_sync(0xffffffffu, c8[j], 16);   // dXk of this token row comes over from group B
             if (ga) {
                 unpack8(kraw[part], kk);
 #pragma unroll
