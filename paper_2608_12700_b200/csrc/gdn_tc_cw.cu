@@ -430,21 +430,21 @@ __global__ void __launch_bounds__(kT, 1) cw_prep_kernel(Problem p, int mode) {
 namespace intracw {
 constexpr uint32_t QKM = 0;                 // [Q~ rows 0..63 ; K- rows 64..127] x 128         32 KB
 constexpr uint32_t KP = 32768;              // K+ [64][128]                                     16 KB
-constexpr uint32_t DOT = KP + 16384;        // dO' [64][128]; later dW^T [128][64]              16 KB
+constexpr uint32_t DOT = KP + 16384;        // dO' [64][128]                                    16 KB
 constexpr uint32_t WT = DOT + 16384;        // W^T  [128][64]                                   16 KB
 constexpr uint32_t UTT = WT + 16384;        // U~^T [128][64]                                   16 KB
 constexpr uint32_t TT = UTT + 16384;        // T [64][64]; later dA                              8 KB
 constexpr uint32_t PT = TT + 8192;          // P [64][64]; later dP                              8 KB
 constexpr uint32_t HH = PT + 8192;          // h [128][128]                                     32 KB
 constexpr uint32_t DH = HH + 32768;         // dh'' = Diag(Gam_e) dh' [128][128]                32 KB
-constexpr uint32_t UT = DH + 32768;         // U^T  [128][64]; later dXk [64][128]              16 KB
+constexpr uint32_t UT = DH + 32768;         // U^T  [128][64]                                   16 KB
 constexpr uint32_t DUT = UT + 16384;        // dU^T [128][64]; later dXv^T [128][64]            16 KB
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
-constexpr uint32_t DWT = DOT, DA = TT, DP = PT, DXK = UT, DXVT = DUT;   // (dXk over U^T, dXv^T over dU^T: the state tiles are free after step 2)
+constexpr uint32_t DA = TT, DP = PT, DXVT = DUT;   // (dA over T, dP over P, dXv^T over dU^T, each after its last reader)
 // TMEM columns (512 allocated, fixed offsets).  Accumulators with features on the lanes use all 128 lanes (M = 128);
 // token-major ones (M = 64) occupy lanes 0..15 of each lane quadrant.
-//   0..63     (W h)^T  -> dW^T -> dXv^T            (M = 128)
-//   64..191   (K- dh'')^T | (P^T dO')^T (M = 128) -> dK+ = dXk + dA K-   (M = 64, 128 columns)
+//   0..63     (W h)^T  -> dXv^T                    (M = 128)
+//   64..191   (K- dh'')^T | (P^T dO')^T (M = 128) -> K-^T U (M = 128) -> dK+ = dXk + dA K-   (M = 64, 128 columns)
 //   192..255  dP -> dA                              (M = 64)
 //   256..383  dQ~ = dO' h^T + dP K-                 (M = 64)
 //   384..511  dK- = U dh''^T + dP^T Q~ + dA^T K+    (M = 64)
@@ -485,9 +485,9 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
     uint32_t mma_phase = 0, in_phase = 0;
     // The tiles of a trip arrive in five groups, each loaded during the previous trip as soon as the last product that
     // reads its region is done (look-ahead without a second buffer):
-    //   s  h, dh'          after step 2      k  K-               after step 5
-    //   a  dO', P          after step 3      q  Q~, K+, T        after step 5 (needed from step 3 on)
-    //   b  W^T, U~^T       after step 4
+    //   b  W^T, U~^T       after the first readout       s  h, dh''          after step 3
+    //   a  dO'             after step 2                  k  K-               after step 4
+    //      P               after step 3                  q  Q~, K+, T        after step 4 (needed from step 2 on)
     bool pend_s = false, pend_a = false, pend_b = false, pend_k = false, pend_q = false;   // thread 0
     auto load_s = [&](size_t c) {
         mbar_expect_tx(&bar_s, 65536);
@@ -577,11 +577,17 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- step 2: dO' U^T ; dW^T = -(dU h^T)^T ; dO' h^T ; U dh''^T
+        if (ok && has_next && threadIdx.x == 0) load_b(chn);   // W^T (step 1) and U~^T (the readout) have been read for the last time
+        // ---- step 2: dP = dO' U^T ; dXv^T = dU^T T ; dO' h^T ; K-^T U ; under the readout U dh''^T
+        if (ok) {
+            ok = mbar_wait(&bar_q, in_phase);   // T (and Q~, K+, needed from step 3 on)
+            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 51);
+            if (ok && threadIdx.x == 0) pend_q = false;
+        }
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 64, 128>(tmem + C_PP, op_k_major(sm + DOT, 64), op_mn_major(sm + UT, 128), false);
-            mma_tile<128, 64, 128>(tmem + C_A, op_k_major(sm + HH, 128), op_mn_major(sm + DUT, 128), false, /*neg_a=*/true);
+            mma_tile<128, 64, 64>(tmem + C_A, op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), false);
             mma_tile<64, 128, 128>(tmem + C_DQ, op_k_major(sm + DOT, 64), op_k_major(sm + HH, 128), false);
             // K-^T U: its row dots with dh'' are the part sum_j k-_j . (U dh''^T)_j of the decay gradient of the chunk end
             mma_tile<128, 128, 64>(tmem + C_X, op_mn_major(sm + QKM, 128, 64), op_k_major(sm + UT, 128), false);
@@ -591,13 +597,19 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
             mma_tile<64, 128, 128>(tmem + C_KM, op_mn_major(sm + UT, 128), op_k_major(sm + DH, 128), false);
         }
         GDN_WAIT_MMA(46)
+        if (ok && has_next && threadIdx.x == 0) {   // dO' has been read for the last time; P (by then dP) follows after step 3
+            mbar_expect_tx(&bar_a, 24576);
+            bulk_load(sm + DOT, p.ws + p.L.img_dO + chn * 16384, 16384, &bar_a);
+            pend_a = true;
+        }
         if (ok) {
             const int j0 = grp * 32, i0 = grp * 32, c0 = grp * 64;
 #pragma unroll 1
             for (int part = 0; part < 4; ++part) {
-                float v[8], w8[8];
+                float v[8], x8[8];
+                const int ib = i0 + part * 8;
                 tmem_ld8(tmem + lane_base + C_PP + j0 + part * 8, v);     // dP rows on lanes 0..15
-                tmem_ld8(tmem + lane_base + C_A + i0 + part * 8, w8);     // dW^T, all lanes
+                tmem_ld8(tmem + lane_base + C_A + ib, x8);                // dXv^T, all lanes
                 tmem_wait_ld();
                 if (ga) {   // dP = tril(dO' U^T)
                     const int jb = j0 + part * 8;
@@ -605,7 +617,10 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
                     for (int j = 0; j < 8; ++j) v[j] = (jb + j <= tr) ? v[j] : 0.f;
                     chunk_store(sm + DP, 64, tr, jb >> 3, v);
                 }
-                chunk_store(sm + DWT, 128, f, (i0 >> 3) + part, w8);   // (every product that reads dO' is done)
+                // dXv^T: operand tile (over dU^T, which its product has read) and, in fp32, the input of dv and dw
+                chunk_store(sm + DXVT, 128, f, ib >> 3, x8);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) scr[S_DXV / 4 + (ib + j) * D + f] = x8[j];   // token-major: a warp writes 128 contiguous bytes
             }
             float xs = 0.f;   // rowdot(dh'', K-^T U): this thread's state row f, its half of the columns
 #pragma unroll 1
@@ -623,56 +638,22 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         fence_async_smem();
         __syncthreads();
         if (ok && threadIdx.x < D) scr[S_HH / 4 + threadIdx.x] = end_sum[0][threadIdx.x] + end_sum[1][threadIdx.x] + end_sum[2][threadIdx.x];
-        // ---- step 3 (K#2, the two applies): dXk = T^T dW ; dXv^T = dU^T T ; and dQ~ += dP K- ; dK- += dP^T Q~
-        if (ok) {
-            ok = mbar_wait(&bar_q, in_phase);
-            if (!ok && threadIdx.x == 0) report_timeout(p.ws, 51);
-            if (ok && threadIdx.x == 0) pend_q = false;
-        }
+        // ---- step 3 (K#2): dA = -stril(dXv U^T) (= -stril(dXk W^T + dXv U~^T): dXk = T^T dW = -dXv h^T, U = U~ - W h) ;
+        // dK+ = dXk = -dXv h^T ; dQ~ += dP K- ; dK- += dP^T Q~
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
-            mma_tile<64, 128, 64>(tmem + C_KP, op_mn_major(sm + TT, 64), op_k_major(sm + DWT, 128), false);
-            mma_tile<128, 64, 64>(tmem + C_A, op_k_major(sm + DUT, 128), op_mn_major(sm + TT, 64), false);
-            mma_commit(&bar_mma);
-            // the two accumulations onto dQ~ and dK- run under the readout (covered by step 4's commit)
+            mma_tile<64, 64, 128>(tmem + C_PP, op_mn_major(sm + DXVT, 128), op_mn_major(sm + UT, 128), false);
+            mma_tile<64, 128, 128>(tmem + C_KP, op_mn_major(sm + DXVT, 128), op_k_major(sm + HH, 128), false, /*neg_a=*/true);
             mma_tile<64, 128, 64>(tmem + C_DQ, op_k_major(sm + DP, 64), op_mn_major(sm + QKM, 128, 64), true);
             mma_tile<64, 128, 64>(tmem + C_KM, op_mn_major(sm + DP, 64), op_mn_major(sm + QKM, 128, 0), true);
-        }
-        GDN_WAIT_MMA(47)
-        if (ok && has_next && threadIdx.x == 0) load_s(chn);   // h and dh'' have been read for the last time (U dh''^T is done)
-        if (ok) {
-            const int i0 = grp * 32, c0 = grp * 64;
-#pragma unroll 1
-            for (int part = 0; part < 4; ++part) {   // dXv^T: operand tile and, in fp32, the input of dv and dw
-                const int ib = i0 + part * 8;
-                float v[8];
-                tmem_ld8(tmem + lane_base + C_A + ib, v);
-                tmem_wait_ld();
-                chunk_store(sm + DXVT, 128, f, ib >> 3, v);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) scr[S_DXV / 4 + (ib + j) * D + f] = v[j];   // token-major: a warp writes 128 contiguous bytes
-            }
-#pragma unroll 1
-            for (int part = 0; part < 8; ++part) {   // dXk: operand tile (the accumulator goes on collecting dK+)
-                float v[8];
-                tmem_ld8(tmem + lane_base + C_KP + c0 + part * 8, v);
-                tmem_wait_ld();
-                if (ga) chunk_store(sm + DXK, 64, tr, (c0 >> 3) + part, v);
-            }
-        }
-        tc_fence_before();
-        fence_async_smem();
-        __syncthreads();
-        // ---- step 4 (K#2, the sandwich): dXk W^T + dXv U~^T
-        if (ok && threadIdx.x == 0) {
-            tc_fence_after();
-            mma_tile<64, 64, 128>(tmem + C_PP, op_k_major(sm + DXK, 64), op_mn_major(sm + WT, 128), false);
-            mma_tile<64, 64, 128>(tmem + C_PP, op_mn_major(sm + DXVT, 128), op_mn_major(sm + UTT, 128), true);
             mma_commit(&bar_mma);
         }
-        GDN_WAIT_MMA(48)
-        if (ok && has_next && threadIdx.x == 0) { load_a(chn); load_b(chn); }   // dW^T (over dO'), dP (over P), W^T, U~^T: all read
-        if (ok) {   // dA = -stril(.)
+        GDN_WAIT_MMA(47)
+        if (ok && has_next && threadIdx.x == 0) {   // h, dh'' (U dh''^T is done too) and dP (over P) have been read for the last time
+            load_s(chn);
+            bulk_load(sm + PT, p.ws + p.L.Pm + chn * 8192, 8192, &bar_a);   // (the second piece of group a)
+        }
+        if (ok) {   // dA = -stril(.)  (over T, which step 2 has read)
             const int j0 = grp * 32;
 #pragma unroll 1
             for (int part = 0; part < 4; ++part) {
@@ -690,7 +671,7 @@ __global__ void __launch_bounds__(kT, 1) cw_intra_kernel(Problem p) {
         tc_fence_before();
         fence_async_smem();
         __syncthreads();
-        // ---- step 5: dK+ += dA K- ; dK- += dA^T K+
+        // ---- step 4: dK+ += dA K- ; dK- += dA^T K+
         if (ok && threadIdx.x == 0) {
             tc_fence_after();
             mma_tile<64, 128, 64>(tmem + C_KP, op_k_major(sm + DA, 64), op_mn_major(sm + QKM, 128, 64), true);
