@@ -952,11 +952,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_scan_cw_kernel(const __grid_co
 // token-token matrices which use M = 64):
 //   phase 1  (W h)^T ; (K dh')^T          (P = tril(Q K^T . D) comes from tc_prep, which forms it anyway)
 //   phase 2  (P^T dO)^T ; then, under the readout, dO h^T          -> U = U~ - W h ; dU = scale P^T dO + Diag(e) K dh'
-//   phase 3  dO U^T ; -(dU h^T)^T                                  -> dPD = scale tril(dO U^T) . D ; dW
-//   phase 4  (dPD K)^T ; (T^T dW)^T ; (T^T dU)^T ; (dPD^T Q)^T ; (U dh'^T)^T
-//                                                                  -> dq ; dXk ; dXv ; dv ; dw
-//   phase 5  dXk W^T + dXv U~^T ; then, under the readout, T^T dW   -> G = -stril(.) . D ; Diag(b) G
-//   phase 6  G K ; += (Diag(b) G)^T K                               -> dk ; db ; dgamma -> dg
+//   phase 3  dO U^T ; T^T dU                                       -> dPD = scale tril(dO U^T) . D ; dXv ; dv ; dw
+//   phase 4  dXv U^T ; dPD K ; -dXv h^T ; under the readout dPD^T Q ; U dh'^T
+//                                                                  -> G = -stril(dXv U^T) . D ; Diag(b) G ; dq ; (dXk)
+//   phase 5  G K ; += (Diag(b) G)^T K                               -> dk ; db ; dgamma -> dg
+// The vector-Jacobian product of the triangular solve (K#2) is taken in a shorter form than its definition
+// dW = -dU h^T, dXk = T^T dW, dXv = T^T dU, dA = -stril(dXk W^T + dXv U~^T):  T^T dW = -(T^T dU) h^T, so dXk = -dXv h^T,
+// and with it dXk W^T + dXv U~^T = dXv (U~ - W h)^T = dXv U^T.  dW is never formed, dXv follows dU directly (beside dP,
+// not after dW), and the sandwich is one product: a phase, a readout and twelve MMA instructions fewer per chunk-head.
 // The decay gradient uses the identities  rowsum(dP.P) + scale Gam <q, dO h^T> = <q, dq>  and its analogues for
 // k:  dgamma_i = <q_i, dq_i> + <k_i, dk_i^row> - <k_i, dk_i^col>, where dk^row = Diag(b)(G K + Diag(Gam) dXk)
 // collects the terms in which k_i enters with exp(+gamma_i) and dk^col those with exp(-gamma_i); the last row
@@ -978,10 +981,10 @@ constexpr uint32_t UT = PT + 8192;         // U^T [128][64]                     
 constexpr uint32_t DUT = UT + 16384;       // dU^T [128][64]                    16 KB   later staged dq
 constexpr uint32_t SMEM_BYTES = DUT + 16384 + 1024;
 constexpr uint32_t DXV = DO, DPD = PT, GT = DO, BGT = DO + 8192;
-// token-major staging of dq (over dU^T, last read by the early products of phase 4), of dv (in place over V: a thread
-// overwrites exactly the chunk it has just read) and of dk (over G, last read by phase 6).  None of these is read by
-// the late products of phase 4 or rewritten within the trip, and of the loads that run ahead only V targets one of
-// them (after its store has read it), so the asynchronous stores need no wait on the critical path.
+// token-major staging of dq (over dU^T, last read by phase 3), of dv (in place over V: a thread overwrites exactly the
+// chunk it has just read) and of dk (over U^T, last read by the products of phase 4).  None of these is read by a later
+// product or rewritten within the trip, and of the loads that run ahead only V targets one of them (after its store
+// has read it), so the asynchronous stores need no wait on the critical path.
 constexpr uint32_t STG_A = DUT, STG_B = VT, STG_K = UT;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 __host__ __device__ constexpr uint32_t slot(int k) { return 64u * k; }   // eight accumulators of 64 columns
@@ -1037,7 +1040,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     //   g1  W, U~^T              once the second readout is done             needed by phase 1
     //       h, dh', P            once the products of phase 4 are done
     //       Q                    once the readout of phase 4 is done
-    //   do  dO;  g2  T, V        once the products of phase 5 are done       needed from phase 2 / 3 on
+    //   do  dO;  g2  T, V        once the products of the last phase are done  needed from phase 2 / 3 on
     //                            (V goes where dv is staged: its store, or the flush of a ragged tail, must have read it)
     //   k   K                    once the last readout holds its K values    needed by phase 1
     constexpr uint32_t K_BYTES = 16384, G1_BYTES = 16384 + 16384 + 32768 + 32768 + 16384 + 8192, G2_BYTES = 8192 + 16384, DO_BYTES = 16384;
@@ -1110,7 +1113,7 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
                     load_piece(2, nx);
                     load_piece(3, nx);
                 }
-                // phase 6 is done and the last readout holds its K values in registers: K first, the next trip starts with
+                // the last phase is done and its readout holds its K values in registers: K first, the next trip starts with
                 // it; dO, T, V are not needed before its second phase (V goes where dv is staged, so that store must have
                 // read its source)
                 if (!(lok = mbar_wait(&bar_ld2, ph))) break;
@@ -1302,10 +1305,10 @@ __global__ void __launch_bounds__(kIntraThreads + 32, 1) tc_intra_kernel(const _
     // accumulator occupies lanes 0..15 of each quadrant ("group A"); a second one sits in lanes 16..31 of the same
     // columns ("group B", address + 16 lanes), and one tcgen05.ld serves both groups.
     //   columns   group A                               group B
-    //   0..127    U dh'^T (ph 4)                        dP (ph 3, 64 cols) -> dXk (ph 4)
-    //   128..255  (dP.D) K (ph 4) -> dXk again (ph 5)   dXv (ph 4)
-    //   256..383  dW^T (ph 3, all lanes) -> dk^col      -
-    //   384..511  dO h^T (ph 2) -> G K (ph 6)           dA (ph 5, 64 cols)
+    //   0..127    U dh'^T (ph 4)                        dP (ph 3, 64 cols)
+    //   128..255  (dP.D) K (ph 4)                       dXv (ph 3)
+    //   256..383  dk^col: (dP.D)^T Q (ph 4) += (bG)^T K  dXk = -dXv h^T (ph 4; read with dk^col, handed over by shuffle)
+    //   384..511  dO h^T (ph 2) -> G K (ph 5)           dXv U^T (ph 4, 64 cols)
     constexpr uint32_t LB = 16u << 16;
     const bool ga = lane < 16;
     const int tr = q4 * 16 + (lane & 15);   // token row of this lane in token-major accumulators

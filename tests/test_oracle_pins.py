@@ -171,6 +171,20 @@ def test_erase_gate_zero_makes_the_solve_vanish():
     assert np.array_equal(r["chunks"][0]["W"], np.zeros((64, 8)))
 
 
+def test_short_form_of_the_triangular_solve_vjp():
+    """The kernels take K#2 in a shorter form than its definition (dW = -dU h^T, dXk = T^T dW, dXv = T^T dU,
+    dA = -stril(dXk W^T + dXv U~^T)): dXk = -dXv h^T and dA = -stril(dXv U^T) with U = U~ - W h.  Checked here on the
+    intermediates of the chunkwise rung, which follows the definition and is itself pinned to the token-serial oracle."""
+    x = draw(12, [200], H=1, dk=8, dv=6)
+    r = chunked.chain_bwd(x["q"][:, 0], x["k"][:, 0], x["v"][:, 0], x["g"][:, 0], x["b"][:, 0], x["w"][:, 0], x["dO"][:, 0],
+                          x["h0"][0, 0], x["dhT"][0, 0], scale=0.7, keep=True)
+    assert len(r["chunks"]) == 4
+    for f, h in zip(r["chunks"], r["h_c"]):
+        assert np.linalg.norm(f["dXk"]) > 0 and np.linalg.norm(f["dA"]) > 0
+        assert rel(-f["dXv"] @ h.T, f["dXk"]) < 1e-12
+        assert rel(-np.tril(f["dXv"] @ f["U"].T, -1), f["dA"]) < 1e-12
+
+
 # ---- P7: split and packing consistency ----
 def test_split_consistency():
     x = draw(10, [90], H=2, dk=6, dv=5)
